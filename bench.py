@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Benchmark of the two-stage verification path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2] [--impl ours|reference]
+
+A step is one pass of the whole hot path — pyramidsd_verify: stage-1 statistics + finalisation, window
+build, stage-2 statistics + finalisation — over one batch of seeded synthetic logits (the BASELINE
+"batched serving" configuration by default: B=64, V=128256, bf16, K_draft=16, K_qual=8). Metric: verified
+positions per second (a position = one row pair actually verified: all B*K_d stage-1 rows plus the
+stage-2 rows inside each sequence's window). Prints ONE JSON line on rank 0.
+
+`--impl reference` times the CPU oracle (the only reference this method has) on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verified positions/s (two-stage verify, B*K*V logits streamed)"
+UNIT = "positions/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_from_name(name: str):
+    from paper_2510_12966_b200 import workloads
+    cfg = int(name.replace("cfg", ""))
+    return cfg, workloads.CONFIGS[cfg]
+
+
+def positions_per_step(w, out) -> int:
+    """Rows actually verified: every stage-1 row, and stage-2 rows inside each sequence's window."""
+    al_q, nt_q = out["accept_len_q"], out["next_token_q"]
+    n2 = torch.clamp(al_q + (nt_q >= 0).to(torch.int32), max=w.K_q)
+    return int(al_q.numel() * w.K_d + int(n2.sum().item()))
+
+
+def run_ours(args):
+    from paper_2510_12966_b200 import binding, workloads
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the verification path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    binding.load_library()
+    binding.set_stream()
+    cfg, w = workload_from_name(args.workload)
+    es = 2 if w.dtype == "bf16" else 4
+
+    # Each rank owns its own batch of B sequences (weak scaling; sequences are independent, no collective
+    # on the data path). Two distinct rounds alternate so that a step never re-reads a buffer it just used;
+    # one round (788 MB for cfg3) already exceeds the 126 MB L2.
+    n_bufs = 2
+    rounds = [workloads.workload_inputs(cfg, 100 * rank + i, device=dev) for i in range(n_bufs)]
+    outs = [{k: torch.empty(w.B, dtype=torch.int32, device=dev)
+             for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")} for _ in range(n_bufs)]
+    mode, seed = binding.FUZZY, 0
+
+    def step(i):
+        zd, zq, zt, tok = rounds[i % n_bufs]
+        binding.verify(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, seed, 2 * i, out=outs[i % n_bufs])
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = binding.launch_count()
+    binding.kernel_timing_begin()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    ms_rs, n_rs, ms_fin, n_fin = binding.kernel_timing_end()
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop()
+    status = binding.last_status()
+    if status != 0:
+        raise SystemExit(f"bench.py: library status {status}")
+
+    # positions and algorithmic bytes of the steps that were timed
+    pos_by_buf = [positions_per_step(w, o) for o in outs]
+    n_pos = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(args.steps))
+    row_bytes = 2 * w.V * es
+    rs_bytes = n_pos * row_bytes   # the statistics kernel streams each verified row pair once
+
+    # ---- end to end through the host-pointer entry point: H2D of the step's inputs + D2H of its results ----
+    e2e = None
+    if not args.no_e2e:
+        zd, zq, zt, tok = [t.cpu().pin_memory() for t in rounds[0]]
+        hout = {k: torch.empty(w.B, dtype=torch.int32).pin_memory()
+                for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+        h2d = sum(t.numel() * t.element_size() for t in (zd, zq, zt, tok))
+        d2h = 4 * w.B * 4
+        e2e_steps = max(2, min(args.steps, 8))
+        for _ in range(2):
+            binding.verify_host(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, seed, 0, out=hout)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(e2e_steps):
+            binding.verify_host(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, seed, 0, out=hout)
+        e1.record()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1)
+        e2e_pos = pos_by_buf[0] * e2e_steps
+        e2e = {"ms": ms_e2e, "pos": e2e_pos, "h2d": h2d, "d2h": d2h, "steps": e2e_steps}
+
+    # ---- max over ranks, sum of positions ----
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e_max = t[0].item(), t[1].item()
+        c = torch.tensor([n_pos, e2e["pos"] if e2e else 0, launches], device=dev, dtype=torch.int64)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        n_pos_all, e2e_pos_all, launches_all = int(c[0]), int(c[1]), int(c[2])
+        if e2e:
+            e2e["ms"] = ms_e2e_max
+    else:
+        n_pos_all, e2e_pos_all, launches_all = n_pos, (e2e["pos"] if e2e else 0), launches
+
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        value = n_pos_all / (ms_total * 1e-3)
+        achieved = rs_bytes / (ms_rs * 1e-3) / 1e9 if ms_rs > 0 else 0.0
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{w.name}: B={w.B} per GPU, V={w.V}, {w.dtype} logits, K_draft={w.K_d}, "
+                                   f"K_qual={w.K_q}, tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0",
+                       "logits_dtype": w.dtype, "positions_per_step": n_pos / args.steps,
+                       "l2_policy": "inputs larger than L2 (one round = %.0f MB), two rounds alternate" %
+                                    ((2 * w.K_d + w.K_q) * w.B * w.V * es / 1e6),
+                       "gb_per_s_whole_step": n_pos_all * row_bytes / (ms_total * 1e-3) / 1e9},
+            "roofline": {"bound": "hbm", "kernel": "rowstats (per-row softmax/divergence statistics)",
+                         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
+                         "traffic": None, "launches": n_rs, "avg_launch_ms": ms_rs / max(n_rs, 1),
+                         "finalize_ms_per_launch": ms_fin / max(n_fin, 1),
+                         "share_of_step": (ms_rs / ms_total) if ms_total > 0 else None},
+            "gpu_launches": launches_all, "clocks": clocks,
+        }
+        if e2e:
+            line["e2e"] = {"value": e2e_pos_all / (e2e["ms"] * 1e-3), "unit": UNIT,
+                           "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                           "ms_per_step": e2e["ms"] / e2e["steps"], "steps": e2e["steps"]}
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w, cfg, rounds[0], seqs=args.cpu_seqs)
+        line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
+        traffic = read_profile_traffic(w)
+        if traffic is not None:
+            line["roofline"]["traffic"] = traffic
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def read_profile_traffic(w):
+    """DRAM bytes per full-size rowstats launch from the committed ncu summary, if present."""
+    path = os.path.join(ROOT, "profiles", "rowstats_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        t = json.load(f)
+    per_row = t.get("dram_bytes_per_row", {}).get(f"V{w.V}_{w.dtype}")
+    return None if per_row is None else per_row * w.B * w.K_d
+
+
+def cpu_baseline(w, cfg, round_inputs, seqs):
+    """The CPU oracle, as it stands, on a bounded sample (the first `seqs` sequences of one round)."""
+    import oracle
+    from paper_2510_12966_b200 import workloads
+    oracle.build()
+    zd, zq, zt, tok = [workloads.to_host_bits(t[:seqs]) for t in round_inputs]
+    cores = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, n_threads=cores)
+    dt = time.perf_counter() - t0
+    n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
+    pos = seqs * w.K_d + int(n2.sum())
+    return {"value": pos / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {seqs} sequences of one {w.name} round ({pos} positions, {dt:.2f} s wall)"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle timed on the host cores (this method has no other reference)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2510_12966_b200 import workloads
+    oracle.build()
+    cfg, w = workload_from_name(args.workload)
+    seqs = args.cpu_seqs
+    cores = os.cpu_count() or 1
+    rounds = [workloads.workload_inputs(cfg, i, device="cpu", B=seqs) for i in range(2)]
+    hosts = [[workloads.to_host_bits(t) for t in r] for r in rounds]
+
+    def step(i):
+        zd, zq, zt, tok = hosts[i % 2]
+        out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 2 * i,
+                            n_threads=cores)
+        n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
+        return seqs * w.K_d + int(n2.sum())
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    pos = sum(step(args.warmup + i) for i in range(args.steps))
+    dt = time.perf_counter() - t0
+    value = pos / dt
+    sample = f"{seqs} sequences per step of {w.name} (B={w.B} in the full workload), {cores} threads"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: V={w.V}, {w.dtype} logits, K_draft={w.K_d}, K_qual={w.K_q}, "
+                               f"tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0; {sample}"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences in the CPU-oracle sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

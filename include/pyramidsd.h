@@ -1,0 +1,184 @@
+/* pyramidsd.h — C ABI of the B200 (sm_100a) two-stage verification library for Pyramid Speculative
+ * Decoding ("3-Model Speculative Decoding").
+ *
+ * What the calls compute, per (sequence b, speculative position k) row r = b*K + k, for a "small" and a
+ * "large" model (draft/qualifier in stage 1, qualifier/target in stage 2 — Fig. 1 and Sec. 3.2):
+ *   1. softmax of both models' full-vocabulary logits (Sec. 3.1: P_M is the next-token distribution);
+ *   2. the divergence Div(P_large, P_small) of Sec. 3.1 — Jensen-Shannon in nats by default;
+ *   3. acceptance: fuzzy mode accepts when Div <= threshold (Sec. 3.1, two-stage criterion of Sec. 3.2);
+ *      strict mode is standard speculative sampling, u < min(1, p_large(x)/p_small(x)) (Sec. 3.1-3.2);
+ *   4. per sequence, the length of the accepted prefix (Sec. 1: fall back to the larger model at the
+ *      first disagreement);
+ *   5. at the first rejection, a token drawn from the normalised residual max(0, p_large - p_small)
+ *      ("standard SD probability rule", Sec. 3.4) by inverse CDF in vocabulary order, or from p_large
+ *      itself in the assisted variant (Sec. 3.4).
+ * Random numbers: one Philox4x32-10 block per row, counter (r, 0, offset_lo, offset_hi), key
+ * (seed_lo, seed_hi); u = (word0 >> 8) * 2^-24 decides the strict coin flip, u' = (word1 >> 8) * 2^-24
+ * drives the inverse CDF. The two-stage wrapper uses `offset` for stage 1 and `offset + 1` for stage 2.
+ *
+ * Conventions shared by every entry point unless stated otherwise:
+ *   - All data pointers are DEVICE pointers owned by the caller; the library never frees or keeps them.
+ *   - Logits are row-major [B, K, V], dtype float32 or bfloat16. Rows whose base address is 16-byte
+ *     aligned with V * sizeof(element) a multiple of 16 take the vector path; other shapes take a
+ *     scalar path — never an error. -inf logits are legal (probability 0). A row holding NaN or +inf,
+ *     or no finite entry, or a token outside [0, V), is flagged and rejected; a flagged non-finite row
+ *     at the first rejection emits token -2.
+ *   - out_accept_len[b] in [0, n_valid[b]]; out_next_token[b] = resampled token at the first rejection,
+ *     or -1 when every valid position was accepted.
+ *   - Work is enqueued on the stream set by pyramidsd_set_stream (default: the legacy default stream)
+ *     or given in the argument struct; calls return without synchronising. Scratch memory comes from
+ *     the caller's workspace when one is supplied (pyramidsd_workspace_bytes), otherwise from a
+ *     library-owned per-device buffer that is grown with cudaMalloc on first use (that growth
+ *     synchronises the device once).
+ *   - Return value: PSD_OK or a negative psd_status. Arguments are validated on the host before any
+ *     launch; nothing is launched on error. Device-side bounded waits that give up report
+ *     PSD_ERR_TIMEOUT through pyramidsd_last_status().
+ */
+#ifndef PYRAMIDSD_H_
+#define PYRAMIDSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { PSD_F32 = 0, PSD_BF16 = 1 } psd_dtype;
+
+typedef enum {
+  PSD_FUZZY = 0,             /* accept iff Div <= threshold (Sec. 3.1, 3.2) */
+  PSD_STRICT = 1,            /* standard speculative sampling (Sec. 3.1 "standard SD", tau = 0 end) */
+  PSD_FUZZY_SD_FALLBACK = 2, /* Div <= threshold OR the strict coin flip succeeds */
+  PSD_ASSISTED = 3           /* strict acceptance; on rejection draw from p_large itself (Sec. 3.4) */
+} psd_mode;
+
+typedef enum { PSD_DIV_JS = 0, PSD_DIV_TV = 1, PSD_DIV_KL = 2 } psd_div_kind;
+
+typedef enum {
+  PSD_OK = 0,
+  PSD_ERR_INVALID_ARG = -1,
+  PSD_ERR_UNSUPPORTED = -2,
+  PSD_ERR_WORKSPACE = -3,
+  PSD_ERR_CUDA = -4,
+  PSD_ERR_TIMEOUT = -5
+} psd_status;
+
+/* Per-row flag bits written to out_row_flags. */
+#define PSD_FLAG_SMALL_NONFINITE 1
+#define PSD_FLAG_LARGE_NONFINITE 2
+#define PSD_FLAG_TOKEN_RANGE 4
+
+/* Kernel selection for the per-row statistics pass. AUTO picks the fastest variant the shape allows. */
+typedef enum {
+  PSD_KERNEL_AUTO = 0,
+  PSD_KERNEL_BASELINE = 1, /* one CTA per row, three passes over global memory */
+  PSD_KERNEL_CLUSTER = 2   /* one thread-block cluster per row, row pair resident in shared memory */
+} psd_kernel_variant;
+
+/* Extended single-stage arguments. Zero-initialise, set struct_size = sizeof(psd_stage_args), fill what
+ * you need; every optional field left zero means "off"/default. */
+typedef struct psd_stage_args {
+  uint32_t struct_size;
+  int32_t dtype;                 /* psd_dtype */
+  const void* logits_small;      /* [B, K, V] device */
+  const void* logits_large;      /* [B, K, V] device */
+  const int32_t* tokens;         /* [B, K] device, each in [0, V) */
+  int32_t B, K, V;
+  int32_t mode;                  /* psd_mode */
+  int32_t div_kind;              /* psd_div_kind */
+  float threshold;
+  float inv_temperature;         /* logits are multiplied by this before the softmax; 0 means 1 (Sec. 4.1 uses T = 0.7) */
+  int64_t seq_stride_small;      /* elements between sequences; 0 means K * V. Rows inside a sequence are V apart. */
+  int64_t seq_stride_large;
+  uint64_t philox_seed, philox_offset;
+  const int32_t* n_valid;        /* [B] device or NULL: only positions k < n_valid[b] take part */
+  int32_t* out_accept_len;       /* [B] device, required */
+  int32_t* out_next_token;       /* [B] device, required */
+  float* out_div;                /* [B, K] device or NULL */
+  float* out_p_small_tok;        /* [B, K] device or NULL */
+  float* out_p_large_tok;        /* [B, K] device or NULL */
+  float* out_resid_mass;         /* [B, K] device or NULL */
+  int32_t* out_row_flags;        /* [B, K] device or NULL */
+  void* workspace;               /* device, >= pyramidsd_workspace_bytes(B, K, V, dtype), 256-byte aligned; NULL = library-owned */
+  size_t workspace_bytes;
+  void* stream;                  /* cudaStream_t, or NULL for the stream set by pyramidsd_set_stream */
+  int32_t use_stream_field;      /* non-zero: take `stream` even when it is NULL (the legacy default stream) */
+  int32_t kernel_variant;        /* psd_kernel_variant */
+} psd_stage_args;
+
+/* One verification stage (Sec. 3.1 for one model pair; Sec. 3.2 applies it twice). Jensen-Shannon
+ * divergence, temperature 1, all K positions valid. Device pointers. Asynchronous on the library stream. */
+int pyramidsd_verify_stage(const void* logits_small, const void* logits_large, const int32_t* draft_tokens,
+                           int B, int K, int V, psd_dtype dtype, float threshold, psd_mode mode,
+                           uint64_t philox_seed, uint64_t offset,
+                           int32_t* out_accept_len, int32_t* out_next_token);
+
+/* Same stage with every option exposed (strides, n_valid, temperature, divergence kind, per-row outputs,
+ * caller workspace, stream, kernel variant). Returns PSD_ERR_INVALID_ARG on a NULL required pointer,
+ * non-positive V, negative B/K, K > 32, an unknown enum value or a wrong struct_size; PSD_ERR_WORKSPACE
+ * when a supplied workspace is too small or misaligned. B == 0 or K == 0 is a valid empty call. */
+int pyramidsd_verify_stage_ex(const psd_stage_args* args);
+
+/* Two-stage pyramid (Fig. 1, Sec. 3.2): stage 1 verifies the K_d draft tokens against the qualifier
+ * with tau_q; the accepted prefix followed by the qualifier's correction token forms the window, cut to
+ * K_q tokens; stage 2 verifies the window against the target with tau_t, with the qualifier's
+ * distribution (rows 0..K_q-1 of each sequence of logits_qual) as the small model. Requires
+ * 1 <= K_q <= K_d <= 32. logits_draft and logits_qual are [B, K_d, V], logits_target is [B, K_q, V].
+ * Stage-1 results go to out_accept_len_q / out_next_token_q, final results to out_accept_len /
+ * out_next_token (all [B], device). Consumes Philox offsets `offset` and `offset + 1`. */
+int pyramidsd_verify(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                     const int32_t* draft_tokens, int B, int K_d, int K_q, int V, psd_dtype dtype,
+                     float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
+                     int32_t* out_accept_len_q, int32_t* out_next_token_q,
+                     int32_t* out_accept_len, int32_t* out_next_token);
+
+/* pyramidsd_verify with HOST pointers for every array: copies the three logits tensors and the tokens
+ * to library-owned device staging buffers, runs both stages, copies the four [B] results back and
+ * synchronises the stream before returning. For callers whose logits live in host memory; the copies
+ * are part of the call. Pinned host memory makes the copies asynchronous up to the final sync. */
+int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                          const int32_t* draft_tokens, int B, int K_d, int K_q, int V, psd_dtype dtype,
+                          float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
+                          int32_t* out_accept_len_q, int32_t* out_next_token_q,
+                          int32_t* out_accept_len, int32_t* out_next_token);
+
+/* The Philox uniforms the verification draws for rows 0..n_rows-1 with this seed and offset (see the
+ * header comment for the counter layout): out_u[r] decides the strict coin flip of row r, out_u2[r]
+ * drives its inverse CDF. Device pointers, float32 [n_rows]; either may be NULL. Lets a caller replay
+ * or audit the random choices of a call. */
+int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, float* out_u, float* out_u2);
+
+/* Scratch bytes one stage call of this shape needs (per-row statistics and the stage-2 window of the
+ * wrapper). Pure host arithmetic; 0 on invalid arguments. */
+size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype);
+
+/* Stream used by the entry points that carry no stream argument (a cudaStream_t; NULL = legacy default
+ * stream). Per host thread. */
+int pyramidsd_set_stream(void* cuda_stream);
+
+/* Synchronises the library stream and returns PSD_OK, PSD_ERR_TIMEOUT if a device-side bounded wait gave
+ * up since the last call, or PSD_ERR_CUDA if the stream reports an error. Clears the status word. */
+int pyramidsd_last_status(void);
+
+/* Per-kernel device timing for benchmarks. Between _begin and _end the library brackets each of its
+ * kernel launches (on the calling thread) with CUDA events on the launch stream, up to 4096 launches.
+ * _end synchronises those events, switches timing off, and returns the summed milliseconds and launch
+ * counts of the row-statistics kernel and of the finalisation kernel (any output may be NULL). */
+int pyramidsd_kernel_timing_begin(void);
+int pyramidsd_kernel_timing_end(double* ms_rowstats, int* n_rowstats, double* ms_finalize, int* n_finalize);
+
+/* Number of kernels the library has launched from this process since load (all entry points). */
+uint64_t pyramidsd_launch_count(void);
+
+/* Largest number of co-resident clusters the device grants the cluster kernel for this shape (0 when
+ * the variant does not apply); lets a caller size batches to whole waves. */
+int pyramidsd_cluster_occupancy(int V, psd_dtype dtype, int* out_cluster_size, int* out_max_active_clusters);
+
+const char* pyramidsd_version(void);
+const char* pyramidsd_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PYRAMIDSD_H_ */

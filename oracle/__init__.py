@@ -102,14 +102,18 @@ def prefix_length(accept, n_valid: int) -> int:
 
 
 def verify_stage(logits_small, logits_large, tokens, tau, mode=FUZZY, seed=0, offset=0, n_valid=None,
-                 inv_temperature=1.0, div_kind=JS, n_threads=1):
-    """One verification stage on host arrays shaped [B, K, V] (tokens [B, K]). Returns a dict."""
+                 inv_temperature=1.0, div_kind=JS, n_threads=1, seq_ids=None):
+    """One verification stage on host arrays shaped [B, K, V] (tokens [B, K]). Returns a dict.
+
+    ``seq_ids`` (optional, [B]) gives each sequence's index in the full batch when the arrays are a
+    sample of it, so that row (b, k) draws the Philox block of row ``seq_ids[b] * K + k``."""
     s, dt = _as_logits(logits_small)
     l, dt2 = _as_logits(logits_large)
     assert dt == dt2 and s.shape == l.shape and s.ndim == 3
     B, K, V = s.shape
     t = np.ascontiguousarray(tokens, dtype=np.int32).reshape(B, K)
     nv = None if n_valid is None else np.ascontiguousarray(n_valid, dtype=np.int32)
+    ids = None if seq_ids is None else np.ascontiguousarray(seq_ids, dtype=np.int32)
     out = {
         "accept_len": np.zeros(B, np.int32), "next_token": np.zeros(B, np.int32),
         "div": np.zeros((B, K)), "p_small_tok": np.zeros((B, K)), "p_large_tok": np.zeros((B, K)),
@@ -119,7 +123,7 @@ def verify_stage(logits_small, logits_large, tokens, tau, mode=FUZZY, seed=0, of
     rc = lib().psd_oracle_verify_stage(
         _ptr(s), _ptr(l), _ptr(t), B, K, V, dt, C.c_int64(V), C.c_int64(V),
         C.c_double(float(tau)), int(mode), C.c_uint64(seed), C.c_uint64(offset), _ptr(nv),
-        C.c_double(inv_temperature), int(div_kind),
+        C.c_double(inv_temperature), int(div_kind), _ptr(ids),
         _ptr(out["accept_len"]), _ptr(out["next_token"]), _ptr(out["div"]), _ptr(out["p_small_tok"]),
         _ptr(out["p_large_tok"]), _ptr(out["resid_mass"]), _ptr(out["row_flags"]), _ptr(out["accept_bits"]),
         int(n_threads))
@@ -129,7 +133,7 @@ def verify_stage(logits_small, logits_large, tokens, tau, mode=FUZZY, seed=0, of
 
 
 def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode=FUZZY, seed=0, offset=0,
-           inv_temperature=1.0, div_kind=JS, n_threads=1):
+           inv_temperature=1.0, div_kind=JS, n_threads=1, seq_ids=None):
     """Two-stage pyramid on host arrays: draft/qual [B, K_d, V], target [B, K_q, V]."""
     d, dt = _as_logits(logits_draft)
     q, dtq = _as_logits(logits_qual)
@@ -138,6 +142,7 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
     B, K_d, V = d.shape
     K_q = t.shape[1]
     tok = np.ascontiguousarray(draft_tokens, dtype=np.int32).reshape(B, K_d)
+    ids = None if seq_ids is None else np.ascontiguousarray(seq_ids, dtype=np.int32)
     out = {
         "accept_len_q": np.zeros(B, np.int32), "next_token_q": np.zeros(B, np.int32),
         "accept_len": np.zeros(B, np.int32), "next_token": np.zeros(B, np.int32),
@@ -147,7 +152,7 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
     rc = lib().psd_oracle_verify(
         _ptr(d), _ptr(q), _ptr(t), _ptr(tok), B, K_d, K_q, V, dt,
         C.c_double(float(tau_q)), C.c_double(float(tau_t)), int(mode), C.c_uint64(seed), C.c_uint64(offset),
-        C.c_double(inv_temperature), int(div_kind),
+        C.c_double(inv_temperature), int(div_kind), _ptr(ids),
         _ptr(out["accept_len_q"]), _ptr(out["next_token_q"]), _ptr(out["accept_len"]), _ptr(out["next_token"]),
         _ptr(out["window"]), _ptr(out["n_window"]), _ptr(out["div_q"]), _ptr(out["div_t"]), int(n_threads))
     if rc:

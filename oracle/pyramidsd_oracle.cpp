@@ -159,6 +159,7 @@ struct StageArgs {
   int64_t stride_small, stride_large;  // elements between consecutive rows
   double tau; int mode; uint64_t seed, offset;
   const int32_t* n_valid; double inv_temperature; int div_kind;
+  const int32_t* seq_ids;  // optional: global sequence index of each local sequence (for the Philox counter)
 };
 
 // Steps for one (sequence, position) row: softmaxes, divergence, residual mass, token probabilities,
@@ -170,7 +171,10 @@ void verify_row(const StageArgs& a, int r, RowResult& out) {
   const int x = a.tokens[r];
   out.flags = (ok_q ? 0 : FLAG_SMALL_NONFINITE) | (ok_p ? 0 : FLAG_LARGE_NONFINITE) |
               ((x < 0 || x >= a.V) ? FLAG_TOKEN_RANGE : 0);
-  row_uniforms(a.seed, a.offset, (uint32_t)r, &out.u, &out.u2);
+  // Philox counter word 0 is the row index b*K + k of the sequence's position in the full batch
+  const int b_local = r / a.K, k_local = r % a.K;
+  const uint32_t r_global = (uint32_t)((a.seq_ids ? a.seq_ids[b_local] : b_local) * a.K + k_local);
+  row_uniforms(a.seed, a.offset, r_global, &out.u, &out.u2);
   const double nan = std::numeric_limits<double>::quiet_NaN();
   out.D = nan; out.R = nan; out.p_small_tok = nan; out.p_large_tok = nan;
   out.accept = 0; out.resample = -2;
@@ -299,13 +303,14 @@ int psd_oracle_verify_stage(const void* logits_small, const void* logits_large, 
                             int B, int K, int V, int dtype, int64_t stride_small, int64_t stride_large,
                             double tau, int mode, uint64_t seed, uint64_t offset,
                             const int32_t* n_valid, double inv_temperature, int div_kind,
+                            const int32_t* seq_ids,
                             int32_t* out_accept_len, int32_t* out_next_token,
                             double* out_div, double* out_p_small_tok, double* out_p_large_tok,
                             double* out_resid_mass, int32_t* out_row_flags, int32_t* out_accept_bits,
                             int n_threads) {
   StageArgs a{logits_small, logits_large, tokens, B, K, V, dtype,
               stride_small ? stride_small : V, stride_large ? stride_large : V,
-              tau, mode, seed, offset, n_valid, inv_temperature, div_kind};
+              tau, mode, seed, offset, n_valid, inv_temperature, div_kind, seq_ids};
   return verify_stage_impl(a, out_accept_len, out_next_token, out_div, out_p_small_tok, out_p_large_tok,
                            out_resid_mass, out_row_flags, out_accept_bits, n_threads);
 }
@@ -317,7 +322,7 @@ int psd_oracle_verify_stage(const void* logits_small, const void* logits_large, 
 int psd_oracle_verify(const void* logits_draft, const void* logits_qual, const void* logits_target,
                       const int32_t* draft_tokens, int B, int K_d, int K_q, int V, int dtype,
                       double tau_q, double tau_t, int mode, uint64_t seed, uint64_t offset,
-                      double inv_temperature, int div_kind,
+                      double inv_temperature, int div_kind, const int32_t* seq_ids,
                       int32_t* out_accept_len_q, int32_t* out_next_token_q,
                       int32_t* out_accept_len, int32_t* out_next_token,
                       int32_t* out_window /* [B,K_q] or null */, int32_t* out_n_window /* [B] or null */,
@@ -325,7 +330,7 @@ int psd_oracle_verify(const void* logits_draft, const void* logits_qual, const v
                       int n_threads) {
   if (K_q > K_d || K_q < 0) return -1;
   StageArgs s1{logits_draft, logits_qual, draft_tokens, B, K_d, V, dtype, V, V,
-               tau_q, mode, seed, offset, nullptr, inv_temperature, div_kind};
+               tau_q, mode, seed, offset, nullptr, inv_temperature, div_kind, seq_ids};
   int rc = verify_stage_impl(s1, out_accept_len_q, out_next_token_q, out_div_q, nullptr, nullptr, nullptr,
                              nullptr, nullptr, n_threads);
   if (rc) return rc;
@@ -347,7 +352,7 @@ int psd_oracle_verify(const void* logits_draft, const void* logits_qual, const v
     std::memcpy(qual_view.data() + (size_t)b * K_q * V * es,
                 (const unsigned char*)logits_qual + (size_t)b * K_d * V * es, (size_t)K_q * V * es);
   StageArgs s2{qual_view.data(), logits_target, window.data(), B, K_q, V, dtype, V, V,
-               tau_t, mode, seed, offset + 1, n2.data(), inv_temperature, div_kind};
+               tau_t, mode, seed, offset + 1, n2.data(), inv_temperature, div_kind, seq_ids};
   rc = verify_stage_impl(s2, out_accept_len, out_next_token, out_div_t, nullptr, nullptr, nullptr,
                          nullptr, nullptr, n_threads);
   if (out_window) std::memcpy(out_window, window.data(), window.size() * sizeof(int32_t));
@@ -387,7 +392,7 @@ int psd_oracle_verify_stage_mixed(const void* logits_small, int dtype_small, con
   const size_t n = (size_t)B * K * V;
   std::vector<double> s(n), l(n);
   for (size_t i = 0; i < n; ++i) { s[i] = logit_at(logits_small, dtype_small, i); l[i] = logit_at(logits_large, dtype_large, i); }
-  StageArgs a{s.data(), l.data(), tokens, B, K, V, DT_F64, V, V, tau, mode, seed, offset, nullptr, 1.0, div_kind};
+  StageArgs a{s.data(), l.data(), tokens, B, K, V, DT_F64, V, V, tau, mode, seed, offset, nullptr, 1.0, div_kind, nullptr};
   return verify_stage_impl(a, out_accept_len, out_next_token, out_div, nullptr, nullptr, out_resid_mass,
                            nullptr, nullptr, n_threads);
 }

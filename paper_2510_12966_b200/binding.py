@@ -1,0 +1,288 @@
+"""Thin ctypes binding over the C ABI declared in ``include/pyramidsd.h``.
+
+Argument marshalling only: every function takes torch tensors (device memory) or plain ints/floats,
+checks dtype / contiguity, and passes raw pointers to the entry point of the same name. There is no
+Python or CPU implementation behind these calls; if the shared library is missing they raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+from .build import LIB_PATH
+
+F32, BF16 = 0, 1
+FUZZY, STRICT, FUZZY_SD_FALLBACK, ASSISTED = 0, 1, 2, 3
+DIV_JS, DIV_TV, DIV_KL = 0, 1, 2
+KERNEL_AUTO, KERNEL_BASELINE, KERNEL_CLUSTER = 0, 1, 2
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+
+EXPORTS = (
+    "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_host",
+    "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
+    "pyramidsd_kernel_timing_begin", "pyramidsd_kernel_timing_end",
+    "pyramidsd_cluster_occupancy", "pyramidsd_version", "pyramidsd_status_string",
+)
+
+
+class StageArgs(C.Structure):
+    """Mirror of ``psd_stage_args``."""
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("dtype", C.c_int32),
+        ("logits_small", C.c_void_p), ("logits_large", C.c_void_p), ("tokens", C.c_void_p),
+        ("B", C.c_int32), ("K", C.c_int32), ("V", C.c_int32),
+        ("mode", C.c_int32), ("div_kind", C.c_int32),
+        ("threshold", C.c_float), ("inv_temperature", C.c_float),
+        ("seq_stride_small", C.c_int64), ("seq_stride_large", C.c_int64),
+        ("philox_seed", C.c_uint64), ("philox_offset", C.c_uint64),
+        ("n_valid", C.c_void_p),
+        ("out_accept_len", C.c_void_p), ("out_next_token", C.c_void_p),
+        ("out_div", C.c_void_p), ("out_p_small_tok", C.c_void_p), ("out_p_large_tok", C.c_void_p),
+        ("out_resid_mass", C.c_void_p), ("out_row_flags", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("stream", C.c_void_p), ("use_stream_field", C.c_int32), ("kernel_variant", C.c_int32),
+    ]
+
+
+class PyramidSDError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None):
+    """dlopen the in-tree shared library (no build, no fallback)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise ImportError(f"{p} is missing: build it with `python -m paper_2510_12966_b200.build` "
+                          "(there is no CPU fallback for the verification path)")
+    lib = C.CDLL(p)
+    i32, u64, f32, vp = C.c_int, C.c_uint64, C.c_float, C.c_void_p
+    lib.pyramidsd_verify_stage.argtypes = [vp, vp, vp, i32, i32, i32, i32, f32, i32, u64, u64, vp, vp]
+    lib.pyramidsd_verify_stage.restype = i32
+    lib.pyramidsd_verify_stage_ex.argtypes = [C.POINTER(StageArgs)]
+    lib.pyramidsd_verify_stage_ex.restype = i32
+    pyr = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, u64, u64, vp, vp, vp, vp]
+    lib.pyramidsd_verify.argtypes = pyr
+    lib.pyramidsd_verify.restype = i32
+    lib.pyramidsd_verify_host.argtypes = pyr
+    lib.pyramidsd_verify_host.restype = i32
+    lib.pyramidsd_row_uniforms.argtypes = [u64, u64, i32, vp, vp]
+    lib.pyramidsd_row_uniforms.restype = i32
+    lib.pyramidsd_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    lib.pyramidsd_workspace_bytes.restype = C.c_size_t
+    lib.pyramidsd_set_stream.argtypes = [vp]
+    lib.pyramidsd_set_stream.restype = i32
+    lib.pyramidsd_last_status.argtypes = []
+    lib.pyramidsd_last_status.restype = i32
+    lib.pyramidsd_kernel_timing_begin.argtypes = []
+    lib.pyramidsd_kernel_timing_begin.restype = i32
+    lib.pyramidsd_kernel_timing_end.argtypes = [C.POINTER(C.c_double), C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i32)]
+    lib.pyramidsd_kernel_timing_end.restype = i32
+    lib.pyramidsd_launch_count.argtypes = []
+    lib.pyramidsd_launch_count.restype = u64
+    lib.pyramidsd_cluster_occupancy.argtypes = [i32, i32, C.POINTER(i32), C.POINTER(i32)]
+    lib.pyramidsd_cluster_occupancy.restype = i32
+    lib.pyramidsd_version.restype = C.c_char_p
+    lib.pyramidsd_status_string.argtypes = [i32]
+    lib.pyramidsd_status_string.restype = C.c_char_p
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().pyramidsd_status_string(int(status)).decode()
+
+
+def version() -> str:
+    return load_library().pyramidsd_version().decode()
+
+
+def _check(rc: int, where: str):
+    if rc != OK:
+        raise PyramidSDError(rc, where)
+
+
+def dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"logits dtype {t.dtype}: want float32 or bfloat16")
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must live in device memory")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def set_stream(stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Use ``stream`` (default: torch's current stream) for the entry points without a stream argument."""
+    s = torch.cuda.current_stream() if stream is None else stream
+    _check(load_library().pyramidsd_set_stream(C.c_void_p(s.cuda_stream)), "pyramidsd_set_stream")
+
+
+def last_status() -> int:
+    return load_library().pyramidsd_last_status()
+
+
+def launch_count() -> int:
+    return int(load_library().pyramidsd_launch_count())
+
+
+def kernel_timing_begin() -> None:
+    _check(load_library().pyramidsd_kernel_timing_begin(), "pyramidsd_kernel_timing_begin")
+
+
+def kernel_timing_end():
+    """Returns (ms_rowstats, n_rowstats, ms_finalize, n_finalize) accumulated since kernel_timing_begin()."""
+    a, b, c, d = C.c_double(0), C.c_int(0), C.c_double(0), C.c_int(0)
+    _check(load_library().pyramidsd_kernel_timing_end(C.byref(a), C.byref(b), C.byref(c), C.byref(d)),
+           "pyramidsd_kernel_timing_end")
+    return a.value, b.value, c.value, d.value
+
+
+def workspace_bytes(B: int, K: int, V: int, dtype: int) -> int:
+    return int(load_library().pyramidsd_workspace_bytes(B, K, V, dtype))
+
+
+def cluster_occupancy(V: int, dtype: int):
+    cs, n = C.c_int(0), C.c_int(0)
+    _check(load_library().pyramidsd_cluster_occupancy(V, dtype, C.byref(cs), C.byref(n)), "pyramidsd_cluster_occupancy")
+    return cs.value, n.value
+
+
+def row_uniforms(philox_seed: int, offset: int, n_rows: int, device="cuda"):
+    """``pyramidsd_row_uniforms``: the (u, u2) pair of every row as two float32 device tensors."""
+    u = torch.empty(n_rows, dtype=torch.float32, device=device)
+    u2 = torch.empty(n_rows, dtype=torch.float32, device=device)
+    _check(load_library().pyramidsd_row_uniforms(int(philox_seed), int(offset), n_rows, u.data_ptr(), u2.data_ptr()),
+           "pyramidsd_row_uniforms")
+    return u, u2
+
+
+def verify_stage(logits_small, logits_large, draft_tokens, threshold, mode=FUZZY, philox_seed=0, offset=0,
+                 out_accept_len=None, out_next_token=None):
+    """``pyramidsd_verify_stage`` on [B, K, V] device tensors; returns (accept_len [B], next_token [B])."""
+    B, K, V = logits_small.shape
+    dt = dtype_code(logits_small)
+    assert logits_large.shape == logits_small.shape and logits_large.dtype == logits_small.dtype
+    dev = logits_small.device
+    if out_accept_len is None:
+        out_accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+    if out_next_token is None:
+        out_next_token = torch.empty(B, dtype=torch.int32, device=dev)
+    rc = load_library().pyramidsd_verify_stage(
+        _dev_ptr(logits_small, name="logits_small"), _dev_ptr(logits_large, name="logits_large"),
+        _dev_ptr(draft_tokens, torch.int32, "draft_tokens"), B, K, V, dt, float(threshold), int(mode),
+        int(philox_seed), int(offset), _dev_ptr(out_accept_len, torch.int32), _dev_ptr(out_next_token, torch.int32))
+    _check(rc, "pyramidsd_verify_stage")
+    return out_accept_len, out_next_token
+
+
+def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
+                    B=None, K=None, V=None, n_valid=None, inv_temperature=0.0, div_kind=DIV_JS,
+                    seq_stride_small=0, seq_stride_large=0, want_rows=True, workspace=None, stream=None,
+                    kernel_variant=KERNEL_AUTO, raise_on_error=True):
+    """``pyramidsd_verify_stage_ex``: every option exposed. Returns a dict of device tensors (+ "status")."""
+    if B is None:
+        B, K, V = logits_small.shape
+    dt = dtype_code(logits_small)
+    dev = logits_small.device
+    out = {"accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+           "next_token": torch.empty(B, dtype=torch.int32, device=dev)}
+    if want_rows:
+        for k in ("div", "p_small_tok", "p_large_tok", "resid_mass"):
+            out[k] = torch.empty((B, K), dtype=torch.float32, device=dev)
+        out["row_flags"] = torch.empty((B, K), dtype=torch.int32, device=dev)
+    a = StageArgs()
+    a.struct_size = C.sizeof(StageArgs)
+    a.dtype = dt
+    a.logits_small = logits_small.data_ptr()
+    a.logits_large = logits_large.data_ptr()
+    a.tokens = _dev_ptr(tokens, torch.int32, "tokens")
+    a.B, a.K, a.V = B, K, V
+    a.mode, a.div_kind = int(mode), int(div_kind)
+    a.threshold, a.inv_temperature = float(threshold), float(inv_temperature)
+    a.seq_stride_small, a.seq_stride_large = int(seq_stride_small), int(seq_stride_large)
+    a.philox_seed, a.philox_offset = int(philox_seed), int(offset)
+    a.n_valid = _dev_ptr(n_valid, torch.int32, "n_valid")
+    a.out_accept_len = out["accept_len"].data_ptr()
+    a.out_next_token = out["next_token"].data_ptr()
+    if want_rows:
+        a.out_div = out["div"].data_ptr()
+        a.out_p_small_tok = out["p_small_tok"].data_ptr()
+        a.out_p_large_tok = out["p_large_tok"].data_ptr()
+        a.out_resid_mass = out["resid_mass"].data_ptr()
+        a.out_row_flags = out["row_flags"].data_ptr()
+    if workspace is not None:
+        a.workspace = workspace.data_ptr()
+        a.workspace_bytes = workspace.numel() * workspace.element_size()
+    s = torch.cuda.current_stream() if stream is None else stream
+    a.stream = s.cuda_stream
+    a.use_stream_field = 1
+    a.kernel_variant = int(kernel_variant)
+    rc = load_library().pyramidsd_verify_stage_ex(C.byref(a))
+    out["status"] = rc
+    if raise_on_error:
+        _check(rc, "pyramidsd_verify_stage_ex")
+    return out
+
+
+def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode=FUZZY, philox_seed=0,
+           offset=0, out=None):
+    """``pyramidsd_verify`` (two-stage pyramid) on device tensors. Returns a dict of four [B] int32 tensors."""
+    B, K_d, V = logits_draft.shape
+    K_q = logits_target.shape[1]
+    dt = dtype_code(logits_draft)
+    assert logits_qual.shape == logits_draft.shape and logits_target.shape == (B, K_q, V)
+    dev = logits_draft.device
+    if out is None:
+        out = {k: torch.empty(B, dtype=torch.int32, device=dev)
+               for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+    rc = load_library().pyramidsd_verify(
+        _dev_ptr(logits_draft, name="logits_draft"), _dev_ptr(logits_qual, name="logits_qual"),
+        _dev_ptr(logits_target, name="logits_target"), _dev_ptr(draft_tokens, torch.int32, "draft_tokens"),
+        B, K_d, K_q, V, dt, float(tau_q), float(tau_t), int(mode), int(philox_seed), int(offset),
+        out["accept_len_q"].data_ptr(), out["next_token_q"].data_ptr(),
+        out["accept_len"].data_ptr(), out["next_token"].data_ptr())
+    _check(rc, "pyramidsd_verify")
+    return out
+
+
+def verify_host(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode=FUZZY, philox_seed=0,
+                offset=0, out=None):
+    """``pyramidsd_verify_host``: all tensors are HOST tensors (pinned for speed); copies are inside the call."""
+    B, K_d, V = logits_draft.shape
+    K_q = logits_target.shape[1]
+    dt = dtype_code(logits_draft)
+    for t in (logits_draft, logits_qual, logits_target, draft_tokens):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("verify_host takes contiguous host tensors")
+    if out is None:
+        out = {k: torch.empty(B, dtype=torch.int32).pin_memory()
+               for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+    rc = load_library().pyramidsd_verify_host(
+        logits_draft.data_ptr(), logits_qual.data_ptr(), logits_target.data_ptr(), draft_tokens.data_ptr(),
+        B, K_d, K_q, V, dt, float(tau_q), float(tau_t), int(mode), int(philox_seed), int(offset),
+        out["accept_len_q"].data_ptr(), out["next_token_q"].data_ptr(),
+        out["accept_len"].data_ptr(), out["next_token"].data_ptr())
+    _check(rc, "pyramidsd_verify_host")
+    return out

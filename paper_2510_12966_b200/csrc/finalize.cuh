@@ -1,0 +1,251 @@
+// Finalisation kernel: one CTA per sequence. Warp 0 turns the per-row statistics into accept bits
+// (fuzzy threshold test of Sec. 3.1/3.2, or the standard-SD coin flip), a ballot gives the accepted
+// prefix length (Sec. 1), and, when a position was rejected, the whole CTA draws the correction token
+// from the residual max(0, p_large - p_small) (Sec. 3.4) — or from p_large in the assisted variant —
+// by a hierarchical inverse CDF in vocabulary order: tiles, then warps, then lanes, then elements,
+// each level picking the first child whose inclusive cumulative weight exceeds the remaining target.
+#pragma once
+
+#include "common.cuh"
+
+namespace psd {
+
+constexpr int kFinThreads = 1024;
+constexpr int kFinElemsPerThread = 8;                      // consecutive vocabulary indices per thread and tile
+constexpr int kFinTile = kFinThreads * kFinElemsPerThread;  // 8192 indices per tile
+constexpr int kFinMaxTiles = 1024;                          // V <= 8,388,608
+
+template <typename T>
+struct RowView {
+  const T* large;
+  const T* small;
+  int V;
+  bool vec_ok;
+  float c, m2l, l2sl, m2s, l2ss;
+  bool from_large;  // weights are p_large itself (assisted variant, or an all-zero residual)
+
+  // weights of the kFinElemsPerThread consecutive indices starting at i0 (0 beyond V)
+  __device__ __forceinline__ void weights(int i0, float* w) const {
+    constexpr int E = Elem<T>::kPerVec;
+    float xl[kFinElemsPerThread], xs[kFinElemsPerThread];
+    if (vec_ok && i0 + kFinElemsPerThread <= V) {
+#pragma unroll
+      for (int h = 0; h < kFinElemsPerThread / E; ++h) {
+        Elem<T>::unpack(ldg_vec(large, i0 / E + h), xl + h * E);
+        Elem<T>::unpack(ldg_vec(small, i0 / E + h), xs + h * E);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < kFinElemsPerThread; ++j) {
+        const bool in = i0 + j < V;
+        xl[j] = in ? Elem<T>::load(large, i0 + j) : -INFINITY;
+        xs[j] = in ? Elem<T>::load(small, i0 + j) : -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kFinElemsPerThread; ++j) {
+      const float p = ex2_approx(fmaf(xl[j], c, -m2l) - l2sl);
+      const float q = ex2_approx(fmaf(xs[j], c, -m2s) - l2ss);
+      w[j] = from_large ? p : fmaxf(p - q, 0.f);
+    }
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads) finalize_kernel(const StageParams P) {
+  __shared__ double tile_total[kFinMaxTiles];
+  __shared__ float warp_total[32];
+  __shared__ double scratch[32];
+  __shared__ int sh_L, sh_nv, sh_flags, sh_tile, sh_warp, sh_token;
+  __shared__ float sh_u2, sh_m2l, sh_l2sl, sh_m2s, sh_l2ss, sh_resid, sh_target;
+
+  const int b = blockIdx.x;
+  const int K = P.K, V = P.V;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const T* large_seq = static_cast<const T*>(P.large) + b * P.seq_stride_large;
+  const T* small_seq = static_cast<const T*>(P.small) + b * P.seq_stride_small;
+
+  int nv = K;
+  if (P.n_valid != nullptr) nv = min(max(P.n_valid[b], 0), K);
+
+  // ---- accept bits and prefix length: lane k of warp 0 owns position k (K <= 32) ----
+  if (warp == 0) {
+    bool acc = true;  // lanes beyond nv never end the prefix
+    RowStats st{};
+    float u = 0.f, u2 = 0.f;
+    int flags = 0;
+    if (lane < nv) {
+      const int r = b * K + lane;
+      st = P.stats[r];
+      const int x = P.tokens[r];
+      flags = st.flags | ((x < 0 || x >= V) ? kFlagTokenRange : 0);
+      row_uniforms(P.seed, P.offset, static_cast<unsigned>(r), &u, &u2);
+      const float nanf_ = __int_as_float(0x7fc00000);
+      float px = nanf_, qx = nanf_;
+      bool coin_ok = false;
+      if (!flags) {
+        const long long off = static_cast<long long>(lane) * V + x;
+        px = ex2_approx(fmaf(Elem<T>::load(large_seq, off), P.c, -st.m2_large) - st.l2s_large);
+        qx = ex2_approx(fmaf(Elem<T>::load(small_seq, off), P.c, -st.m2_small) - st.l2s_small);
+        // standard SD: accept with probability min(1, p_large(x) / p_small(x))
+        const float rho = (qx > 0.f) ? __fdiv_rn(px, qx) : (px > 0.f ? INFINITY : 0.f);
+        coin_ok = u < fminf(1.f, rho);
+      }
+      const bool fuzzy_ok = st.div <= P.threshold;
+      if (P.mode == kModeFuzzy) acc = fuzzy_ok;
+      else if (P.mode == kModeStrict || P.mode == kModeAssisted) acc = coin_ok;
+      else acc = fuzzy_ok || coin_ok;
+      if (flags) acc = false;
+      if (P.out_div) P.out_div[r] = st.div;
+      if (P.out_resid_mass) P.out_resid_mass[r] = st.resid;
+      if (P.out_p_small_tok) P.out_p_small_tok[r] = qx;
+      if (P.out_p_large_tok) P.out_p_large_tok[r] = px;
+      if (P.out_row_flags) P.out_row_flags[r] = flags;
+    } else if (lane < K) {
+      const int r = b * K + lane;
+      if (P.out_div) P.out_div[r] = 0.f;
+      if (P.out_resid_mass) P.out_resid_mass[r] = 0.f;
+      if (P.out_p_small_tok) P.out_p_small_tok[r] = 0.f;
+      if (P.out_p_large_tok) P.out_p_large_tok[r] = 0.f;
+      if (P.out_row_flags) P.out_row_flags[r] = 0;
+    }
+    const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
+    const int L = rejected ? (__ffs(rejected) - 1) : nv;  // first rejected position, or all accepted
+    if (lane == min(L, 31)) {  // L < nv <= 32 when a rejection exists; otherwise the row data go unused
+      sh_L = L;
+      sh_nv = nv;
+      sh_flags = flags;
+      sh_u2 = u2;
+      sh_m2l = st.m2_large; sh_l2sl = st.l2s_large;
+      sh_m2s = st.m2_small; sh_l2ss = st.l2s_small;
+      sh_resid = st.resid;
+    }
+  }
+  __syncthreads();
+  const int L = sh_L;
+  int next = -1;
+  bool need_draw = false;
+  if (L < sh_nv) {
+    if (sh_flags & (kFlagSmallNonfinite | kFlagLargeNonfinite)) next = -2;  // no distribution to draw from
+    else need_draw = true;
+  }
+
+  if (need_draw) {  // uniform across the CTA
+    RowView<T> row;
+    row.large = large_seq + static_cast<long long>(L) * V;
+    row.small = small_seq + static_cast<long long>(L) * V;
+    row.V = V;
+    row.vec_ok = ((reinterpret_cast<uintptr_t>(row.large) | reinterpret_cast<uintptr_t>(row.small)) & 15u) == 0 &&
+                 (V % Elem<T>::kPerVec) == 0;
+    row.c = P.c;
+    row.m2l = sh_m2l; row.l2sl = sh_l2sl;
+    row.m2s = sh_m2s; row.l2ss = sh_l2ss;
+    row.from_large = (P.mode == kModeAssisted) || !(sh_resid > 0.f);
+
+    const int n_tiles = (V + kFinTile - 1) / kFinTile;
+    float w[kFinElemsPerThread];
+    // level 0: total weight of every tile
+    for (int j = 0; j < n_tiles; ++j) {
+      row.weights(j * kFinTile + tid * kFinElemsPerThread, w);
+      float ts = 0.f;
+#pragma unroll
+      for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
+      const double tt = block_reduce<OpSum>(static_cast<double>(ts), scratch, 0.0);
+      if (tid == 0) tile_total[j] = tt;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      double total = 0.0;
+      for (int j = 0; j < n_tiles; ++j) total += tile_total[j];
+      const double target = static_cast<double>(sh_u2) * total;
+      // first tile whose inclusive cumulative weight exceeds the target; else the last non-empty tile
+      int pick = -1, last_pos = -1;
+      double cum = 0.0, cum_before_pick = 0.0, cum_before_last = 0.0;
+      for (int j = 0; j < n_tiles; ++j) {
+        const double nxt = cum + tile_total[j];
+        if (tile_total[j] > 0.0) { last_pos = j; cum_before_last = cum; }
+        if (pick < 0 && nxt > target && tile_total[j] > 0.0) { pick = j; cum_before_pick = cum; }
+        cum = nxt;
+      }
+      if (pick < 0) { pick = last_pos; cum_before_pick = cum_before_last; }
+      sh_tile = pick;
+      sh_token = -1;
+      sh_target = static_cast<float>(target - cum_before_pick);
+    }
+    __syncthreads();
+    const int tile = sh_tile;
+    if (tile >= 0) {
+      // level 1: warps of the chosen tile
+      const int i0 = tile * kFinTile + tid * kFinElemsPerThread;
+      row.weights(i0, w);
+      float ts = 0.f;
+#pragma unroll
+      for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
+      // inclusive scan of thread sums across the warp (fixed shuffle tree)
+      float incl = ts;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      if (lane == 31) warp_total[warp] = incl;
+      __syncthreads();
+      if (tid == 0) {
+        const float target = sh_target;
+        int pick = -1, last_pos = -1;
+        float cum = 0.f, before_pick = 0.f, before_last = 0.f;
+        for (int j = 0; j < kFinThreads / 32; ++j) {
+          const float nxt = cum + warp_total[j];
+          if (warp_total[j] > 0.f) { last_pos = j; before_last = cum; }
+          if (pick < 0 && nxt > target && warp_total[j] > 0.f) { pick = j; before_pick = cum; }
+          cum = nxt;
+        }
+        if (pick < 0) { pick = last_pos; before_pick = before_last; }
+        sh_warp = pick;
+        sh_target = target - before_pick;
+      }
+      __syncthreads();
+      if (warp == sh_warp) {
+        // level 2: lanes of the chosen warp
+        const float target = sh_target;
+        const float excl = incl - ts;  // only used as the offset handed to the next level
+        const unsigned hit = __ballot_sync(0xffffffffu, incl > target && ts > 0.f);
+        const unsigned pos = __ballot_sync(0xffffffffu, ts > 0.f);
+        const int pick_lane = hit ? (__ffs(hit) - 1) : (pos ? 31 - __clz(pos) : -1);
+        if (lane == pick_lane) {
+          // level 3: the thread's own consecutive elements
+          const float t3 = target - excl;
+          float run = 0.f;
+          int choice = -1, last_pos = -1;
+#pragma unroll
+          for (int e = 0; e < kFinElemsPerThread; ++e) {
+            run += w[e];
+            if (w[e] > 0.f) {
+              last_pos = e;
+              if (choice < 0 && run > t3) choice = e;
+            }
+          }
+          if (choice < 0) choice = last_pos;
+          sh_token = (choice >= 0) ? i0 + choice : -1;
+        }
+      }
+      __syncthreads();
+      next = sh_token;
+    }
+  }
+
+  if (tid == 0) {
+    P.out_accept_len[b] = L;
+    P.out_next_token[b] = next;
+    if (P.window != nullptr) {
+      // stage-2 window of the two-stage wrapper (Fig. 1): accepted draft tokens, then the correction token
+      const int have = L + (next >= 0 ? 1 : 0);
+      const int n2 = min(have, P.K_window);
+      P.n_window[b] = n2;
+      for (int j = 0; j < P.K_window; ++j)
+        P.window[b * P.K_window + j] = (j < n2) ? ((j < L) ? P.tokens[b * K + j] : next) : 0;
+    }
+  }
+}
+
+}  // namespace psd

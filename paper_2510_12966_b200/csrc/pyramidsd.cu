@@ -1,0 +1,495 @@
+// C ABI of the verification library (declared in include/pyramidsd.h): argument validation, scratch
+// management and kernel launches. No torch types, no CPU fallback: every step of the path runs in the
+// kernels of this directory.
+#include "../../include/pyramidsd.h"
+
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+#include "finalize.cuh"
+#include "rowstats_baseline.cuh"
+#include "rowstats_cluster.cuh"
+
+namespace {
+
+using psd::RowStats;
+using psd::StageParams;
+
+std::atomic<uint64_t> g_launches{0};
+thread_local cudaStream_t t_stream = nullptr;
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kAlign = 256;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Library-owned scratch of one device: workspace for calls that bring none, the status word, and the
+// staging buffers of the host-pointer entry point. Grown on demand, never shrunk, freed at process exit
+// by the driver.
+struct DeviceState {
+  std::mutex mu;
+  void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int* status = nullptr;
+  void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
+  size_t stage_bytes[4] = {0, 0, 0, 0};
+  int32_t* out4 = nullptr;  // 4 x [B] results of the host entry point
+  size_t out4_elems = 0;
+};
+DeviceState g_dev[kMaxDevices];
+
+int current_device_state(DeviceState** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PSD_ERR_CUDA;
+  *out = &g_dev[dev];
+  return PSD_OK;
+}
+
+int grow(void** ptr, size_t* have, size_t want) {
+  if (*have >= want) return PSD_OK;
+  if (*ptr) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return PSD_ERR_CUDA;
+    cudaFree(*ptr);
+    *ptr = nullptr;
+    *have = 0;
+  }
+  if (cudaMalloc(ptr, want) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+  *have = want;
+  return PSD_OK;
+}
+
+int ensure_status(DeviceState* ds) {
+  if (ds->status) return PSD_OK;
+  if (cudaMalloc(reinterpret_cast<void**>(&ds->status), kAlign) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+  if (cudaMemset(ds->status, 0, kAlign) != cudaSuccess) return PSD_ERR_CUDA;
+  return PSD_OK;
+}
+
+size_t stats_bytes(long long rows) { return align_up(static_cast<size_t>(rows) * sizeof(RowStats)); }
+
+size_t stage_workspace_bytes(int B, int K) {
+  // per-row statistics, a [B, K] window and a [B] length (the last two are used by the wrapper only)
+  return stats_bytes(static_cast<long long>(B) * K) + align_up(static_cast<size_t>(B) * K * 4) +
+         align_up(static_cast<size_t>(B) * 4) + kAlign;
+}
+
+bool valid_dtype(int d) { return d == PSD_F32 || d == PSD_BF16; }
+bool valid_mode(int m) { return m >= PSD_FUZZY && m <= PSD_ASSISTED; }
+bool valid_div(int d) { return d >= PSD_DIV_JS && d <= PSD_DIV_KL; }
+size_t elem_size(int dtype) { return dtype == PSD_F32 ? 4 : 2; }
+
+constexpr int kMaxV = psd::kFinTile * psd::kFinMaxTiles;
+
+__global__ void row_uniforms_kernel(unsigned long long seed, unsigned long long offset, int n_rows, float* out_u,
+                                    float* out_u2) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= n_rows) return;
+  float u, u2;
+  psd::row_uniforms(seed, offset, static_cast<unsigned>(r), &u, &u2);
+  if (out_u) out_u[r] = u;
+  if (out_u2) out_u2[r] = u2;
+}
+
+// Optional event bracketing of each launch (pyramidsd_kernel_timing_begin/_end).
+constexpr int kMaxTimed = 4096;
+struct Timing {
+  bool on = false;
+  int n = 0;
+  cudaEvent_t ev[kMaxTimed][2];
+  int created = 0;
+  int tag[kMaxTimed];
+};
+thread_local Timing t_timing;
+
+struct TimedLaunch {
+  cudaStream_t s;
+  int slot = -1;
+  TimedLaunch(cudaStream_t stream, int tag) : s(stream) {
+    Timing& t = t_timing;
+    if (!t.on || t.n >= kMaxTimed) return;
+    if (t.n >= t.created) {
+      if (cudaEventCreate(&t.ev[t.n][0]) != cudaSuccess || cudaEventCreate(&t.ev[t.n][1]) != cudaSuccess) return;
+      t.created = t.n + 1;
+    }
+    slot = t.n++;
+    t.tag[slot] = tag;
+    cudaEventRecord(t.ev[slot][0], s);
+  }
+  ~TimedLaunch() {
+    if (slot >= 0) cudaEventRecord(t_timing.ev[slot][1], s);
+  }
+};
+
+int check_launch() {
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "pyramidsd: kernel launch failed: %s\n", cudaGetErrorString(e));
+    return PSD_ERR_CUDA;
+  }
+  return PSD_OK;
+}
+
+// Statistics pass for one stage: picks the kernel variant and launches it.
+int launch_rowstats(const StageParams& P, int dtype, int variant, cudaStream_t stream) {
+  const long long rows = static_cast<long long>(P.B) * P.K;
+  if (rows == 0) return PSD_OK;
+  bool use_cluster = false;
+  if (variant == PSD_KERNEL_CLUSTER || variant == PSD_KERNEL_AUTO) {
+    use_cluster = psd::cluster_kernel_applicable(P, dtype);
+    if (!use_cluster && variant == PSD_KERNEL_CLUSTER) return PSD_ERR_UNSUPPORTED;
+  }
+  TimedLaunch timed(stream, 0);
+  if (use_cluster) {
+    const int rc = psd::launch_rowstats_cluster(P, dtype, stream);
+    if (rc != PSD_OK) return rc;
+  } else {
+    const dim3 grid(static_cast<unsigned>(rows)), block(1024);
+    if (dtype == PSD_F32) psd::rowstats_baseline_kernel<float><<<grid, block, 0, stream>>>(P);
+    else psd::rowstats_baseline_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(P);
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return check_launch();
+}
+
+int launch_finalize(const StageParams& P, int dtype, cudaStream_t stream) {
+  if (P.B == 0) return PSD_OK;
+  const dim3 grid(static_cast<unsigned>(P.B)), block(psd::kFinThreads);
+  TimedLaunch timed(stream, 1);
+  if (dtype == PSD_F32) psd::finalize_kernel<float><<<grid, block, 0, stream>>>(P);
+  else psd::finalize_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(P);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return check_launch();
+}
+
+int validate_stage(const psd_stage_args* a) {
+  if (a == nullptr || a->struct_size != sizeof(psd_stage_args)) return PSD_ERR_INVALID_ARG;
+  if (!valid_dtype(a->dtype) || !valid_mode(a->mode) || !valid_div(a->div_kind)) return PSD_ERR_INVALID_ARG;
+  if (a->B < 0 || a->K < 0 || a->K > 32 || a->V < 1) return PSD_ERR_INVALID_ARG;
+  if (a->V > kMaxV) return PSD_ERR_UNSUPPORTED;
+  if (static_cast<long long>(a->B) * a->K > (1ll << 30)) return PSD_ERR_UNSUPPORTED;
+  if (a->inv_temperature < 0.f || std::isnan(a->inv_temperature) || std::isinf(a->inv_temperature)) return PSD_ERR_INVALID_ARG;
+  if (std::isnan(a->threshold)) return PSD_ERR_INVALID_ARG;
+  if (a->seq_stride_small < 0 || a->seq_stride_large < 0) return PSD_ERR_INVALID_ARG;
+  if (a->B > 0) {
+    if (!a->out_accept_len || !a->out_next_token) return PSD_ERR_INVALID_ARG;
+    if (a->K > 0 && (!a->logits_small || !a->logits_large || !a->tokens)) return PSD_ERR_INVALID_ARG;
+    const long long min_stride = static_cast<long long>(a->K) * a->V;
+    if (a->seq_stride_small != 0 && a->seq_stride_small < min_stride) return PSD_ERR_INVALID_ARG;
+    if (a->seq_stride_large != 0 && a->seq_stride_large < min_stride) return PSD_ERR_INVALID_ARG;
+  }
+  if (a->workspace != nullptr) {
+    if ((reinterpret_cast<uintptr_t>(a->workspace) % kAlign) != 0) return PSD_ERR_WORKSPACE;
+    if (a->workspace_bytes < stage_workspace_bytes(a->B, a->K)) return PSD_ERR_WORKSPACE;
+  }
+  return PSD_OK;
+}
+
+StageParams make_params(const psd_stage_args* a, void* ws, int* status) {
+  StageParams P{};
+  P.small = a->logits_small;
+  P.large = a->logits_large;
+  P.tokens = a->tokens;
+  P.n_valid = a->n_valid;
+  P.B = a->B; P.K = a->K; P.V = a->V;
+  const long long dense = static_cast<long long>(a->K) * a->V;
+  P.seq_stride_small = a->seq_stride_small ? a->seq_stride_small : dense;
+  P.seq_stride_large = a->seq_stride_large ? a->seq_stride_large : dense;
+  const double invT = a->inv_temperature > 0.f ? static_cast<double>(a->inv_temperature) : 1.0;
+  P.c = static_cast<float>(1.4426950408889634 * invT);
+  P.threshold = a->threshold;
+  P.mode = a->mode;
+  P.div_kind = a->div_kind;
+  P.seed = a->philox_seed;
+  P.offset = a->philox_offset;
+  P.stats = static_cast<RowStats*>(ws);
+  P.out_accept_len = a->out_accept_len;
+  P.out_next_token = a->out_next_token;
+  P.out_div = a->out_div;
+  P.out_p_small_tok = a->out_p_small_tok;
+  P.out_p_large_tok = a->out_p_large_tok;
+  P.out_resid_mass = a->out_resid_mass;
+  P.out_row_flags = a->out_row_flags;
+  P.window = nullptr;
+  P.n_window = nullptr;
+  P.K_window = 0;
+  P.status = status;
+  return P;
+}
+
+cudaStream_t pick_stream(const psd_stage_args* a) {
+  if (a->stream != nullptr || a->use_stream_field) return static_cast<cudaStream_t>(a->stream);
+  return t_stream;
+}
+
+// Runs one stage; `window_out`/`n_window_out`/`K_window` non-null make the finalisation also build the
+// stage-2 window of the wrapper.
+int run_stage(const psd_stage_args* a, int32_t* window_out, int32_t* n_window_out, int K_window) {
+  int rc = validate_stage(a);
+  if (rc != PSD_OK) return rc;
+  if (a->B == 0) return PSD_OK;
+  DeviceState* ds = nullptr;
+  rc = current_device_state(&ds);
+  if (rc != PSD_OK) return rc;
+  void* ws = a->workspace;
+  {
+    std::lock_guard<std::mutex> lock(ds->mu);
+    rc = ensure_status(ds);
+    if (rc != PSD_OK) return rc;
+    if (ws == nullptr) {
+      rc = grow(&ds->ws, &ds->ws_bytes, stage_workspace_bytes(a->B, a->K));
+      if (rc != PSD_OK) return rc;
+      ws = ds->ws;
+    }
+  }
+  StageParams P = make_params(a, ws, ds->status);
+  P.window = window_out;
+  P.n_window = n_window_out;
+  P.K_window = K_window;
+  const cudaStream_t stream = pick_stream(a);
+  if (a->K > 0) {
+    rc = launch_rowstats(P, a->dtype, a->kernel_variant, stream);
+    if (rc != PSD_OK) return rc;
+  }
+  return launch_finalize(P, a->dtype, stream);
+}
+
+int verify_two_stage(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                     const int32_t* draft_tokens, int B, int K_d, int K_q, int V, int dtype, float tau_q,
+                     float tau_t, int mode, uint64_t seed, uint64_t offset, int32_t* out_accept_len_q,
+                     int32_t* out_next_token_q, int32_t* out_accept_len, int32_t* out_next_token,
+                     cudaStream_t stream, int variant) {
+  if (K_q < 1 || K_d < K_q || K_d > 32 || B < 0 || V < 1) return PSD_ERR_INVALID_ARG;
+  if (B == 0) return PSD_OK;
+  DeviceState* ds = nullptr;
+  int rc = current_device_state(&ds);
+  if (rc != PSD_OK) return rc;
+  // scratch: [stage-1 workspace][stage-2 workspace]; the window and its length live in stage 1's tail
+  const size_t ws1 = stage_workspace_bytes(B, K_d), ws2 = stage_workspace_bytes(B, K_q);
+  char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(ds->mu);
+    rc = grow(&ds->ws, &ds->ws_bytes, ws1 + ws2);
+    if (rc != PSD_OK) return rc;
+    base = static_cast<char*>(ds->ws);
+  }
+  int32_t* window = reinterpret_cast<int32_t*>(base + stats_bytes(static_cast<long long>(B) * K_d));
+  int32_t* n_window = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(window) + align_up(static_cast<size_t>(B) * K_d * 4));
+
+  psd_stage_args s1;
+  std::memset(&s1, 0, sizeof(s1));
+  s1.struct_size = sizeof(s1);
+  s1.dtype = dtype;
+  s1.logits_small = logits_draft;
+  s1.logits_large = logits_qual;
+  s1.tokens = draft_tokens;
+  s1.B = B; s1.K = K_d; s1.V = V;
+  s1.mode = mode;
+  s1.div_kind = PSD_DIV_JS;
+  s1.threshold = tau_q;
+  s1.philox_seed = seed;
+  s1.philox_offset = offset;
+  s1.out_accept_len = out_accept_len_q;
+  s1.out_next_token = out_next_token_q;
+  s1.workspace = base;
+  s1.workspace_bytes = ws1;
+  s1.stream = stream;
+  s1.use_stream_field = 1;
+  s1.kernel_variant = variant;
+  rc = run_stage(&s1, window, n_window, K_q);
+  if (rc != PSD_OK) return rc;
+
+  psd_stage_args s2 = s1;
+  s2.logits_small = logits_qual;   // P_MQ takes the place of P_MD in the target comparison (Fig. 1)
+  s2.logits_large = logits_target;
+  s2.seq_stride_small = static_cast<int64_t>(K_d) * V;  // rows 0..K_q-1 of each [K_d, V] qualifier sequence
+  s2.seq_stride_large = 0;
+  s2.tokens = window;
+  s2.n_valid = n_window;
+  s2.K = K_q;
+  s2.threshold = tau_t;
+  s2.philox_offset = offset + 1;
+  s2.out_accept_len = out_accept_len;
+  s2.out_next_token = out_next_token;
+  s2.workspace = base + ws1;
+  s2.workspace_bytes = ws2;
+  return run_stage(&s2, nullptr, nullptr, 0);
+}
+
+}  // namespace
+
+extern "C" {
+
+int pyramidsd_verify_stage_ex(const psd_stage_args* args) { return run_stage(args, nullptr, nullptr, 0); }
+
+int pyramidsd_verify_stage(const void* logits_small, const void* logits_large, const int32_t* draft_tokens,
+                           int B, int K, int V, psd_dtype dtype, float threshold, psd_mode mode,
+                           uint64_t philox_seed, uint64_t offset, int32_t* out_accept_len,
+                           int32_t* out_next_token) {
+  psd_stage_args a;
+  std::memset(&a, 0, sizeof(a));
+  a.struct_size = sizeof(a);
+  a.dtype = dtype;
+  a.logits_small = logits_small;
+  a.logits_large = logits_large;
+  a.tokens = draft_tokens;
+  a.B = B; a.K = K; a.V = V;
+  a.mode = mode;
+  a.div_kind = PSD_DIV_JS;
+  a.threshold = threshold;
+  a.philox_seed = philox_seed;
+  a.philox_offset = offset;
+  a.out_accept_len = out_accept_len;
+  a.out_next_token = out_next_token;
+  return run_stage(&a, nullptr, nullptr, 0);
+}
+
+int pyramidsd_verify(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                     const int32_t* draft_tokens, int B, int K_d, int K_q, int V, psd_dtype dtype,
+                     float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
+                     int32_t* out_accept_len_q, int32_t* out_next_token_q, int32_t* out_accept_len,
+                     int32_t* out_next_token) {
+  if (!valid_dtype(dtype) || !valid_mode(mode)) return PSD_ERR_INVALID_ARG;
+  if (B > 0 && (!logits_draft || !logits_qual || !logits_target || !draft_tokens || !out_accept_len_q ||
+                !out_next_token_q || !out_accept_len || !out_next_token))
+    return PSD_ERR_INVALID_ARG;
+  return verify_two_stage(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype, tau_q,
+                          tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q, out_accept_len,
+                          out_next_token, t_stream, PSD_KERNEL_AUTO);
+}
+
+int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                          const int32_t* draft_tokens, int B, int K_d, int K_q, int V, psd_dtype dtype,
+                          float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
+                          int32_t* out_accept_len_q, int32_t* out_next_token_q, int32_t* out_accept_len,
+                          int32_t* out_next_token) {
+  if (!valid_dtype(dtype) || !valid_mode(mode)) return PSD_ERR_INVALID_ARG;
+  if (K_q < 1 || K_d < K_q || K_d > 32 || B < 0 || V < 1) return PSD_ERR_INVALID_ARG;
+  if (B == 0) return PSD_OK;
+  if (!logits_draft || !logits_qual || !logits_target || !draft_tokens || !out_accept_len_q ||
+      !out_next_token_q || !out_accept_len || !out_next_token)
+    return PSD_ERR_INVALID_ARG;
+  DeviceState* ds = nullptr;
+  int rc = current_device_state(&ds);
+  if (rc != PSD_OK) return rc;
+  const size_t es = elem_size(dtype);
+  const size_t n_d = static_cast<size_t>(B) * K_d * V * es, n_t = static_cast<size_t>(B) * K_q * V * es;
+  const size_t n_tok = static_cast<size_t>(B) * K_d * 4;
+  {
+    std::lock_guard<std::mutex> lock(ds->mu);
+    const size_t want[4] = {n_d, n_d, n_t, n_tok};
+    for (int i = 0; i < 4; ++i) {
+      rc = grow(&ds->stage[i], &ds->stage_bytes[i], want[i]);
+      if (rc != PSD_OK) return rc;
+    }
+    if (ds->out4_elems < static_cast<size_t>(4) * B) {
+      size_t have = ds->out4_elems * 4;
+      void* p = ds->out4;
+      rc = grow(&p, &have, static_cast<size_t>(4) * B * 4);
+      if (rc != PSD_OK) return rc;
+      ds->out4 = static_cast<int32_t*>(p);
+      ds->out4_elems = static_cast<size_t>(4) * B;
+    }
+  }
+  const cudaStream_t s = t_stream;
+  const void* src[4] = {logits_draft, logits_qual, logits_target, draft_tokens};
+  const size_t nbytes[4] = {n_d, n_d, n_t, n_tok};
+  for (int i = 0; i < 4; ++i)
+    if (cudaMemcpyAsync(ds->stage[i], src[i], nbytes[i], cudaMemcpyHostToDevice, s) != cudaSuccess) return PSD_ERR_CUDA;
+  int32_t* o = ds->out4;
+  rc = verify_two_stage(ds->stage[0], ds->stage[1], ds->stage[2], static_cast<const int32_t*>(ds->stage[3]), B, K_d,
+                        K_q, V, dtype, tau_q, tau_t, mode, philox_seed, offset, o, o + B, o + 2 * B, o + 3 * B, s,
+                        PSD_KERNEL_AUTO);
+  if (rc != PSD_OK) return rc;
+  int32_t* dst[4] = {out_accept_len_q, out_next_token_q, out_accept_len, out_next_token};
+  for (int i = 0; i < 4; ++i)
+    if (cudaMemcpyAsync(dst[i], o + static_cast<size_t>(i) * B, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+      return PSD_ERR_CUDA;
+  return cudaStreamSynchronize(s) == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
+}
+
+int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, float* out_u, float* out_u2) {
+  if (n_rows < 0) return PSD_ERR_INVALID_ARG;
+  if (n_rows == 0 || (!out_u && !out_u2)) return PSD_OK;
+  row_uniforms_kernel<<<(n_rows + 255) / 256, 256, 0, t_stream>>>(philox_seed, offset, n_rows, out_u, out_u2);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return check_launch();
+}
+
+size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype) {
+  if (B < 0 || K < 0 || K > 32 || V < 1 || !valid_dtype(dtype)) return 0;
+  return stage_workspace_bytes(B, K);
+}
+
+int pyramidsd_set_stream(void* cuda_stream) {
+  t_stream = static_cast<cudaStream_t>(cuda_stream);
+  return PSD_OK;
+}
+
+int pyramidsd_last_status(void) {
+  DeviceState* ds = nullptr;
+  int rc = current_device_state(&ds);
+  if (rc != PSD_OK) return rc;
+  if (cudaStreamSynchronize(t_stream) != cudaSuccess) return PSD_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(ds->mu);
+  if (!ds->status) return PSD_OK;
+  int host = 0;
+  if (cudaMemcpy(&host, ds->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PSD_ERR_CUDA;
+  if (host != 0) {
+    cudaMemset(ds->status, 0, sizeof(int));
+    return PSD_ERR_TIMEOUT;
+  }
+  return PSD_OK;
+}
+
+int pyramidsd_kernel_timing_begin(void) {
+  t_timing.n = 0;
+  t_timing.on = true;
+  return PSD_OK;
+}
+
+int pyramidsd_kernel_timing_end(double* ms_rowstats, int* n_rowstats, double* ms_finalize, int* n_finalize) {
+  Timing& t = t_timing;
+  t.on = false;
+  double ms[2] = {0.0, 0.0};
+  int cnt[2] = {0, 0};
+  for (int i = 0; i < t.n; ++i) {
+    if (cudaEventSynchronize(t.ev[i][1]) != cudaSuccess) return PSD_ERR_CUDA;
+    float f = 0.f;
+    if (cudaEventElapsedTime(&f, t.ev[i][0], t.ev[i][1]) != cudaSuccess) return PSD_ERR_CUDA;
+    ms[t.tag[i]] += f;
+    cnt[t.tag[i]] += 1;
+  }
+  t.n = 0;
+  if (ms_rowstats) *ms_rowstats = ms[0];
+  if (n_rowstats) *n_rowstats = cnt[0];
+  if (ms_finalize) *ms_finalize = ms[1];
+  if (n_finalize) *n_finalize = cnt[1];
+  return PSD_OK;
+}
+
+uint64_t pyramidsd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int pyramidsd_cluster_occupancy(int V, psd_dtype dtype, int* out_cluster_size, int* out_max_active_clusters) {
+  if (V < 1 || !valid_dtype(dtype)) return PSD_ERR_INVALID_ARG;
+  return psd::cluster_occupancy(V, dtype, out_cluster_size, out_max_active_clusters);
+}
+
+const char* pyramidsd_version(void) { return "pyramidsd-b200 0.1.0 (sm_100a)"; }
+
+const char* pyramidsd_status_string(int status) {
+  switch (status) {
+    case PSD_OK: return "ok";
+    case PSD_ERR_INVALID_ARG: return "invalid argument";
+    case PSD_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case PSD_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case PSD_ERR_CUDA: return "CUDA runtime error";
+    case PSD_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,94 @@
+"""Host-side checks that need no GPU: the shared library builds for sm_100a, loads, exports every
+symbol the header declares, and rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2510_12966_b200 import binding, build
+    build.build()
+    return binding.load_library()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "pyramidsd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pyramidsd_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    from paper_2510_12966_b200 import binding
+    names = declared_symbols()
+    assert len(names) >= 10
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/pyramidsd.h but not exported"
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_struct_layout_matches_header(lib, tmp_path):
+    """sizeof(psd_stage_args) as the C compiler sees it equals the ctypes mirror."""
+    import subprocess
+    from paper_2510_12966_b200 import binding
+    src = tmp_path / "sz.c"
+    src.write_text('#include "pyramidsd.h"\n#include <stdio.h>\n#include <stddef.h>\n'
+                   'int main(void){printf("%zu %zu %zu\\n", sizeof(psd_stage_args), offsetof(psd_stage_args, workspace),'
+                   ' offsetof(psd_stage_args, kernel_variant));return 0;}\n')
+    exe = tmp_path / "sz"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    size, off_ws, off_kv = map(int, subprocess.check_output([str(exe)]).split())
+    assert size == C.sizeof(binding.StageArgs)
+    assert off_ws == binding.StageArgs.workspace.offset and off_kv == binding.StageArgs.kernel_variant.offset
+
+
+def test_version_and_status_strings(lib):
+    from paper_2510_12966_b200 import binding
+    assert "sm_100a" in binding.version()
+    assert binding.status_string(0) == "ok" and "invalid" in binding.status_string(-1)
+
+
+def test_workspace_bytes_is_host_arithmetic(lib):
+    from paper_2510_12966_b200 import binding
+    small = binding.workspace_bytes(1, 4, 32000, binding.F32)
+    big = binding.workspace_bytes(256, 32, 152064, binding.BF16)
+    assert 0 < small < big and big >= 256 * 32 * 32
+    assert binding.workspace_bytes(1, 33, 100, binding.F32) == 0 and binding.workspace_bytes(1, 4, 0, binding.F32) == 0
+
+
+def test_invalid_arguments_are_rejected_before_any_launch(lib):
+    from paper_2510_12966_b200 import binding
+    a = binding.StageArgs()
+    assert lib.pyramidsd_verify_stage_ex(C.byref(a)) == binding.ERR_INVALID_ARG          # struct_size 0
+    a.struct_size = C.sizeof(binding.StageArgs)
+    a.B, a.K, a.V = 1, 1, 0
+    assert lib.pyramidsd_verify_stage_ex(C.byref(a)) == binding.ERR_INVALID_ARG          # V < 1
+    a.V = 16
+    assert lib.pyramidsd_verify_stage_ex(C.byref(a)) == binding.ERR_INVALID_ARG          # NULL outputs
+    a.K = 40
+    assert lib.pyramidsd_verify_stage_ex(C.byref(a)) == binding.ERR_INVALID_ARG          # K > 32
+    a.K, a.V = 1, 1 << 30
+    assert lib.pyramidsd_verify_stage_ex(C.byref(a)) == binding.ERR_UNSUPPORTED          # V beyond the limit
+    assert lib.pyramidsd_verify_stage_ex(None) == binding.ERR_INVALID_ARG
+    assert lib.pyramidsd_verify(None, None, None, None, 1, 4, 8, 100, 1, 0.1, 0.1, 0, 0, 0, None, None, None, None) \
+        == binding.ERR_INVALID_ARG                                                        # K_q > K_d, NULLs
+    assert lib.pyramidsd_verify_stage(None, None, None, 0, 4, 100, 0, 0.1, 0, 0, 0, None, None) == binding.OK  # B == 0
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    from paper_2510_12966_b200 import binding
+    with pytest.raises(ImportError):
+        binding.load_library(str(tmp_path / "libpyramidsd.so"))
+
+
+def test_product_path_does_not_touch_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2510_12966_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower() or f == "workloads.py", f

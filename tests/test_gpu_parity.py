@@ -1,0 +1,311 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded
+inputs and the same Philox stream. Sizes span several tiles and ragged tails; reduced versions of the
+BASELINE workloads run element by element, and the full-size bench configuration is checked on sampled
+sequences."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from parity_utils import TOL, compare_stage, dtype_name, gpu_stage_to_numpy, host_bits
+
+pytestmark = pytest.mark.gpu
+
+LN2 = math.log(2.0)
+
+
+@pytest.fixture(scope="module")
+def psd():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2510_12966_b200 import binding
+    binding.load_library()
+    torch.cuda.set_device(0)
+    return binding
+
+
+@pytest.fixture(scope="module")
+def wl():
+    from paper_2510_12966_b200 import workloads
+    return workloads
+
+
+def run_stage_both(psd, oracle, zs, zl, tok, tau, mode=0, seed=0, offset=0, n_valid=None, inv_temperature=0.0,
+                   div_kind=0, variant=0):
+    """Library on the GPU, oracle on the host, same bits. Returns (gpu dict, oracle dict, report)."""
+    dev = torch.device("cuda:0")
+    zs_d, zl_d, tok_d = zs.to(dev), zl.to(dev), tok.to(dev)
+    nv_d = None if n_valid is None else torch.as_tensor(n_valid, dtype=torch.int32, device=dev)
+    out = psd.verify_stage_ex(zs_d, zl_d, tok_d, tau, mode, seed, offset, n_valid=nv_d,
+                              inv_temperature=inv_temperature, div_kind=div_kind, kernel_variant=variant)
+    torch.cuda.synchronize()
+    assert psd.last_status() == 0
+    gpu = gpu_stage_to_numpy(out)
+    zs_h, zl_h = host_bits(zs), host_bits(zl)
+    invT = inv_temperature if inv_temperature > 0 else 1.0
+    orc = oracle.verify_stage(zs_h, zl_h, tok.numpy(), np.float32(tau), mode, seed, offset, n_valid=n_valid,
+                              inv_temperature=float(np.float32(invT)), div_kind=div_kind, n_threads=8)
+    rep = compare_stage(oracle, gpu, orc, zs_h, zl_h, dtype=dtype_name(zs), mode=mode, tau=float(np.float32(tau)),
+                        seed=seed, offset=offset, n_valid=n_valid, div_kind=div_kind,
+                        inv_temperature=float(np.float32(invT)))
+    return gpu, orc, rep
+
+
+# --------------------------------------------------------------------------------------------------
+def test_row_uniforms_match_oracle_philox(psd, oracle):
+    seed, offset, n = 0x9E3779B97F4A7C15, (1 << 40) + 12345, 100_000
+    u, u2 = psd.row_uniforms(seed, offset, n)
+    u, u2 = u.cpu().numpy(), u2.cpu().numpy()
+    rows = np.r_[0:2000, n - 2000:n]
+    for r in rows:
+        a, b = oracle.row_uniforms(seed, offset, int(r))
+        assert u[r] == np.float32(a) and u2[r] == np.float32(b)
+    assert 0.0 <= u.min() and u.max() < 1.0
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [5, 16, 17, 1000, 4099, 8192, 8200, 32000, 50257])
+def test_stage_fuzzy_small_shapes(psd, oracle, wl, dtype, V):
+    B, K = 3, 5
+    zs, zl, tok = wl.make_stage_inputs(B, K, V, dtype, seed=100 + V, sigma=0.8)
+    for tau in (0.02, 0.1, 0.3):
+        _, _, rep = run_stage_both(psd, oracle, zs, zl, tok, tau, seed=V, offset=7)
+        assert rep["tie_div"] + rep["tie_cdf"] <= 2
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mode", [1, 2, 3])
+def test_stage_coin_flip_modes(psd, oracle, wl, dtype, mode):
+    B, K, V = 16, 6, 12000
+    zs, zl, tok = wl.make_stage_inputs(B, K, V, dtype, seed=7, sigma=0.6)
+    ties = 0
+    for offset in range(4):
+        _, orc, rep = run_stage_both(psd, oracle, zs, zl, tok, 0.05, mode=mode, seed=3, offset=offset)
+        ties += rep["tie_coin"] + rep["tie_cdf"] + rep["tie_div"]
+        assert 0 < orc["accept_len"].sum() < B * K   # the case exercises both outcomes
+    assert ties <= 4
+
+
+@pytest.mark.parametrize("div_kind", [1, 2])
+def test_other_divergences(psd, oracle, wl, div_kind):
+    zs, zl, tok = wl.make_stage_inputs(4, 4, 20000, "f32", seed=8, sigma=0.5)
+    tau = 0.3 if div_kind == 1 else 0.5
+    run_stage_both(psd, oracle, zs, zl, tok, tau, div_kind=div_kind)
+
+
+def test_temperature(psd, oracle, wl):
+    zs, zl, tok = wl.make_stage_inputs(4, 4, 20000, "f32", seed=9, sigma=0.5)
+    run_stage_both(psd, oracle, zs, zl, tok, 0.2, inv_temperature=1 / 0.7)   # Sec. 4.1: temperature 0.7
+
+
+def test_cfg1_tiny_fp32(psd, oracle, wl):
+    """BASELINE config 1: B=1, K=4, V=32000 fp32, fuzzy tau=0.3 and strict, Philox seed 0, several rounds."""
+    ties = 0
+    for rnd in range(8):
+        zs, zl, tok = wl.workload_inputs(1, rnd)
+        for mode in (0, 1):
+            _, _, rep = run_stage_both(psd, oracle, zs, zl, tok, 0.3, mode=mode, seed=0, offset=rnd)
+            ties += rep["tie_div"] + rep["tie_coin"] + rep["tie_cdf"]
+            assert rep["max_err_div"] < 1e-5
+    assert ties <= 1
+
+
+def test_edge_identical_rows_and_thresholds(psd, oracle, wl):
+    zs, zl, tok = wl.make_stage_inputs(2, 4, 5000, "bf16", seed=10)
+    gpu, orc, _ = run_stage_both(psd, oracle, zl, zl, tok, 0.0)
+    assert np.all(gpu["div"] == 0.0) and np.all(gpu["resid_mass"] == 0.0)
+    assert np.all(gpu["accept_len"] == 4) and np.all(gpu["next_token"] == -1)
+    gpu, _, _ = run_stage_both(psd, oracle, zs, zl, tok, np.float32(LN2) + 1e-6)   # tau >= max JS: all accepted
+    assert np.all(gpu["accept_len"] == 4)
+    gpu, _, _ = run_stage_both(psd, oracle, zs, zl, tok, -1e-6)                    # tau < 0: none accepted
+    assert np.all(gpu["accept_len"] == 0) and np.all(gpu["next_token"] >= 0)
+    # strict mode on identical rows: ratio 1, always accepted
+    gpu, _, _ = run_stage_both(psd, oracle, zl, zl, tok, 0.0, mode=1)
+    assert np.all(gpu["accept_len"] == 4)
+    # disjoint supports: JS = ln 2, TV = 1
+    z1 = torch.full((1, 1, 64), -float("inf"))
+    z2 = z1.clone()
+    z1[0, 0, 3] = 0.0
+    z2[0, 0, 40] = 1.0
+    gpu, orc, _ = run_stage_both(psd, oracle, z1, z2, torch.tensor([[3]], dtype=torch.int32), 0.5)
+    assert abs(gpu["div"][0, 0] - LN2) < 1e-6 and abs(gpu["resid_mass"][0, 0] - 1.0) < 1e-6
+    assert gpu["next_token"][0] == 40
+
+
+def test_edge_masked_and_flagged_rows(psd, oracle, wl):
+    zs, zl, tok = wl.make_stage_inputs(4, 3, 3000, "f32", seed=11, sigma=0.3)
+    zs[0, 1, 100:900] = -float("inf")          # masked vocabulary on one side only
+    zl[1, 0, :] = -float("inf")
+    zl[1, 0, 5] = 2.0                           # a single live token
+    zs[2, 1, 17] = float("nan")
+    zl[3, 0, 2999] = float("inf")
+    tok[0, 2] = 3000                             # out of range
+    gpu, orc, _ = run_stage_both(psd, oracle, zs, zl, tok, 1.0)
+    assert gpu["next_token"][2] == -2 and gpu["accept_len"][2] == 1
+    assert gpu["next_token"][3] == -2 and gpu["accept_len"][3] == 0
+    assert gpu["row_flags"][0, 2] == 4 and gpu["accept_len"][0] == 2
+    zs2, zl2, tok2 = wl.make_stage_inputs(1, 2, 64, "f32", seed=12)
+    zl2[0, 0, :] = -float("inf")                # a row with no finite entry is flagged too
+    gpu, _, _ = run_stage_both(psd, oracle, zs2, zl2, tok2, 1.0)
+    assert gpu["row_flags"][0, 0] == 2 and gpu["next_token"][0] == -2
+
+
+def test_edge_empty_and_n_valid(psd, oracle, wl):
+    dev = torch.device("cuda:0")
+    zs, zl, tok = wl.make_stage_inputs(4, 6, 2048, "bf16", seed=13, sigma=0.2)
+    gpu, orc, _ = run_stage_both(psd, oracle, zs, zl, tok, 0.5, n_valid=[0, 2, 6, 3])
+    assert gpu["accept_len"][0] == 0 and gpu["next_token"][0] == -1
+    empty = torch.empty((0, 6, 2048), dtype=torch.bfloat16, device=dev)
+    out = psd.verify_stage_ex(empty, empty, torch.empty((0, 6), dtype=torch.int32, device=dev), 0.1)
+    assert out["status"] == 0
+    z0 = torch.empty((3, 0, 2048), dtype=torch.bfloat16, device=dev)
+    out = psd.verify_stage_ex(z0, z0, torch.empty((3, 0), dtype=torch.int32, device=dev), 0.1, want_rows=False)
+    torch.cuda.synchronize()
+    assert out["accept_len"].tolist() == [0, 0, 0] and out["next_token"].tolist() == [-1, -1, -1]
+    # K = 32, the widest window the scan takes
+    zs, zl, tok = wl.make_stage_inputs(2, 32, 1024, "f32", seed=14, sigma=0.05)
+    gpu, orc, _ = run_stage_both(psd, oracle, zs, zl, tok, 1.0)
+    assert np.all(gpu["accept_len"] == 32)
+    run_stage_both(psd, oracle, zs, zl, tok, 0.0005)
+
+
+def test_bad_arguments_return_codes(psd, wl):
+    dev = torch.device("cuda:0")
+    zs, zl, tok = [t.to(dev) for t in wl.make_stage_inputs(1, 2, 64, "f32", seed=15)]
+    assert psd.verify_stage_ex(zs, zl, tok, 0.1, mode=9, raise_on_error=False)["status"] == psd.ERR_INVALID_ARG
+    assert psd.verify_stage_ex(zs, zl, tok, 0.1, div_kind=5, raise_on_error=False)["status"] == psd.ERR_INVALID_ARG
+    assert psd.verify_stage_ex(zs, zl, tok, 0.1, K=33, B=1, V=64, raise_on_error=False)["status"] == psd.ERR_INVALID_ARG
+    assert psd.verify_stage_ex(zs, zl, tok, float("nan"), raise_on_error=False)["status"] == psd.ERR_INVALID_ARG
+    small_ws = torch.empty(256, dtype=torch.uint8, device=dev)
+    assert psd.verify_stage_ex(zs, zl, tok, 0.1, workspace=small_ws, raise_on_error=False)["status"] == psd.ERR_WORKSPACE
+    ws = torch.empty(psd.workspace_bytes(1, 2, 64, psd.F32), dtype=torch.uint8, device=dev)
+    assert psd.verify_stage_ex(zs, zl, tok, 0.1, workspace=ws)["status"] == 0
+    with pytest.raises(psd.PyramidSDError):
+        psd.verify(zs, zs, zs, tok, 0.1, 0.1, mode=7)
+    torch.cuda.synchronize()
+    assert psd.last_status() == 0
+
+
+def test_results_are_bit_identical_run_to_run(psd, wl):
+    dev = torch.device("cuda:0")
+    zs, zl, tok = [t.to(dev) for t in wl.make_stage_inputs(8, 8, 32000, "bf16", seed=16, sigma=0.7)]
+    ref = None
+    for _ in range(5):
+        out = psd.verify_stage_ex(zs, zl, tok, 0.05, mode=2, philox_seed=1, offset=2)
+        torch.cuda.synchronize()
+        cur = {k: v.clone() for k, v in out.items() if isinstance(v, torch.Tensor)}
+        if ref is not None:
+            for k in ref:
+                assert torch.equal(ref[k].view(torch.int32), cur[k].view(torch.int32)), k
+        ref = cur
+
+
+# -------------------------------------------------------------------------------------------------- wrapper
+def run_pyramid_both(psd, oracle, zd, zq, zt, tok, tau_q, tau_t, mode=0, seed=0, offset=0):
+    dev = torch.device("cuda:0")
+    out = psd.verify(zd.to(dev), zq.to(dev), zt.to(dev), tok.to(dev), tau_q, tau_t, mode, seed, offset)
+    torch.cuda.synchronize()
+    assert psd.last_status() == 0
+    gpu = gpu_stage_to_numpy(out)
+    zd_h, zq_h, zt_h = host_bits(zd), host_bits(zq), host_bits(zt)
+    orc = oracle.verify(zd_h, zq_h, zt_h, tok.numpy(), np.float32(tau_q), np.float32(tau_t), mode, seed, offset,
+                        n_threads=8)
+    return gpu, orc, (zd_h, zq_h, zt_h)
+
+
+def check_pyramid(oracle, gpu, orc, hosts, dtype, mode, tau_q, tau_t, seed, offset, tok, seq_ids=None):
+    """Stage 1 against the oracle; when stage 1 agrees for a sequence, stage 2 must agree as well."""
+    zd_h, zq_h, zt_h = hosts
+    B, K_d = tok.shape
+    K_q = zt_h.shape[1]
+    s1g = dict(accept_len=gpu["accept_len_q"], next_token=gpu["next_token_q"])
+    o1 = oracle.verify_stage(zd_h, zq_h, tok, np.float32(tau_q), mode, seed, offset, n_threads=8, seq_ids=seq_ids)
+    assert np.array_equal(o1["accept_len"], orc["accept_len_q"])
+    rep1 = compare_stage(oracle, s1g, o1, zd_h, zq_h, dtype=dtype, mode=mode, tau=float(np.float32(tau_q)), seed=seed,
+                         offset=offset, seq_ids=seq_ids, check_rows=False)
+    same = (gpu["accept_len_q"] == orc["accept_len_q"]) & (gpu["next_token_q"] == orc["next_token_q"])
+    idx = np.nonzero(same)[0]
+    rep2 = dict(tie_div=0, tie_coin=0, tie_cdf=0)
+    if len(idx):
+        zq2 = np.ascontiguousarray(zq_h[idx][:, :K_q])
+        ids = idx if seq_ids is None else np.asarray(seq_ids)[idx]
+        o2 = oracle.verify_stage(zq2, zt_h[idx], orc["window"][idx], np.float32(tau_t), mode, seed, offset + 1,
+                                 n_valid=orc["n_window"][idx], n_threads=8, seq_ids=ids)
+        assert np.array_equal(o2["accept_len"], orc["accept_len"][idx])
+        s2g = dict(accept_len=gpu["accept_len"][idx], next_token=gpu["next_token"][idx])
+        rep2 = compare_stage(oracle, s2g, o2, zq2, zt_h[idx], dtype=dtype, mode=mode, tau=float(np.float32(tau_t)),
+                             seed=seed, offset=offset + 1, n_valid=orc["n_window"][idx], seq_ids=ids,
+                             check_rows=False)
+    ties = sum(rep1[k] + rep2[k] for k in ("tie_div", "tie_coin", "tie_cdf"))
+    return ties, len(idx)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_pyramid_reduced_cfg2(psd, oracle, wl, mode):
+    """BASELINE config 2 (single stream, V=128256 bf16, K_d=8, K_q=4), a few rounds."""
+    ties = 0
+    for rnd in range(3):
+        zd, zq, zt, tok = wl.workload_inputs(2, rnd)
+        gpu, orc, hosts = run_pyramid_both(psd, oracle, zd, zq, zt, tok, 0.4, 0.2, mode, 0, 2 * rnd)
+        t, _ = check_pyramid(oracle, gpu, orc, hosts, "bf16", mode, 0.4, 0.2, 0, 2 * rnd, tok.numpy())
+        ties += t
+    assert ties <= 1
+
+
+def test_pyramid_reduced_cfg3(psd, oracle, wl):
+    """BASELINE config 3 recipe at B=6 (V=128256 bf16, K_d=16, K_q=8, per-sequence boost U[4,12])."""
+    zd, zq, zt, tok = wl.workload_inputs(3, 0, B=6)
+    ties = 0
+    for tau_q, tau_t in ((0.4, 0.2), (0.69, 0.5)):
+        gpu, orc, hosts = run_pyramid_both(psd, oracle, zd, zq, zt, tok, tau_q, tau_t, 0, 0, 0)
+        t, n = check_pyramid(oracle, gpu, orc, hosts, "bf16", 0, tau_q, tau_t, 0, 0, tok.numpy())
+        ties += t
+        assert n >= 5
+    assert ties <= 1
+
+
+def test_pyramid_small_vocab_all_paths(psd, oracle, wl):
+    """Small V so that windows of every length (cut, short, full) occur; fp32; every mode."""
+    zd, zq, zt, tok = wl.make_pyramid_inputs(24, 6, 4, 777, "f32", seed=21, sigma_q=0.3, sigma_d=0.5)
+    for mode in (0, 1, 2, 3):
+        gpu, orc, hosts = run_pyramid_both(psd, oracle, zd, zq, zt, tok, 0.03, 0.02, mode, 5, 10)
+        ties, n = check_pyramid(oracle, gpu, orc, hosts, "f32", mode, 0.03, 0.02, 5, 10, tok.numpy())
+        assert ties <= 2 and n >= 22
+        lens = set(orc["n_window"].tolist())
+        assert len(lens) >= 2
+
+
+def test_host_entry_point_equals_device_entry_point(psd, wl):
+    dev = torch.device("cuda:0")
+    zd, zq, zt, tok = wl.make_pyramid_inputs(5, 8, 4, 9000, "bf16", seed=22)
+    a = psd.verify(zd.to(dev), zq.to(dev), zt.to(dev), tok.to(dev), 0.4, 0.2, 0, 3, 4)
+    torch.cuda.synchronize()
+    b = psd.verify_host(zd.pin_memory(), zq.pin_memory(), zt.pin_memory(), tok.pin_memory(), 0.4, 0.2, 0, 3, 4)
+    for k in a:
+        assert torch.equal(a[k].cpu(), b[k]), k
+
+
+def test_full_size_bench_config_sampled(psd, oracle, wl):
+    """The bench workload (config 3 at full size, B=64) in the launch configuration bench.py times;
+    the oracle checks a sample of sequences one by one."""
+    dev = torch.device("cuda:0")
+    w = wl.CONFIGS[3]
+    zd, zq, zt, tok = wl.workload_inputs(3, 1, device=dev)
+    psd.set_stream()
+    out = psd.verify(zd, zq, zt, tok, w.tau_q, w.tau_t, 0, 0, 2)
+    torch.cuda.synchronize()
+    assert psd.last_status() == 0
+    pick = np.array([0, 13, 37, 63])
+    gpu = {k: v.cpu().numpy()[pick] for k, v in out.items()}
+    hosts = tuple(host_bits(t[pick]) for t in (zd, zq, zt))
+    tok_h = tok.cpu().numpy()[pick]
+    orc = oracle.verify(*hosts, tok_h, np.float32(w.tau_q), np.float32(w.tau_t), 0, 0, 2, n_threads=8, seq_ids=pick)
+    ties, n = check_pyramid(oracle, gpu, orc, hosts, "bf16", 0, w.tau_q, w.tau_t, 0, 2, tok_h, seq_ids=pick)
+    assert ties <= 1 and n >= 3
+    # properties that hold for every sequence at any size
+    al_q, nt_q = out["accept_len_q"].cpu().numpy(), out["next_token_q"].cpu().numpy()
+    al, nt = out["accept_len"].cpu().numpy(), out["next_token"].cpu().numpy()
+    assert np.all((0 <= al_q) & (al_q <= w.K_d)) and np.all((nt_q >= 0) == (al_q < w.K_d))
+    n2 = np.minimum(w.K_q, al_q + (nt_q >= 0))
+    assert np.all(al <= n2) and np.all((nt >= 0) == (al < n2)) and np.all(nt < w.V)

@@ -389,3 +389,16 @@ def test_mixed_stage_equals_plain_stage_on_same_values(oracle):
     b = oracle.verify_stage(zs.double().numpy(), zl.double().numpy(), tok, 0.3, seed=2, offset=9)
     assert np.array_equal(a["accept_len"], b["accept_len"]) and np.array_equal(a["next_token"], b["next_token"])
     np.testing.assert_array_equal(a["div"], b["div"])
+
+
+def test_seq_ids_select_the_philox_rows_of_the_full_batch(oracle):
+    rng = np.random.default_rng(12)
+    B, K, V = 6, 3, 24
+    zl = rng.normal(0, 2, (B, K, V))
+    zs = zl + rng.normal(0, 1, (B, K, V))
+    tok = rng.integers(0, V, (B, K))
+    full = oracle.verify_stage(zs, zl, tok, 0.0, mode=oracle.STRICT, seed=4, offset=2)
+    pick = [4, 1]
+    part = oracle.verify_stage(zs[pick], zl[pick], tok[pick], 0.0, mode=oracle.STRICT, seed=4, offset=2, seq_ids=pick)
+    assert np.array_equal(part["accept_len"], full["accept_len"][pick])
+    assert np.array_equal(part["next_token"], full["next_token"][pick])
