@@ -105,6 +105,7 @@ typedef struct psd_stage_args {
   void* stream;                  /* cudaStream_t, or NULL for the stream set by pyramidsd_set_stream */
   int32_t use_stream_field;      /* non-zero: take `stream` even when it is NULL (the legacy default stream) */
   int32_t kernel_variant;        /* psd_kernel_variant */
+  int32_t cluster_size;          /* CTAs per cluster for the cluster kernel (power of two <= 16); 0 = chosen by the library */
 } psd_stage_args;
 
 /* One verification stage (Sec. 3.1 for one model pair; Sec. 3.2 applies it twice). Jensen-Shannon
@@ -171,9 +172,10 @@ int pyramidsd_kernel_timing_end(double* ms_rowstats, int* n_rowstats, double* ms
 /* Number of kernels the library has launched from this process since load (all entry points). */
 uint64_t pyramidsd_launch_count(void);
 
-/* Largest number of co-resident clusters the device grants the cluster kernel for this shape (0 when
- * the variant does not apply); lets a caller size batches to whole waves. */
-int pyramidsd_cluster_occupancy(int V, psd_dtype dtype, int* out_cluster_size, int* out_max_active_clusters);
+/* The cluster size (CTAs per row pair) the library picks for a [B, K, V] stage of this dtype and the
+ * number of such clusters the current device keeps resident at once; 0 and 0 when the shape takes the
+ * baseline kernel. Lets a caller size batches to whole waves. Needs a CUDA device. */
+int pyramidsd_cluster_occupancy(int B, int K, int V, psd_dtype dtype, int* out_cluster_size, int* out_max_active_clusters);
 
 const char* pyramidsd_version(void);
 const char* pyramidsd_status_string(int status);

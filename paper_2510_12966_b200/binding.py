@@ -44,6 +44,7 @@ class StageArgs(C.Structure):
         ("out_resid_mass", C.c_void_p), ("out_row_flags", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("stream", C.c_void_p), ("use_stream_field", C.c_int32), ("kernel_variant", C.c_int32),
+        ("cluster_size", C.c_int32),
     ]
 
 
@@ -90,7 +91,7 @@ def load_library(path: Optional[str] = None):
     lib.pyramidsd_kernel_timing_end.restype = i32
     lib.pyramidsd_launch_count.argtypes = []
     lib.pyramidsd_launch_count.restype = u64
-    lib.pyramidsd_cluster_occupancy.argtypes = [i32, i32, C.POINTER(i32), C.POINTER(i32)]
+    lib.pyramidsd_cluster_occupancy.argtypes = [i32, i32, i32, i32, C.POINTER(i32), C.POINTER(i32)]
     lib.pyramidsd_cluster_occupancy.restype = i32
     lib.pyramidsd_version.restype = C.c_char_p
     lib.pyramidsd_status_string.argtypes = [i32]
@@ -163,9 +164,10 @@ def workspace_bytes(B: int, K: int, V: int, dtype: int) -> int:
     return int(load_library().pyramidsd_workspace_bytes(B, K, V, dtype))
 
 
-def cluster_occupancy(V: int, dtype: int):
+def cluster_occupancy(B: int, K: int, V: int, dtype: int):
+    """(cluster size, co-resident clusters) the library uses for this stage shape; (0, 0) = baseline kernel."""
     cs, n = C.c_int(0), C.c_int(0)
-    _check(load_library().pyramidsd_cluster_occupancy(V, dtype, C.byref(cs), C.byref(n)), "pyramidsd_cluster_occupancy")
+    _check(load_library().pyramidsd_cluster_occupancy(B, K, V, dtype, C.byref(cs), C.byref(n)), "pyramidsd_cluster_occupancy")
     return cs.value, n.value
 
 
@@ -200,7 +202,7 @@ def verify_stage(logits_small, logits_large, draft_tokens, threshold, mode=FUZZY
 def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
                     B=None, K=None, V=None, n_valid=None, inv_temperature=0.0, div_kind=DIV_JS,
                     seq_stride_small=0, seq_stride_large=0, want_rows=True, workspace=None, stream=None,
-                    kernel_variant=KERNEL_AUTO, raise_on_error=True):
+                    kernel_variant=KERNEL_AUTO, cluster_size=0, raise_on_error=True):
     """``pyramidsd_verify_stage_ex``: every option exposed. Returns a dict of device tensors (+ "status")."""
     if B is None:
         B, K, V = logits_small.shape
@@ -239,6 +241,7 @@ def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, p
     a.stream = s.cuda_stream
     a.use_stream_field = 1
     a.kernel_variant = int(kernel_variant)
+    a.cluster_size = int(cluster_size)
     rc = load_library().pyramidsd_verify_stage_ex(C.byref(a))
     out["status"] = rc
     if raise_on_error:

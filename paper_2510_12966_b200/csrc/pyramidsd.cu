@@ -134,18 +134,22 @@ int check_launch() {
 }
 
 // Statistics pass for one stage: picks the kernel variant and launches it.
-int launch_rowstats(const StageParams& P, int dtype, int variant, cudaStream_t stream) {
+int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_size, cudaStream_t stream) {
   const long long rows = static_cast<long long>(P.B) * P.K;
   if (rows == 0) return PSD_OK;
   bool use_cluster = false;
+  psd::ClusterGeom geom{};
   if (variant == PSD_KERNEL_CLUSTER || variant == PSD_KERNEL_AUTO) {
-    use_cluster = psd::cluster_kernel_applicable(P, dtype);
+    use_cluster = psd::cluster_geometry(P, dtype, cluster_size, &geom);
     if (!use_cluster && variant == PSD_KERNEL_CLUSTER) return PSD_ERR_UNSUPPORTED;
   }
   TimedLaunch timed(stream, 0);
   if (use_cluster) {
-    const int rc = psd::launch_rowstats_cluster(P, dtype, stream);
-    if (rc != PSD_OK) return rc;
+    if (psd::launch_rowstats_cluster(P, dtype, geom, stream) != 0) {
+      const cudaError_t e = cudaGetLastError();
+      std::fprintf(stderr, "pyramidsd: cluster kernel launch failed: %s\n", cudaGetErrorString(e));
+      return PSD_ERR_CUDA;
+    }
   } else {
     const dim3 grid(static_cast<unsigned>(rows)), block(1024);
     if (dtype == PSD_F32) psd::rowstats_baseline_kernel<float><<<grid, block, 0, stream>>>(P);
@@ -169,6 +173,7 @@ int validate_stage(const psd_stage_args* a) {
   if (a == nullptr || a->struct_size != sizeof(psd_stage_args)) return PSD_ERR_INVALID_ARG;
   if (!valid_dtype(a->dtype) || !valid_mode(a->mode) || !valid_div(a->div_kind)) return PSD_ERR_INVALID_ARG;
   if (a->B < 0 || a->K < 0 || a->K > 32 || a->V < 1) return PSD_ERR_INVALID_ARG;
+  if (a->kernel_variant < PSD_KERNEL_AUTO || a->kernel_variant > PSD_KERNEL_CLUSTER || a->cluster_size < 0) return PSD_ERR_INVALID_ARG;
   if (a->V > kMaxV) return PSD_ERR_UNSUPPORTED;
   if (static_cast<long long>(a->B) * a->K > (1ll << 30)) return PSD_ERR_UNSUPPORTED;
   if (a->inv_temperature < 0.f || std::isnan(a->inv_temperature) || std::isinf(a->inv_temperature)) return PSD_ERR_INVALID_ARG;
@@ -251,7 +256,7 @@ int run_stage(const psd_stage_args* a, int32_t* window_out, int32_t* n_window_ou
   P.K_window = K_window;
   const cudaStream_t stream = pick_stream(a);
   if (a->K > 0) {
-    rc = launch_rowstats(P, a->dtype, a->kernel_variant, stream);
+    rc = launch_rowstats(P, a->dtype, a->kernel_variant, a->cluster_size, stream);
     if (rc != PSD_OK) return rc;
   }
   return launch_finalize(P, a->dtype, stream);
@@ -473,9 +478,21 @@ int pyramidsd_kernel_timing_end(double* ms_rowstats, int* n_rowstats, double* ms
 
 uint64_t pyramidsd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-int pyramidsd_cluster_occupancy(int V, psd_dtype dtype, int* out_cluster_size, int* out_max_active_clusters) {
-  if (V < 1 || !valid_dtype(dtype)) return PSD_ERR_INVALID_ARG;
-  return psd::cluster_occupancy(V, dtype, out_cluster_size, out_max_active_clusters);
+int pyramidsd_cluster_occupancy(int B, int K, int V, psd_dtype dtype, int* out_cluster_size, int* out_max_active_clusters) {
+  if (B < 0 || K < 0 || K > 32 || V < 1 || !valid_dtype(dtype)) return PSD_ERR_INVALID_ARG;
+  StageParams P{};
+  P.B = B; P.K = K; P.V = V;
+  P.seq_stride_small = P.seq_stride_large = static_cast<long long>(K) * V;
+  P.div_kind = PSD_DIV_JS;
+  psd::ClusterGeom g{};
+  const bool ok = B > 0 && K > 0 && psd::cluster_geometry(P, dtype, 0, &g);
+  if (out_cluster_size) *out_cluster_size = ok ? g.cs : 0;
+  if (out_max_active_clusters) {
+    int log2cs = 0;
+    while (ok && (1 << log2cs) < g.cs) ++log2cs;
+    *out_max_active_clusters = ok ? psd::cluster_max_active_any(dtype, PSD_DIV_JS, log2cs) : 0;
+  }
+  return PSD_OK;
 }
 
 const char* pyramidsd_version(void) { return "pyramidsd-b200 0.1.0 (sm_100a)"; }

@@ -32,13 +32,14 @@ def wl():
 
 
 def run_stage_both(psd, oracle, zs, zl, tok, tau, mode=0, seed=0, offset=0, n_valid=None, inv_temperature=0.0,
-                   div_kind=0, variant=0):
+                   div_kind=0, variant=0, cluster_size=0):
     """Library on the GPU, oracle on the host, same bits. Returns (gpu dict, oracle dict, report)."""
     dev = torch.device("cuda:0")
     zs_d, zl_d, tok_d = zs.to(dev), zl.to(dev), tok.to(dev)
     nv_d = None if n_valid is None else torch.as_tensor(n_valid, dtype=torch.int32, device=dev)
     out = psd.verify_stage_ex(zs_d, zl_d, tok_d, tau, mode, seed, offset, n_valid=nv_d,
-                              inv_temperature=inv_temperature, div_kind=div_kind, kernel_variant=variant)
+                              inv_temperature=inv_temperature, div_kind=div_kind, kernel_variant=variant,
+                              cluster_size=cluster_size)
     torch.cuda.synchronize()
     assert psd.last_status() == 0
     gpu = gpu_stage_to_numpy(out)
@@ -199,6 +200,89 @@ def test_results_are_bit_identical_run_to_run(psd, wl):
             for k in ref:
                 assert torch.equal(ref[k].view(torch.int32), cur[k].view(torch.int32)), k
         ref = cur
+
+
+# -------------------------------------------------------------------------------------------------- cluster kernel
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("cs", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("V", [2048, 8200, 32000, 128256])
+def test_cluster_kernel_every_cluster_size(psd, oracle, wl, dtype, cs, V):
+    """The cluster kernel with the cluster size forced: slices with ragged tails, empty slices (small V
+    over many CTAs), one and several chunks per slice; shapes it cannot hold are refused, not run."""
+    B, K = 3, 5
+    zs, zl, tok = wl.make_stage_inputs(B, K, V, dtype, seed=300 + V + cs, sigma=0.8)
+    dev = torch.device("cuda:0")
+    es = 4 if dtype == "f32" else 2
+    chunks = -(-(-(-V // cs)) // (8192 // es))
+    out = psd.verify_stage_ex(zs.to(dev), zl.to(dev), tok.to(dev), 0.1, kernel_variant=psd.KERNEL_CLUSTER,
+                              cluster_size=cs, raise_on_error=False)
+    if chunks > 12:
+        assert out["status"] == psd.ERR_UNSUPPORTED
+        return
+    assert out["status"] == 0
+    for tau in (0.02, 0.3):
+        _, _, rep = run_stage_both(psd, oracle, zs, zl, tok, tau, seed=V, offset=cs, variant=psd.KERNEL_CLUSTER,
+                                   cluster_size=cs)
+        assert rep["tie_div"] + rep["tie_cdf"] <= 1
+
+
+@pytest.mark.parametrize("dtype,V,B,K", [("bf16", 32768, 48, 8), ("f32", 16384, 40, 7), ("bf16", 128256, 24, 16)])
+def test_cluster_kernel_many_rows_per_cluster(psd, oracle, wl, dtype, V, B, K):
+    """More rows than resident clusters: every cluster walks several rows, so the ring, the exchange
+    buffers and the barrier phases wrap around. Also checked against the baseline kernel."""
+    zs, zl, tok = wl.make_stage_inputs(B, K, V, dtype, seed=400 + B, boost=(4.0, 12.0), sigma=0.7)
+    cs = 1 if V <= 32768 and dtype == "bf16" else 0
+    nv = [(3 * b) % (K + 1) for b in range(B)]
+    g1, orc, rep = run_stage_both(psd, oracle, zs, zl, tok, 0.15, mode=2, seed=4, offset=9, n_valid=nv,
+                                  variant=psd.KERNEL_CLUSTER, cluster_size=cs)
+    g2, _, _ = run_stage_both(psd, oracle, zs, zl, tok, 0.15, mode=2, seed=4, offset=9, n_valid=nv,
+                              variant=psd.KERNEL_BASELINE)
+    valid = np.arange(K)[None, :] < np.asarray(nv)[:, None]
+    tol = TOL[dtype]["val"]
+    assert np.abs(g1["div"][valid] - g2["div"][valid]).max() < tol
+    assert np.abs(g1["resid_mass"][valid] - g2["resid_mass"][valid]).max() < tol
+    assert rep["tie_div"] + rep["tie_coin"] + rep["tie_cdf"] <= 2
+
+
+def test_cluster_kernel_masked_flagged_and_identical_rows(psd, oracle, wl):
+    B, K, V = 4, 3, 16384
+    zs, zl, tok = wl.make_stage_inputs(B, K, V, "bf16", seed=31, sigma=0.3)
+    zs[0, 1, 100:9000] = -float("inf")          # masked vocabulary on one side, across a chunk boundary
+    zl[1, 0, :] = -float("inf")
+    zl[1, 0, 12345] = 2.0                        # a single live token
+    zs[2, 1, 17] = float("nan")
+    zl[3, 0, V - 1] = float("inf")
+    zl[3, 2] = zs[3, 2]                          # bitwise identical pair
+    zs[0, 0, :4096] = -3.0e38                    # huge negative finite logits
+    for cs in (1, 2):
+        gpu, orc, _ = run_stage_both(psd, oracle, zs, zl, tok, 1.0, variant=psd.KERNEL_CLUSTER, cluster_size=cs)
+        assert gpu["next_token"][2] == -2 and gpu["accept_len"][2] == 1
+        assert gpu["next_token"][3] == -2 and gpu["accept_len"][3] == 0
+        assert gpu["next_token"][1] == 12345 or gpu["accept_len"][1] > 0
+        assert np.all(np.isfinite(gpu["div"][0])) and np.all(np.isfinite(gpu["div"][1]))
+    zs2, zl2, tok2 = wl.make_stage_inputs(1, 3, 4096, "f32", seed=32)
+    zl2[0, 0, :] = -float("inf")                 # a row with no finite entry is flagged
+    zl2[0, 2] = zs2[0, 2]
+    gpu, _, _ = run_stage_both(psd, oracle, zs2, zl2, tok2, 1.0, variant=psd.KERNEL_CLUSTER, cluster_size=2)
+    assert gpu["row_flags"][0, 0] == 2 and gpu["next_token"][0] == -2
+
+
+@pytest.mark.parametrize("div_kind", [1, 2])
+def test_cluster_kernel_other_divergences(psd, oracle, wl, div_kind):
+    zs, zl, tok = wl.make_stage_inputs(4, 4, 20000, "f32", seed=8, sigma=0.5)
+    tau = 0.3 if div_kind == 1 else 0.5
+    run_stage_both(psd, oracle, zs, zl, tok, tau, div_kind=div_kind, variant=psd.KERNEL_CLUSTER)
+    zs, zl, tok = wl.make_stage_inputs(4, 4, 20000, "bf16", seed=8, sigma=0.5)
+    zs[1, 1, 50:60] = -float("inf")             # KL(large || small) is +inf where small has no mass
+    run_stage_both(psd, oracle, zs, zl, tok, tau, div_kind=div_kind, variant=psd.KERNEL_CLUSTER)
+
+
+def test_cluster_occupancy_query(psd):
+    cs, n = psd.cluster_occupancy(64, 16, 128256, psd.BF16)
+    assert cs == 4 and n >= 16
+    cs, n = psd.cluster_occupancy(1, 4, 32000, psd.F32)
+    assert cs >= 2 and n >= 1
+    assert psd.cluster_occupancy(4, 4, 1001, psd.F32) == (0, 0)
 
 
 # -------------------------------------------------------------------------------------------------- wrapper
