@@ -118,13 +118,16 @@ def run_ours(args):
     binding.load_library()
     binding.set_stream()
     cfg, w = workload_from_name(args.workload)
+    if args.batch > 0:
+        import dataclasses
+        w = dataclasses.replace(w, B=args.batch, name=f"{w.name}[B={args.batch}]")
     es = 2 if w.dtype == "bf16" else 4
 
     # Each rank owns its own batch of B sequences (weak scaling; sequences are independent, no collective
     # on the data path). Two distinct rounds alternate so that a step never re-reads a buffer it just used;
     # one round (788 MB for cfg3) already exceeds the 126 MB L2.
     n_bufs = 2
-    rounds = [workloads.workload_inputs(cfg, 100 * rank + i, device=dev) for i in range(n_bufs)]
+    rounds = [workloads.workload_inputs(cfg, 100 * rank + i, device=dev, B=w.B) for i in range(n_bufs)]
     outs = [{k: torch.empty(w.B, dtype=torch.int32, device=dev)
              for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")} for _ in range(n_bufs)]
     mode, seed = binding.FUZZY, 0
@@ -230,7 +233,7 @@ def run_ours(args):
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": e2e["ms"] / e2e["steps"], "steps": e2e["steps"]}
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w, cfg, rounds[0], seqs=args.cpu_seqs)
+            line["cpu_baseline"] = cpu_baseline(w, rounds)
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
         traffic = read_profile_traffic(w)
         if traffic is not None:
@@ -252,20 +255,24 @@ def read_profile_traffic(w):
     return None if per_row is None else per_row * w.B * w.K_d
 
 
-def cpu_baseline(w, cfg, round_inputs, seqs):
-    """The CPU oracle, as it stands, on a bounded sample (the first `seqs` sequences of one round)."""
+def cpu_baseline(w, rounds):
+    """The CPU oracle, as it stands, on a bounded sample: the resident rounds of the workload (two rounds
+    of B sequences each), one oracle call per round on all host cores."""
     import oracle
     from paper_2510_12966_b200 import workloads
     oracle.build()
-    zd, zq, zt, tok = [workloads.to_host_bits(t[:seqs]) for t in round_inputs]
     cores = os.cpu_count() or 1
-    t0 = time.perf_counter()
-    out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, n_threads=cores)
-    dt = time.perf_counter() - t0
-    n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
-    pos = seqs * w.K_d + int(n2.sum())
+    pos, dt = 0, 0.0
+    for r in rounds:
+        zd, zq, zt, tok = [workloads.to_host_bits(t) for t in r]
+        t0 = time.perf_counter()
+        out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, n_threads=cores)
+        dt += time.perf_counter() - t0
+        n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
+        pos += w.B * w.K_d + int(n2.sum())
     return {"value": pos / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {seqs} sequences of one {w.name} round ({pos} positions, {dt:.2f} s wall)"}
+            "sample": f"{len(rounds)} rounds of {w.name} ({w.B} sequences each, {pos} positions, {dt:.2f} s wall, "
+                      f"about {dt * cores:.0f} core-seconds)"}
 
 
 def run_reference(args):
@@ -315,7 +322,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
-    ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences in the CPU-oracle sample")
+    ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences per step of the CPU-oracle reference arm")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (small profiling cases)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -8,24 +8,29 @@
 //   pass B  with the row's normalisers known: p, q, the Jensen-Shannon terms and the residual mass.
 // Pass B of a row needs the normalisers of the WHOLE row, so the CTAs of a cluster exchange their
 // (reference, sum) partials through distributed shared memory. Nothing waits on that exchange in line:
-// the ring holds more than one row slice, each warp runs pass A ahead of pass B for as long as loaded
-// chunks are available, and an agent warp carries partials between CTAs. Warps are independent of each
-// other; they meet only on mbarriers (chunk landed / chunk free / row partials complete).
+// the ring holds more than one row slice, the pass-A warps run ahead of the pass-B warps for as long as
+// loaded chunks are available, and an agent warp carries partials between CTAs. Warps are independent
+// of each other; they meet only on mbarriers (chunk landed / chunk free / row partials complete), and
+// every one of those waits is a blocking mbarrier wait on a single condition.
 //
-// Roles: warps 0..15 consumers (each owns 32 consecutive 16-byte vectors of every chunk), warp 16 lane 0
-// issues the bulk copies, warp 17 is the agent (reduces the warps' partials, talks to the peers; on
-// rank 0 it also writes the row's RowStats). Every wait is bounded: on giving up a thread records
-// PSD_ERR_TIMEOUT in the status word and stops waiting, so the kernel always terminates.
+// Roles: warps 0..7 run pass A, warps 8..15 run pass B (each warp owns 2 x 32 16-byte vectors of every
+// chunk and model; the hardware scheduler interleaves the two instruction streams on each SM
+// sub-partition), warp 16 lane 0 issues the bulk copies, warp 17 is the agent (reduces the warps'
+// partials, talks to the peers; on rank 0 it also writes the row's RowStats). Every wait is bounded: on
+// giving up a thread records PSD_ERR_TIMEOUT in the status word and stops waiting, so the kernel always
+// terminates.
 #pragma once
 
 #include "common.cuh"
 
 namespace psd {
 
-constexpr int kClConsumerWarps = 16;
+constexpr int kClPassWarps = 8;                    // warps per pass (A: 0..7, B: 8..15)
+constexpr int kClConsumerWarps = 2 * kClPassWarps;
 constexpr int kClConsumers = kClConsumerWarps * 32;
 constexpr int kClThreads = kClConsumers + 64;      // + loader warp + agent warp
-constexpr int kClHalfBytes = 8192;                 // one model's part of a chunk: 512 threads x 16 bytes
+constexpr int kClHalfBytes = 8192;                 // one model's part of a chunk: 256 threads x 2 x 16 bytes
+constexpr int kClVecPerLane = 2;                   // 16-byte vectors per lane, chunk and model
 constexpr int kClSlotBytes = 2 * kClHalfBytes;
 constexpr int kClSlots = 13;                       // ring slots
 constexpr int kClDepth = 4;                        // rows of exchange buffers in flight
@@ -40,14 +45,23 @@ struct ClusterGeom {
   int n_clusters;
 };
 
+// Per-row constants of pass B: -log2 of the normalisers in the scaled base-2 domain and the clamp floors.
+struct __align__(16) RowConsts {
+  float off_small, off_large;        // log2(sum_i exp(z_i / T)) of each model
+  float floor_small, floor_large;    // logits below these would give log2 p < -125
+  unsigned floor2_small, floor2_large;   // the same floors as packed bf16 pairs
+  unsigned pad0, pad1;
+};
+
 // Shared-memory control block behind the ring.
 struct __align__(16) ClusterCtl {
   unsigned long long full[kClSlots];
   unsigned long long empty[kClSlots];
-  unsigned long long a_done[kClDepth], b_done[kClDepth], lse_ready[kClDepth], fin_ready[kClDepth];
-  float4 a_part[kClDepth][kClConsumerWarps];       // (ref_small, sum_small, ref_large, sum_large) per warp
-  double b_part[kClDepth][kClConsumerWarps][4];    // (sum p*a + q*b, sum s*lg s, sum max(p,q), differ bits)
+  unsigned long long a_done[kClDepth], b_done[kClDepth], lse_ready[kClDepth], fin_ready[kClDepth], b_go[kClDepth];
+  float4 a_part[kClDepth][kClPassWarps];           // (ref_small, sum_small, ref_large, sum_large) per pass-A warp
+  float4 b_part[kClDepth][kClPassWarps];           // (divergence sum in bits, sum max(p,q), rows differ, unused) per pass-B warp
   float4 row_lse[kClDepth];                        // (m2_small, l2s_small, m2_large, l2s_large) of the row
+  RowConsts row_consts[kClDepth];                  // what pass B needs of the row, published by the agent
   float4 lse_in[kClDepth][kClMaxRanks];            // partials received from every rank of the cluster
   double fin_in[kClDepth][kClMaxRanks][4];         // pass-B partials received (rank 0 only)
 };
@@ -66,19 +80,28 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// non-blocking: has the phase with this parity completed?
 __device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned parity) {
   unsigned ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+  asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
 // same, observing writes made by other CTAs of the cluster before their arrive
 __device__ __forceinline__ bool mbar_test_cluster(unsigned long long* bar, unsigned parity) {
   unsigned ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+  asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// may suspend the thread for a hardware-chosen time before answering
+__device__ __forceinline__ bool mbar_try(unsigned long long* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void fence_acquire_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 __device__ __forceinline__ unsigned map_to_rank(const void* local, unsigned rank) {
   unsigned r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(local)), "r"(rank));
@@ -143,32 +166,128 @@ __device__ __forceinline__ const T* row_ptr(const void* base, long long seq_stri
   return static_cast<const T*>(base) + b * seq_stride + static_cast<long long>(k) * V;
 }
 
-// ---- pass A: streaming log-sum-exp -------------------------------------------------------------------
-// State per thread and model: a reference `ref` (in the scaled base-2 domain), the sum S of 2^(x*c - ref)
-// and `thr`, the largest logit that may still be added without moving the reference (ref + 64 in the
-// scaled domain). The reference starts at a finite floor so that -inf logits give exactly 0.
-struct LseState {
-  float ref, thr, s0, s1;
-  __device__ __forceinline__ void reset(float inv_c) { ref = -1e30f; thr = (-1e30f + 64.f) * inv_c; s0 = 0.f; s1 = 0.f; }
+// ---- packed fp32 pairs: float2 through the sm_100 packed add / mul / fma (one issue slot for two lanes) ----
+__device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float2 ex2_2(float2 v) { return make_float2(ex2_approx(v.x), ex2_approx(v.y)); }
+
+// One 16-byte vector of logits as packed pairs of consecutive vocabulary indices.
+template <typename T> struct Pairs;
+template <> struct Pairs<float> {
+  static constexpr int kN = 2;
+  __device__ static __forceinline__ void load(const uint4& u, float2 (&x)[2]) {
+    x[0] = make_float2(__uint_as_float(u.x), __uint_as_float(u.y));
+    x[1] = make_float2(__uint_as_float(u.z), __uint_as_float(u.w));
+  }
+  // the same with every logit raised to at least `floor_x`
+  __device__ static __forceinline__ void load_clamped(const uint4& u, float floor_x, unsigned, float2 (&x)[2]) {
+    x[0] = make_float2(fmaxf(__uint_as_float(u.x), floor_x), fmaxf(__uint_as_float(u.y), floor_x));
+    x[1] = make_float2(fmaxf(__uint_as_float(u.z), floor_x), fmaxf(__uint_as_float(u.w), floor_x));
+  }
+  __device__ static __forceinline__ unsigned floor_bits(float) { return 0u; }
+};
+template <> struct Pairs<__nv_bfloat16> {
+  static constexpr int kN = 4;
+  // bf16 is the upper half of a binary32: widen by shifting / masking
+  __device__ static __forceinline__ float2 widen(unsigned w) {
+    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+  }
+  __device__ static __forceinline__ void load(const uint4& u, float2 (&x)[4]) {
+    x[0] = widen(u.x); x[1] = widen(u.y); x[2] = widen(u.z); x[3] = widen(u.w);
+  }
+  __device__ static __forceinline__ unsigned max_bf16x2(unsigned a, unsigned b) {
+    unsigned r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+  }
+  // the clamp runs on the packed bf16 words, one instruction per two logits
+  __device__ static __forceinline__ void load_clamped(const uint4& u, float, unsigned floor2, float2 (&x)[4]) {
+    x[0] = widen(max_bf16x2(u.x, floor2)); x[1] = widen(max_bf16x2(u.y, floor2));
+    x[2] = widen(max_bf16x2(u.z, floor2)); x[3] = widen(max_bf16x2(u.w, floor2));
+  }
+  // `floor_x` rounded up to bf16, in both halves of a word
+  __device__ static __forceinline__ unsigned floor_bits(float floor_x) {
+    unsigned b = __float_as_uint(floor_x);
+    if (floor_x == floor_x && fabsf(floor_x) < INFINITY) {
+      const unsigned low = b & 0xffffu;
+      b &= 0xffff0000u;
+      if (low != 0u && floor_x > 0.f) b += 0x10000u;   // towards +inf; negative values round up by truncation
+    } else {
+      b = 0xff800000u;                                  // no usable floor: -inf clamps nothing
+    }
+    return (b >> 16) | (b & 0xffff0000u);
+  }
 };
 
-template <int E>
-__device__ __forceinline__ void lse_accumulate(const float (&x)[E], float c, float inv_c, LseState& st) {
-  float gm = x[0];
+// ---- pass A: streaming log-sum-exp -------------------------------------------------------------------
+// State per warp and model: a reference `ref` in the scaled base-2 domain, the same in every lane, and
+// per lane the sum S of 2^(x*c - ref). No running maximum is kept: the exps of one vector are summed on
+// their own, and only when some lane's vector sum is not finite (a logit more than 2^127 above the
+// reference, which includes the first finite vector of a row because the reference starts at -1e30, or a
+// NaN / +inf logit) does the warp take the slow path, which moves the reference to the warp's maximum of
+// that vector and redoes it. The finite starting reference makes -inf logits (masked vocabulary)
+// contribute exactly 0. With one reference per warp the row-end reduction is a plain sum.
+struct LseState {
+  float ref, s;
+  __device__ __forceinline__ void reset() { ref = -1e30f; s = 0.f; }
+};
+
+// sum of 2^(x*c - ref) over one 16-byte vector; `live` false (vector outside the slice) gives 0
+template <typename T>
+__device__ __forceinline__ float lse_vector_sum(const uint4& u, float c, float ref) {
+  constexpr int N = Pairs<T>::kN;
+  float2 x[N];
+  Pairs<T>::load(u, x);
+  const float2 cc = splat2(c), nref = splat2(-ref);
+  float2 v = ex2_2(__ffma2_rn(x[0], cc, nref));
 #pragma unroll
-  for (int j = 1; j < E; ++j) gm = fmaxf(gm, x[j]);
-  if (gm > st.thr) {  // rare: the group holds a logit far above the reference (always true for the first finite group)
-    const float nr = gm * c;
-    const float sc = ex2_approx(st.ref - nr);
-    st.s0 *= sc; st.s1 *= sc;
-    st.ref = nr;
-    st.thr = gm + 64.f * inv_c;
+  for (int j = 1; j < N; ++j) v = __fadd2_rn(v, ex2_2(__ffma2_rn(x[j], cc, nref)));
+  return v.x + v.y;
+}
+
+// Warp-wide: move the reference up to the largest logit of this vector (over the live lanes) and
+// return this lane's vector sum against the new reference.
+template <typename T>
+__device__ __noinline__ float lse_slow_path(uint4 u, bool live, float c, float ref_in, float s_in, float* ref_out,
+                                            float* s_out) {
+  constexpr int N = Pairs<T>::kN;
+  float2 x[N];
+  Pairs<T>::load(u, x);
+  float gm = -INFINITY;
+  if (live) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) gm = fmaxf(gm, fmaxf(x[j].x, x[j].y));
   }
 #pragma unroll
-  for (int j = 0; j < E; j += 2) {
-    st.s0 += ex2_approx(fmaf(x[j], c, -st.ref));
-    st.s1 += ex2_approx(fmaf(x[j + 1], c, -st.ref));
+  for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
+  const float nr = gm * c;
+  float ref = ref_in, s = s_in;
+  if (nr > ref) {   // false for NaN; +inf poisons the sum below, as it should
+    s *= ex2_approx(ref - nr);
+    ref = nr;
   }
+  float t = 0.f;
+  if (live) {
+#pragma unroll
+    for (int j = 0; j < N; ++j) t += ex2_approx(fmaf(x[j].x, c, -ref)) + ex2_approx(fmaf(x[j].y, c, -ref));
+  }
+  *ref_out = ref;
+  *s_out = s;
+  return t;
+}
+
+// Add one vector sum, taken against `ref_used`, to the state; all 32 lanes call this together. When an
+// earlier vector of the same step has moved the reference the sum is taken again, so that the result
+// does not depend on how many vectors a step happened to group.
+template <typename T>
+__device__ __forceinline__ void lse_commit(float t, float ref_used, const uint4& u, bool live, float c, LseState& st) {
+  if (st.ref != ref_used) t = lse_vector_sum<T>(u, c, st.ref);
+  if (__any_sync(0xffffffffu, live && !(t < INFINITY))) {
+    float r2, s2;
+    t = lse_slow_path<T>(u, live, c, st.ref, st.s, &r2, &s2);
+    st.ref = r2;
+    st.s = s2;
+  }
+  st.s += live ? t : 0.f;
 }
 
 // Combine (ref, S) partials: returns the pair for the union. Fixed order, NaN-preserving in S.
@@ -178,32 +297,57 @@ __device__ __forceinline__ void lse_merge(float& ref, float& s, float oref, floa
   ref = m;
 }
 
-// ---- pass B accumulators ----------------------------------------------------------------------------
+// ---- pass B ------------------------------------------------------------------------------------------
+// With a = log2 p and b = log2 q (both linear in the logits once the normalisers are known), each
+// vocabulary index adds to the Jensen-Shannon divergence, in bits and before the factor 1/2,
+//     p lg p + q lg q - (p + q) lg((p + q) / 2)  =  2^M * h(d),   M = max(a, b),  d = -|a - b|,
+//     h(d) = u d + psi(u),   u = 2^d in (0, 1],   psi(u) = (1 + u) (1 - lg(1 + u)),
+// which costs two ex2 (2^M and 2^d) and a polynomial for psi instead of two ex2 and one lg2 plus
+// cancelling sums: every term is >= 0 (h(0) = 0 for equal probabilities, h -> 1 when one side vanishes).
+// 2^M is max(p, q), so the residual mass sum max(0, p - q) = sum max(p, q) - 1 falls out of the same ex2.
+// psi is a degree-7 minimax polynomial on [0, 1] (max abs error 5.6e-8, a least-squares/Remez fit).
+// Logits arrive clamped from below so that a, b >= -125: nothing is -inf, NaN cannot arise, and the terms
+// clamped away are below 2^-125.
+__device__ __forceinline__ float2 psi_poly(float2 u) {
+  float2 p = __ffma2_rn(splat2(3.571110749e-03f), u, splat2(-1.966644044e-02f));
+  p = __ffma2_rn(p, u, splat2(5.437676601e-02f));
+  p = __ffma2_rn(p, u, splat2(-1.133036196e-01f));
+  p = __ffma2_rn(p, u, splat2(2.388960843e-01f));
+  p = __ffma2_rn(p, u, splat2(-7.211711122e-01f));
+  p = __ffma2_rn(p, u, splat2(-4.427027888e-01f));
+  p = __ffma2_rn(p, u, splat2(1.000000056e+00f));
+  return p;
+}
+
 struct DivAcc {
-  float pa, qb, sl, big;
-  unsigned differ;
-  __device__ __forceinline__ void reset() { pa = qb = sl = big = 0.f; differ = 0u; }
+  float2 js, big;    // sum 2^M h(d); sum 2^M
+  unsigned differ;   // OR of (small bits XOR large bits)
+  __device__ __forceinline__ void reset() { js = big = make_float2(0.f, 0.f); differ = 0u; }
 };
 
-template <int DIV, int E>
-__device__ __forceinline__ void div_accumulate(const float (&xl_in)[E], const float (&xs_in)[E], float c, float off_l,
+template <int DIV, int N>
+__device__ __forceinline__ void div_accumulate(const float2 (&xl)[N], const float2 (&xs)[N], float c, float off_l,
                                                float off_s, DivAcc& acc) {
+  const float2 cc = splat2(c), nl = splat2(-off_l), ns = splat2(-off_s);
 #pragma unroll
-  for (int j = 0; j < E; ++j) {
-    // -inf (masked vocabulary) and huge negative logits: clamp so that 0 * log 0 stays 0
-    const float xl = fmaxf(xl_in[j], -1e30f), xs = fmaxf(xs_in[j], -1e30f);
-    const float a = fmaf(xl, c, -off_l), b = fmaf(xs, c, -off_s);   // log2 p, log2 q
-    const float p = ex2_approx(a), q = ex2_approx(b);
-    acc.big += fmaxf(p, q);
-    if (DIV == kDivJS) {
-      const float s = p + q;
-      const float l = lg2_approx(s + 1e-36f);
-      acc.pa = fmaf(p, a, acc.pa);
-      acc.qb = fmaf(q, b, acc.qb);
-      acc.sl = fmaf(s, l, acc.sl);
-    } else if (DIV == kDivKL) {
-      // p * (log2 p - log2 q); q == 0 with p > 0 gives +inf, as it should
-      if (p > 0.f) acc.pa = (q > 0.f) ? fmaf(p, a - b, acc.pa) : INFINITY;
+  for (int j = 0; j < N; ++j) {
+    const float2 a = __ffma2_rn(xl[j], cc, nl), b = __ffma2_rn(xs[j], cc, ns);   // log2 p, log2 q
+    if (DIV == kDivKL) {
+      // KL(large || small) on unclamped logits: q == 0 with p > 0 gives +inf, as it should
+      const float2 p = ex2_2(a), q = ex2_2(b);
+      acc.big = __fadd2_rn(acc.big, make_float2(fmaxf(p.x, q.x), fmaxf(p.y, q.y)));
+      if (p.x > 0.f) acc.js.x = (q.x > 0.f) ? fmaf(p.x, a.x - b.x, acc.js.x) : INFINITY;
+      if (p.y > 0.f) acc.js.y = (q.y > 0.f) ? fmaf(p.y, a.y - b.y, acc.js.y) : INFINITY;
+    } else {
+      const float2 e = make_float2(ex2_approx(fmaxf(a.x, b.x)), ex2_approx(fmaxf(a.y, b.y)));   // max(p, q)
+      acc.big = __fadd2_rn(acc.big, e);
+      if (DIV == kDivJS) {
+        const float2 dd = __ffma2_rn(b, splat2(-1.f), a);
+        const float2 u = make_float2(ex2_approx(-fabsf(dd.x)), ex2_approx(-fabsf(dd.y)));
+        const float2 ps = psi_poly(u);
+        const float2 h = make_float2(fmaf(u.x, -fabsf(dd.x), ps.x), fmaf(u.y, -fabsf(dd.y), ps.y));
+        acc.js = __ffma2_rn(e, h, acc.js);
+      }
     }
   }
 }
@@ -229,12 +373,13 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
   const int C = G.chunks, R = G.ring;
 
   if (tid == 0) {
-    for (int s = 0; s < kClSlots; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], kClConsumerWarps); }
+    for (int s = 0; s < kClSlots; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], kClPassWarps); }
     for (int d = 0; d < kClDepth; ++d) {
-      mbar_init(&ctl->a_done[d], kClConsumerWarps);
-      mbar_init(&ctl->b_done[d], kClConsumerWarps);
+      mbar_init(&ctl->a_done[d], kClPassWarps);
+      mbar_init(&ctl->b_done[d], kClPassWarps);
       mbar_init(&ctl->lse_ready[d], G.cs);
       mbar_init(&ctl->fin_ready[d], G.cs);
+      mbar_init(&ctl->b_go[d], 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -246,133 +391,112 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     dead = true;
     atomicExch(P.status, 1);
   };
+  // blocking wait on one mbarrier phase, bounded
+  auto wait_phase = [&](unsigned long long* bar, unsigned parity) {
+    unsigned spins = 0;
+    while (!dead && !mbar_try(bar, parity))
+      if (++spins > kClSpinLimit) give_up();
+  };
 
   if (warp < kClConsumerWarps) {
-    // ================================ consumers ================================
-    const float c = P.c, inv_c = 1.f / P.c;
-    RowWalk wa, wb;
-    wa.init(P, cluster_id, G.n_clusters);
-    wb.init(P, cluster_id, G.n_clusters);
-    bool a_row = wa.advance(), b_row = wb.advance();
-    int ca = 0, cb = 0;          // chunk inside the current row of each pass
-    unsigned ga = 0, gb = 0;     // chunks finished by each pass since kernel start
-    bool b_ready = false;        // normalisers of pass B's current row are in registers
-    float off_l = 0.f, off_s = 0.f;
-    LseState ls, ll;
-    ls.reset(inv_c); ll.reset(inv_c);
-    DivAcc acc;
-    acc.reset();
-    const int vec_in_chunk = warp * 32 + lane;
-    unsigned idle = 0;
-
-    while (b_row) {
-      bool progressed = false;
-      // ---- pass A on the next chunk, if it has landed ----
-      if (a_row) {
-        const unsigned slot = ga % R;
-        if (dead || mbar_test(&ctl->full[slot], (ga / R) & 1u)) {
-          const int e0 = ca * CH + vec_in_chunk * E;
-          if (e0 < slice_len) {
-            const unsigned char* base = ring + static_cast<size_t>(slot) * kClSlotBytes + vec_in_chunk * 16;
-            float xs[E], xl[E];
-            Elem<T>::unpack(lds128(base), xs);
-            Elem<T>::unpack(lds128(base + kClHalfBytes), xl);
-            lse_accumulate<E>(xs, c, inv_c, ls);
-            lse_accumulate<E>(xl, c, inv_c, ll);
-          }
-          ++ga;
-          if (++ca == C) {
-            // row finished: warp partial -> a_part, then tell the agent
-            float rs = ls.ref, ss = ls.s0 + ls.s1, rl = ll.ref, sl = ll.s0 + ll.s1;
+    const float c = P.c;
+    const int pw = warp % kClPassWarps;               // index among the warps of this pass
+    // vectors pw*32 + lane and that + 256 of every chunk; `len[i]` > chunk offset while vector i lies inside the slice
+    const unsigned char* my = ring + (pw * 32 + lane) * 16;
+    int len[kClVecPerLane];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              lse_merge(rs, ss, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, ss, o));
-              lse_merge(rl, sl, __shfl_xor_sync(0xffffffffu, rl, o), __shfl_xor_sync(0xffffffffu, sl, o));
-            }
-            const int d = wa.n % kClDepth;
-            if (lane == 0) {
-              ctl->a_part[d][warp] = make_float4(rs, ss, rl, sl);
-              mbar_arrive(&ctl->a_done[d]);
-            }
-            ls.reset(inv_c); ll.reset(inv_c);
-            ca = 0;
-            a_row = wa.advance();
+    for (int i = 0; i < kClVecPerLane; ++i) len[i] = slice_len - (pw * 32 + lane + i * kClPassWarps * 32) * E;
+    constexpr int kVecStride = kClPassWarps * 32 * 16;   // bytes between a lane's two vectors
+    RowWalk w;
+    w.init(P, cluster_id, G.n_clusters);
+    unsigned slot = 0, par = 0;
+
+    if (warp < kClPassWarps) {
+      // ================================ pass A ================================
+      LseState ls, ll;
+      while (w.advance()) {
+        ls.reset(); ll.reset();
+        int off = 0;   // chunk offset inside the slice, in logits
+        for (int cidx = 0; cidx < C; ++cidx, off += CH) {
+          wait_phase(&ctl->full[slot], par);
+          const unsigned char* base = my + slot * kClSlotBytes;
+          uint4 us[kClVecPerLane], ul[kClVecPerLane];
+          float ts[kClVecPerLane], tl[kClVecPerLane];
+#pragma unroll
+          for (int i = 0; i < kClVecPerLane; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+          const float ref_s = ls.ref, ref_l = ll.ref;
+#pragma unroll
+          for (int i = 0; i < kClVecPerLane; ++i) { ts[i] = lse_vector_sum<T>(us[i], c, ref_s); tl[i] = lse_vector_sum<T>(ul[i], c, ref_l); }
+#pragma unroll
+          for (int i = 0; i < kClVecPerLane; ++i) {
+            lse_commit<T>(ts[i], ref_s, us[i], len[i] > off, c, ls);
+            lse_commit<T>(tl[i], ref_l, ul[i], len[i] > off, c, ll);
           }
-          progressed = true;
+          if (++slot == static_cast<unsigned>(R)) { slot = 0; par ^= 1u; }
+        }
+        // row finished: the warp's partial (one reference, summed S) -> a_part, then tell the agent
+        const float ss = warp_reduce<OpSum>(ls.s), sl = warp_reduce<OpSum>(ll.s);
+        const int d = w.n % kClDepth;
+        if (lane == 0) {
+          ctl->a_part[d][pw] = make_float4(ls.ref, ss, ll.ref, sl);
+          mbar_arrive(&ctl->a_done[d]);
         }
       }
-      // ---- pass B on its next chunk, if pass A has been there and the row's normalisers are known ----
-      if (gb < ga) {
-        const int d = wb.n % kClDepth;
-        if (!b_ready && (dead || mbar_test_cluster(&ctl->lse_ready[d], (wb.n / kClDepth) & 1u))) {
-          float ms = -INFINITY, ml = -INFINITY;
-          for (int j = 0; j < G.cs; ++j) { ms = fmaxf(ms, ctl->lse_in[d][j].x); ml = fmaxf(ml, ctl->lse_in[d][j].z); }
-          float ss = 0.f, sl = 0.f;
-          for (int j = 0; j < G.cs; ++j) {
-            const float4 v = ctl->lse_in[d][j];
-            ss += v.y * ex2_approx(v.x - ms);
-            sl += v.w * ex2_approx(v.z - ml);
-          }
-          const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl);
-          off_s = ms + l2ss;
-          off_l = ml + l2sl;
-          if (warp == 0 && lane == 0) ctl->row_lse[d] = make_float4(ms, l2ss, ml, l2sl);
-          b_ready = true;
-        }
-        if (b_ready) {
-          const unsigned slot = gb % R;
-          const int e0 = cb * CH + vec_in_chunk * E;
-          if (e0 < slice_len) {
-            const unsigned char* base = ring + static_cast<size_t>(slot) * kClSlotBytes + vec_in_chunk * 16;
-            const uint4 us = lds128(base), ul = lds128(base + kClHalfBytes);
-            acc.differ |= (us.x ^ ul.x) | (us.y ^ ul.y) | (us.z ^ ul.z) | (us.w ^ ul.w);
-            float xs[E], xl[E];
-            Elem<T>::unpack(us, xs);
-            Elem<T>::unpack(ul, xl);
-            div_accumulate<DIV, E>(xl, xs, c, off_l, off_s, acc);
+    } else {
+      // ================================ pass B ================================
+      constexpr int N = Pairs<T>::kN;
+      while (w.advance()) {
+        const int d = w.n % kClDepth;
+        wait_phase(&ctl->b_go[d], (w.n / kClDepth) & 1u);   // the row's constants are published: pass A is through
+        const RowConsts rc = ctl->row_consts[d];
+        DivAcc acc;
+        acc.reset();
+        int off = 0;
+        for (int cidx = 0; cidx < C; ++cidx, off += CH) {
+          const unsigned char* base = my + slot * kClSlotBytes;
+          uint4 us[kClVecPerLane], ul[kClVecPerLane];
+#pragma unroll
+          for (int i = 0; i < kClVecPerLane; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+#pragma unroll
+          for (int i = 0; i < kClVecPerLane; ++i) {
+            float2 xs[N], xl[N];
+            Pairs<T>::load_clamped(us[i], rc.floor_small, rc.floor2_small, xs);
+            Pairs<T>::load_clamped(ul[i], rc.floor_large, rc.floor2_large, xl);
+            DivAcc local;
+            local.reset();
+            local.differ = (us[i].x ^ ul[i].x) | (us[i].y ^ ul[i].y) | (us[i].z ^ ul[i].z) | (us[i].w ^ ul[i].w);
+            div_accumulate<DIV, N>(xl, xs, c, rc.off_large, rc.off_small, local);
+            if (len[i] > off) {   // a vector beyond the slice adds nothing
+              acc.js = __fadd2_rn(acc.js, local.js);
+              acc.big = __fadd2_rn(acc.big, local.big);
+              acc.differ |= local.differ;
+            }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&ctl->empty[slot]);   // this warp is done with the slot
-          ++gb;
-          if (++cb == C) {
-            const double pab = warp_sum(static_cast<double>(acc.pa) + static_cast<double>(acc.qb));
-            const double sl = warp_sum(static_cast<double>(acc.sl));
-            const double big = warp_sum(static_cast<double>(acc.big));
-            const unsigned differ = __reduce_or_sync(0xffffffffu, acc.differ);
-            if (lane == 0) {
-              ctl->b_part[d][warp][0] = pab;
-              ctl->b_part[d][warp][1] = sl;
-              ctl->b_part[d][warp][2] = big;
-              ctl->b_part[d][warp][3] = differ ? 1.0 : 0.0;
-              mbar_arrive(&ctl->b_done[d]);
-            }
-            acc.reset();
-            cb = 0;
-            b_ready = false;
-            b_row = wb.advance();
-          }
-          progressed = true;
+          if (++slot == static_cast<unsigned>(R)) slot = 0;
+        }
+        const float js = warp_reduce<OpSum>(acc.js.x + acc.js.y);
+        const float big = warp_reduce<OpSum>(acc.big.x + acc.big.y);
+        const unsigned differ = __reduce_or_sync(0xffffffffu, acc.differ);
+        if (lane == 0) {
+          ctl->b_part[d][pw] = make_float4(js, big, differ ? 1.f : 0.f, 0.f);
+          mbar_arrive(&ctl->b_done[d]);
         }
       }
-      if (progressed) idle = 0;
-      else if (!dead && ++idle > kClSpinLimit) give_up();
     }
   } else if (warp == kClConsumerWarps) {
     // ================================ loader ================================
     if (lane == 0) {
       RowWalk w;
       w.init(P, cluster_id, G.n_clusters);
-      unsigned g = 0;
+      unsigned slot = 0, fills = 0;   // ring position; how often the ring has wrapped
       while (w.advance()) {
         const T* rs = row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V) + slice_begin;
         const T* rl = row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V) + slice_begin;
-        for (int cidx = 0; cidx < C; ++cidx, ++g) {
-          const unsigned slot = g % R;
-          if (g >= static_cast<unsigned>(R)) {
-            const unsigned parity = ((g / R) - 1u) & 1u;
-            unsigned spins = 0;
-            while (!dead && !mbar_test(&ctl->empty[slot], parity))
-              if (++spins > kClSpinLimit) give_up();
+        for (int cidx = 0; cidx < C; ++cidx) {
+          if (fills > 0) {
+            wait_phase(&ctl->empty[slot], (fills - 1u) & 1u);
           }
           const int e0 = cidx * CH;
           const int n = min(CH, slice_len - e0);
@@ -385,33 +509,40 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
           } else {
             mbar_arrive(&ctl->full[slot]);   // nothing of this chunk falls into this CTA's slice
           }
+          if (++slot == static_cast<unsigned>(R)) { slot = 0; ++fills; }
         }
       }
       // every copy issued above is waited for by pass A of the consumers before they leave
     }
   } else {
     // ================================ agent ================================
-    RowWalk wa, wb, wf;
+    // Four kinds of events, each taken in row order:
+    //   a(n)  the pass-A warps' partials of row n are in -> merge, send the CTA's partial to every rank
+    //   g(n)  every rank's partial of row n has arrived     -> row constants for pass B, release the consumers
+    //   b(n)  the pass-B warps' partials of row n are in -> sum, send to rank 0
+    //   f(n)  (rank 0) every rank's pass-B partial arrived  -> write the row's statistics
+    // The exchange buffers of row n are reused by row n + kClDepth. Nothing of row n + kClDepth can be produced
+    // anywhere in the cluster before this agent has sent a(n + kClDepth), so a(m) is held back until b and (on
+    // rank 0) f of row m - kClDepth + 1 are done; and a(m) waits for g(m - 2), so that no peer can overwrite
+    // lse_in of a row this agent has not combined yet.
+    RowWalk wa, wg, wb, wf;
     wa.init(P, cluster_id, G.n_clusters);
+    wg.init(P, cluster_id, G.n_clusters);
     wb.init(P, cluster_id, G.n_clusters);
     wf.init(P, cluster_id, G.n_clusters);
-    bool a_row = wa.advance(), b_row = wb.advance();
+    bool a_row = wa.advance(), g_row = wg.advance(), b_row = wb.advance();
     bool f_row = (rank == 0) ? wf.advance() : false;
+    const float inv_c = 1.f / P.c;
     unsigned idle = 0;
-    // Events are taken in row order within each kind. A row's exchange buffers are reused kClDepth rows
-    // later, and nothing of row m + kClDepth can be produced anywhere in the cluster before this agent has
-    // sent the pass-A partial of that row; so that partial is held back until the pass-B partial of row m
-    // has been forwarded (and, on rank 0, row m's statistics written).
-    int na = 0, nb = 0, nf = 0;
-    while (a_row || b_row || f_row) {
+    int na = 0, ng = 0, nb = 0, nf = 0;
+    while (a_row || g_row || b_row || f_row) {
       bool progressed = false;
-      if (a_row && na - nb < kClDepth - 1 && (rank != 0 || na - nf < kClDepth - 1)) {
+      if (a_row && na - nb < kClDepth - 1 && na - ng < 2 && (rank != 0 || na - nf < kClDepth - 1)) {
         const int d = wa.n % kClDepth;
         if (dead || mbar_test(&ctl->a_done[d], (wa.n / kClDepth) & 1u)) {
-          // reduce the 16 warp partials (fixed tree) and hand the CTA's partial to every rank
-          float4 v = (lane < kClConsumerWarps) ? ctl->a_part[d][lane] : make_float4(-1e30f, 0.f, -1e30f, 0.f);
+          float4 v = (lane < kClPassWarps) ? ctl->a_part[d][lane] : make_float4(-1e30f, 0.f, -1e30f, 0.f);
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
+          for (int o = 16; o > 0; o >>= 1) {   // fixed tree
             lse_merge(v.x, v.y, __shfl_xor_sync(0xffffffffu, v.x, o), __shfl_xor_sync(0xffffffffu, v.y, o));
             lse_merge(v.z, v.w, __shfl_xor_sync(0xffffffffu, v.z, o), __shfl_xor_sync(0xffffffffu, v.w, o));
           }
@@ -424,19 +555,49 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
           progressed = true;
         }
       }
-      if (b_row && nb < na) {
+      if (g_row && ng < na) {
+        const int d = wg.n % kClDepth;
+        if (dead || mbar_test(&ctl->lse_ready[d], (wg.n / kClDepth) & 1u)) {
+          fence_acquire_cluster();   // the partials were written by the peers' agents before they arrived
+          float ms = -INFINITY, ml = -INFINITY;
+          for (int j = 0; j < G.cs; ++j) { ms = fmaxf(ms, ctl->lse_in[d][j].x); ml = fmaxf(ml, ctl->lse_in[d][j].z); }
+          float ss = 0.f, sl = 0.f;
+          for (int j = 0; j < G.cs; ++j) {   // rank order: every CTA of the cluster gets the same bits
+            const float4 v = ctl->lse_in[d][j];
+            ss += v.y * ex2_approx(v.x - ms);
+            sl += v.w * ex2_approx(v.z - ml);
+          }
+          const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl);
+          if (lane == 0) {
+            RowConsts rc;
+            rc.off_small = ms + l2ss;
+            rc.off_large = ml + l2sl;
+            // logits below the floors give log2 p < -125; the KL variant needs true zeros and clamps nothing
+            rc.floor_small = (DIV == kDivKL) ? -INFINITY : (rc.off_small - 125.f) * inv_c;
+            rc.floor_large = (DIV == kDivKL) ? -INFINITY : (rc.off_large - 125.f) * inv_c;
+            rc.floor2_small = Pairs<T>::floor_bits(rc.floor_small);
+            rc.floor2_large = Pairs<T>::floor_bits(rc.floor_large);
+            rc.pad0 = rc.pad1 = 0u;
+            ctl->row_consts[d] = rc;
+            ctl->row_lse[d] = make_float4(ms, l2ss, ml, l2sl);
+            mbar_arrive(&ctl->b_go[d]);
+          }
+          g_row = wg.advance();
+          ++ng;
+          progressed = true;
+        }
+      }
+      if (b_row && nb < ng) {
         const int d = wb.n % kClDepth;
         if (dead || mbar_test(&ctl->b_done[d], (wb.n / kClDepth) & 1u)) {
-          double v0 = 0.0, v1 = 0.0, v2 = 0.0, v3 = 0.0;
-          if (lane < kClConsumerWarps) {
-            v0 = ctl->b_part[d][lane][0]; v1 = ctl->b_part[d][lane][1];
-            v2 = ctl->b_part[d][lane][2]; v3 = ctl->b_part[d][lane][3];
-          }
-          v0 = warp_sum(v0); v1 = warp_sum(v1); v2 = warp_sum(v2); v3 = warp_sum(v3);
+          const float4 v = (lane < kClPassWarps) ? ctl->b_part[d][lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+          const double js = warp_sum(static_cast<double>(v.x));
+          const double big = warp_sum(static_cast<double>(v.y));
+          const double differ = warp_sum(static_cast<double>(v.z));
           if (lane == 0) {
             const unsigned dst = map_to_rank(&ctl->fin_in[d][rank][0], 0);
-            remote_store_d2(dst, v0, v1);
-            remote_store_d2(dst + 16, v2, v3);
+            remote_store_d2(dst, js, 0.0);
+            remote_store_d2(dst + 16, big, differ);
             remote_arrive(map_to_rank(&ctl->fin_ready[d], 0));
           }
           b_row = wb.advance();
@@ -446,11 +607,12 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       }
       if (f_row && nf < nb) {
         const int d = wf.n % kClDepth;
-        if (dead || mbar_test_cluster(&ctl->fin_ready[d], (wf.n / kClDepth) & 1u)) {
+        if (dead || mbar_test(&ctl->fin_ready[d], (wf.n / kClDepth) & 1u)) {
+          fence_acquire_cluster();
           if (lane == 0) {
-            double pab = 0.0, sl = 0.0, big = 0.0, differ = 0.0;
+            double js = 0.0, big = 0.0, differ = 0.0;
             for (int j = 0; j < G.cs; ++j) {
-              pab += ctl->fin_in[d][j][0]; sl += ctl->fin_in[d][j][1];
+              js += ctl->fin_in[d][j][0];
               big += ctl->fin_in[d][j][2]; differ += ctl->fin_in[d][j][3];
             }
             const float4 lse = ctl->row_lse[d];
@@ -463,8 +625,8 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
             } else {
               double D;
               const double res = big - 1.0;   // sum max(p,q) - sum q = sum max(0, p - q)
-              if (DIV == kDivJS) D = 0.5 * 0.6931471805599453 * (pab - sl + 2.0);   // sum s*(lg s - 1) = sl - 2
-              else if (DIV == kDivKL) D = 0.6931471805599453 * pab;
+              if (DIV == kDivJS) D = 0.5 * 0.6931471805599453 * js;   // bits -> nats, and the 1/2 of the definition
+              else if (DIV == kDivKL) D = 0.6931471805599453 * js;
               else D = res;
               st.m2_small = lse.x; st.l2s_small = lse.y; st.m2_large = lse.z; st.l2s_large = lse.w;
               st.div = fmaxf(static_cast<float>(D), 0.f);
@@ -480,7 +642,10 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
         }
       }
       if (progressed) idle = 0;
-      else if (!dead && ++idle > kClSpinLimit) give_up();
+      else if (!dead) {
+        if (++idle > kClSpinLimit) give_up();
+        __nanosleep(200);   // the agent shares an issue port with consumer warps: poll gently
+      }
     }
   }
   // no CTA may leave while a peer can still write into its shared memory
