@@ -21,6 +21,8 @@
 // terminates.
 #pragma once
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace psd {
@@ -63,7 +65,7 @@ struct __align__(16) ClusterCtl {
   float4 row_lse[kClDepth];                        // (m2_small, l2s_small, m2_large, l2s_large) of the row
   RowConsts row_consts[kClDepth];                  // what pass B needs of the row, published by the agent
   float4 lse_in[kClDepth][kClMaxRanks];            // partials received from every rank of the cluster
-  double fin_in[kClDepth][kClMaxRanks][4];         // pass-B partials received (rank 0 only)
+  float4 fin_in[kClDepth][kClMaxRanks];            // pass-B partials received (rank 0 only)
 };
 
 constexpr size_t kClSmemBytes = static_cast<size_t>(kClSlots) * kClSlotBytes + sizeof(ClusterCtl) + 128;
@@ -87,13 +89,6 @@ __device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned pari
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// same, observing writes made by other CTAs of the cluster before their arrive
-__device__ __forceinline__ bool mbar_test_cluster(unsigned long long* bar, unsigned parity) {
-  unsigned ok;
-  asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
 // may suspend the thread for a hardware-chosen time before answering
 __device__ __forceinline__ bool mbar_try(unsigned long long* bar, unsigned parity) {
   unsigned ok;
@@ -101,20 +96,17 @@ __device__ __forceinline__ bool mbar_try(unsigned long long* bar, unsigned parit
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void fence_acquire_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 __device__ __forceinline__ unsigned map_to_rank(const void* local, unsigned rank) {
   unsigned r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(local)), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void remote_arrive(unsigned cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void remote_store_f4(unsigned cluster_addr, float4 v) {
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
-__device__ __forceinline__ void remote_store_d2(unsigned cluster_addr, double a, double b) {
-  asm volatile("st.shared::cluster.v2.f64 [%0], {%1, %2};" ::"r"(cluster_addr), "d"(a), "d"(b) : "memory");
+// 16 bytes into another CTA's shared memory; the bytes are counted on that CTA's mbarrier when they land,
+// so the receiver needs no fence: a completed phase means the data is there.
+__device__ __forceinline__ void remote_post_f4(unsigned cluster_addr, float4 v, unsigned cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(cluster_addr), "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)),
+                 "r"(__float_as_uint(v.w)), "r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -377,8 +369,8 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     for (int d = 0; d < kClDepth; ++d) {
       mbar_init(&ctl->a_done[d], kClPassWarps);
       mbar_init(&ctl->b_done[d], kClPassWarps);
-      mbar_init(&ctl->lse_ready[d], G.cs);
-      mbar_init(&ctl->fin_ready[d], G.cs);
+      mbar_init(&ctl->lse_ready[d], 1);   // the local agent's arrive; the peers' partials count as bytes
+      mbar_init(&ctl->fin_ready[d], 1);
       mbar_init(&ctl->b_go[d], 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -540,16 +532,24 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       if (a_row && na - nb < kClDepth - 1 && na - ng < 2 && (rank != 0 || na - nf < kClDepth - 1)) {
         const int d = wa.n % kClDepth;
         if (dead || mbar_test(&ctl->a_done[d], (wa.n / kClDepth) & 1u)) {
-          float4 v = (lane < kClPassWarps) ? ctl->a_part[d][lane] : make_float4(-1e30f, 0.f, -1e30f, 0.f);
+          // merge the pass-A warps' partials (every lane does the same arithmetic, warp order) ...
+          float4 part[kClPassWarps];
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {   // fixed tree
-            lse_merge(v.x, v.y, __shfl_xor_sync(0xffffffffu, v.x, o), __shfl_xor_sync(0xffffffffu, v.y, o));
-            lse_merge(v.z, v.w, __shfl_xor_sync(0xffffffffu, v.z, o), __shfl_xor_sync(0xffffffffu, v.w, o));
+          for (int k = 0; k < kClPassWarps; ++k) part[k] = ctl->a_part[d][k];
+          float ms = part[0].x, ml = part[0].z;
+#pragma unroll
+          for (int k = 1; k < kClPassWarps; ++k) { ms = fmaxf(ms, part[k].x); ml = fmaxf(ml, part[k].z); }
+          float ss = 0.f, sl = 0.f;
+#pragma unroll
+          for (int k = 0; k < kClPassWarps; ++k) {
+            ss = fmaf(part[k].y, ex2_approx(part[k].x - ms), ss);
+            sl = fmaf(part[k].w, ex2_approx(part[k].z - ml), sl);
           }
-          if (lane < G.cs) {
-            remote_store_f4(map_to_rank(&ctl->lse_in[d][rank], lane), v);
-            remote_arrive(map_to_rank(&ctl->lse_ready[d], lane));
-          }
+          // ... open this row's phase of the local barrier for one partial per rank, and post ours to every rank
+          if (lane == 0) mbar_arrive_expect_tx(&ctl->lse_ready[d], static_cast<unsigned>(G.cs) * 16u);
+          if (lane < G.cs)
+            remote_post_f4(map_to_rank(&ctl->lse_in[d][rank], lane), make_float4(ms, ss, ml, sl),
+                           map_to_rank(&ctl->lse_ready[d], lane));
           a_row = wa.advance();
           ++na;
           progressed = true;
@@ -558,14 +558,13 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       if (g_row && ng < na) {
         const int d = wg.n % kClDepth;
         if (dead || mbar_test(&ctl->lse_ready[d], (wg.n / kClDepth) & 1u)) {
-          fence_acquire_cluster();   // the partials were written by the peers' agents before they arrived
           float ms = -INFINITY, ml = -INFINITY;
           for (int j = 0; j < G.cs; ++j) { ms = fmaxf(ms, ctl->lse_in[d][j].x); ml = fmaxf(ml, ctl->lse_in[d][j].z); }
           float ss = 0.f, sl = 0.f;
           for (int j = 0; j < G.cs; ++j) {   // rank order: every CTA of the cluster gets the same bits
             const float4 v = ctl->lse_in[d][j];
-            ss += v.y * ex2_approx(v.x - ms);
-            sl += v.w * ex2_approx(v.z - ml);
+            ss = fmaf(v.y, ex2_approx(v.x - ms), ss);
+            sl = fmaf(v.w, ex2_approx(v.z - ml), sl);
           }
           const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl);
           if (lane == 0) {
@@ -590,15 +589,16 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       if (b_row && nb < ng) {
         const int d = wb.n % kClDepth;
         if (dead || mbar_test(&ctl->b_done[d], (wb.n / kClDepth) & 1u)) {
-          const float4 v = (lane < kClPassWarps) ? ctl->b_part[d][lane] : make_float4(0.f, 0.f, 0.f, 0.f);
-          const double js = warp_sum(static_cast<double>(v.x));
-          const double big = warp_sum(static_cast<double>(v.y));
-          const double differ = warp_sum(static_cast<double>(v.z));
+          float js = 0.f, big = 0.f, differ = 0.f;
+#pragma unroll
+          for (int k = 0; k < kClPassWarps; ++k) {   // warp order
+            const float4 v = ctl->b_part[d][k];
+            js += v.x; big += v.y; differ += v.z;
+          }
           if (lane == 0) {
-            const unsigned dst = map_to_rank(&ctl->fin_in[d][rank][0], 0);
-            remote_store_d2(dst, js, 0.0);
-            remote_store_d2(dst + 16, big, differ);
-            remote_arrive(map_to_rank(&ctl->fin_ready[d], 0));
+            if (rank == 0) mbar_arrive_expect_tx(&ctl->fin_ready[d], static_cast<unsigned>(G.cs) * 16u);
+            remote_post_f4(map_to_rank(&ctl->fin_in[d][rank], 0), make_float4(js, big, differ, 0.f),
+                           map_to_rank(&ctl->fin_ready[d], 0));
           }
           b_row = wb.advance();
           ++nb;
@@ -608,12 +608,11 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       if (f_row && nf < nb) {
         const int d = wf.n % kClDepth;
         if (dead || mbar_test(&ctl->fin_ready[d], (wf.n / kClDepth) & 1u)) {
-          fence_acquire_cluster();
           if (lane == 0) {
             double js = 0.0, big = 0.0, differ = 0.0;
-            for (int j = 0; j < G.cs; ++j) {
-              js += ctl->fin_in[d][j][0];
-              big += ctl->fin_in[d][j][2]; differ += ctl->fin_in[d][j][3];
+            for (int j = 0; j < G.cs; ++j) {   // rank order
+              const float4 v = ctl->fin_in[d][j];
+              js += v.x; big += v.y; differ += v.z;
             }
             const float4 lse = ctl->row_lse[d];
             RowStats st{};
@@ -644,7 +643,7 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       if (progressed) idle = 0;
       else if (!dead) {
         if (++idle > kClSpinLimit) give_up();
-        __nanosleep(200);   // the agent shares an issue port with consumer warps: poll gently
+        __nanosleep(40);   // the agent shares an issue port with consumer warps: poll gently
       }
     }
   }
@@ -762,6 +761,11 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
   const int es = dtype == 0 ? 4 : 2;
   const long long rows = static_cast<long long>(P.B) * P.K;
   int cs = 0, slice = 0, chunks = 0;
+  if (forced_cs <= 0) {
+    // tuning aid: PYRAMIDSD_CLUSTER_SIZE=<power of two> overrides the library's choice for every call
+    static const int env_cs = [] { const char* e = std::getenv("PYRAMIDSD_CLUSTER_SIZE"); return e ? std::atoi(e) : 0; }();
+    if (env_cs > 0) forced_cs = env_cs;
+  }
   if (forced_cs > 0) {
     if (forced_cs > kClMaxRanks || (forced_cs & (forced_cs - 1)) != 0) return false;
     cs = forced_cs;
