@@ -144,6 +144,34 @@ int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, con
                           int32_t* out_accept_len_q, int32_t* out_next_token_q,
                           int32_t* out_accept_len, int32_t* out_next_token);
 
+/* (No counterpart in the paper: a packaging variant of pyramidsd_verify_stage.)
+ * The same single stage for callers that must not allocate device memory: a component running inside
+ * somebody else's memory plan (an inference server that hands every byte out at start-up and treats a
+ * later cudaMalloc as a bug, a plug-in loaded into a process whose allocator it may not touch, code
+ * running where an allocation would stall the whole device). The other entry points keep their per-row
+ * statistics in a workspace the caller supplies or the library cudaMallocs on first use; this one keeps
+ * them in an array built into the library image: PSD_NOALLOC_MAX_ROWS rows of 32 bytes plus one 256-byte
+ * line, 256.25 KiB on every device that loads the library, until the process ends. It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.
+ *   - Same arguments, results, Jensen-Shannon divergence and kernels as pyramidsd_verify_stage; the work
+ *     is enqueued on `cuda_stream` (a cudaStream_t; NULL = the legacy default stream) and the call returns
+ *     without synchronising.
+ *   - B * K must not exceed PSD_NOALLOC_MAX_ROWS: a larger stage returns PSD_ERR_UNSUPPORTED (with a line on
+ *     stderr) and launches nothing. Split such a batch over several calls, one after the other.
+ *   - out_wait_timeout: device pointer to one int32, or NULL. It receives 0, or 1 if a bounded wait inside
+ *     the kernels gave up (results are then invalid); pyramidsd_last_status() does not cover this call.
+ *   - The first call on each device looks up the built-in array's device address
+ *     (cudaGetSymbolAddress, with that device current). Make that first call outside any stream capture.
+ *   - Every call on a device shares the one array, and the array keeps what the last call left in it.
+ *     The call clears the only word that must start at zero. Two calls whose kernels overlap on the GPU
+ *     (different streams, or several host threads) race on it: keep calls on one device in stream order. */
+#define PSD_NOALLOC_MAX_ROWS 8192
+int pyramidsd_verify_stage_noalloc(const void* logits_small, const void* logits_large, const int32_t* draft_tokens,
+                                   int B, int K, int V, psd_dtype dtype, float threshold, psd_mode mode,
+                                   uint64_t philox_seed, uint64_t offset,
+                                   int32_t* out_accept_len, int32_t* out_next_token,
+                                   int32_t* out_wait_timeout, void* cuda_stream);
+
 /* The Philox uniforms the verification draws for rows 0..n_rows-1 with this seed and offset (see the
  * header comment for the counter layout): out_u[r] decides the strict coin flip of row r, out_u2[r]
  * drives its inverse CDF. Device pointers, float32 [n_rows]; either may be NULL. Lets a caller replay

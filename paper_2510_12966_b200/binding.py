@@ -22,6 +22,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, 
 
 EXPORTS = (
     "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_host",
+    "pyramidsd_verify_stage_noalloc",
     "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
     "pyramidsd_kernel_timing_begin", "pyramidsd_kernel_timing_end",
     "pyramidsd_cluster_occupancy", "pyramidsd_version", "pyramidsd_status_string",
@@ -70,6 +71,8 @@ def load_library(path: Optional[str] = None):
     i32, u64, f32, vp = C.c_int, C.c_uint64, C.c_float, C.c_void_p
     lib.pyramidsd_verify_stage.argtypes = [vp, vp, vp, i32, i32, i32, i32, f32, i32, u64, u64, vp, vp]
     lib.pyramidsd_verify_stage.restype = i32
+    lib.pyramidsd_verify_stage_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, f32, i32, u64, u64, vp, vp, vp, vp]
+    lib.pyramidsd_verify_stage_noalloc.restype = i32
     lib.pyramidsd_verify_stage_ex.argtypes = [C.POINTER(StageArgs)]
     lib.pyramidsd_verify_stage_ex.restype = i32
     pyr = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, u64, u64, vp, vp, vp, vp]
@@ -197,6 +200,26 @@ def verify_stage(logits_small, logits_large, draft_tokens, threshold, mode=FUZZY
         int(philox_seed), int(offset), _dev_ptr(out_accept_len, torch.int32), _dev_ptr(out_next_token, torch.int32))
     _check(rc, "pyramidsd_verify_stage")
     return out_accept_len, out_next_token
+
+
+NOALLOC_MAX_ROWS = 8192
+
+
+def verify_stage_noalloc(logits_small, logits_large, draft_tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
+                         out_accept_len, out_next_token, out_wait_timeout=None, stream=None, raise_on_error=True):
+    """``pyramidsd_verify_stage_noalloc``: the single stage with its scratch inside the library image, for
+    callers that may not allocate device memory. Every output tensor is the caller's (this wrapper
+    creates none); B * K is limited to NOALLOC_MAX_ROWS. Returns the status code."""
+    B, K, V = logits_small.shape
+    s = torch.cuda.current_stream() if stream is None else stream
+    rc = load_library().pyramidsd_verify_stage_noalloc(
+        _dev_ptr(logits_small, name="logits_small"), _dev_ptr(logits_large, name="logits_large"),
+        _dev_ptr(draft_tokens, torch.int32, "draft_tokens"), B, K, V, dtype_code(logits_small), float(threshold),
+        int(mode), int(philox_seed), int(offset), _dev_ptr(out_accept_len, torch.int32),
+        _dev_ptr(out_next_token, torch.int32), _dev_ptr(out_wait_timeout, torch.int32), C.c_void_p(s.cuda_stream))
+    if raise_on_error:
+        _check(rc, "pyramidsd_verify_stage_noalloc")
+    return rc
 
 
 def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,

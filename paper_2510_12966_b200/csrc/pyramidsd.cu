@@ -25,6 +25,15 @@ thread_local cudaStream_t t_stream = nullptr;
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 
+// Scratch of pyramidsd_verify_stage_noalloc: per-row statistics for up to PSD_NOALLOC_MAX_ROWS rows, then one
+// 256-byte line whose first word is the wait-timeout flag. It is part of the library image, so every
+// device that loads the library carries it until the process ends. In host code this name is only a
+// handle for cudaGetSymbolAddress; the device address it yields is what kernels are given.
+constexpr size_t kNoAllocStatsBytes = static_cast<size_t>(PSD_NOALLOC_MAX_ROWS) * sizeof(RowStats);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocStatsBytes + kAlign];
+void* g_noalloc_ptr[kMaxDevices] = {};
+std::mutex g_noalloc_mu;
+
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 // Library-owned scratch of one device: workspace for calls that bring none, the status word, and the
@@ -414,6 +423,69 @@ int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, con
     if (cudaMemcpyAsync(dst[i], o + static_cast<size_t>(i) * B, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
       return PSD_ERR_CUDA;
   return cudaStreamSynchronize(s) == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
+}
+
+int pyramidsd_verify_stage_noalloc(const void* logits_small, const void* logits_large, const int32_t* draft_tokens,
+                                   int B, int K, int V, psd_dtype dtype, float threshold, psd_mode mode,
+                                   uint64_t philox_seed, uint64_t offset, int32_t* out_accept_len,
+                                   int32_t* out_next_token, int32_t* out_wait_timeout, void* cuda_stream) {
+  if (B < 0 || K < 0) return PSD_ERR_INVALID_ARG;
+  if (static_cast<long long>(B) * K > PSD_NOALLOC_MAX_ROWS) {
+    std::fprintf(stderr, "pyramidsd_verify_stage_noalloc: B * K = %lld rows exceed the built-in scratch of %d rows\n",
+                 static_cast<long long>(B) * K, PSD_NOALLOC_MAX_ROWS);
+    return PSD_ERR_UNSUPPORTED;
+  }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PSD_ERR_CUDA;
+  void* scratch = nullptr;
+  {
+    // first call on this device: look the array's device address up, with this device current
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (g_noalloc_ptr[dev] == nullptr) {
+      void* p = nullptr;
+      const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+      if (e != cudaSuccess || p == nullptr) {
+        std::fprintf(stderr, "pyramidsd_verify_stage_noalloc: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+        cudaGetLastError();
+        return PSD_ERR_CUDA;
+      }
+      g_noalloc_ptr[dev] = p;
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  psd_stage_args a;
+  std::memset(&a, 0, sizeof(a));
+  a.struct_size = sizeof(a);
+  a.dtype = dtype;
+  a.logits_small = logits_small;
+  a.logits_large = logits_large;
+  a.tokens = draft_tokens;
+  a.B = B; a.K = K; a.V = V;
+  a.mode = mode;
+  a.div_kind = PSD_DIV_JS;
+  a.threshold = threshold;
+  a.philox_seed = philox_seed;
+  a.philox_offset = offset;
+  a.out_accept_len = out_accept_len;
+  a.out_next_token = out_next_token;
+  int rc = validate_stage(&a);
+  if (rc != PSD_OK) return rc;
+  if (B == 0) return PSD_OK;
+  const cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int* flag = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + kNoAllocStatsBytes);
+  // the flag is the one thing that has to start at zero; the statistics of every row read are written first
+  if (cudaMemsetAsync(flag, 0, sizeof(int), stream) != cudaSuccess) return PSD_ERR_CUDA;
+  const StageParams P = make_params(&a, scratch, flag);
+  if (K > 0) {
+    rc = launch_rowstats(P, dtype, PSD_KERNEL_AUTO, 0, stream);
+    if (rc != PSD_OK) return rc;
+  }
+  rc = launch_finalize(P, dtype, stream);
+  if (rc != PSD_OK) return rc;
+  if (out_wait_timeout != nullptr &&
+      cudaMemcpyAsync(out_wait_timeout, flag, sizeof(int), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+    return PSD_ERR_CUDA;
+  return PSD_OK;
 }
 
 int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, float* out_u, float* out_u2) {
