@@ -385,6 +385,7 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
   };
   // blocking wait on one mbarrier phase, bounded
   auto wait_phase = [&](unsigned long long* bar, unsigned parity) {
+    if (mbar_test(bar, parity)) return;   // the common case: already complete, no suspension
     unsigned spins = 0;
     while (!dead && !mbar_try(bar, parity))
       if (++spins > kClSpinLimit) give_up();
@@ -508,143 +509,128 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     }
   } else {
     // ================================ agent ================================
-    // Four kinds of events, each taken in row order:
-    //   a(n)  the pass-A warps' partials of row n are in -> merge, send the CTA's partial to every rank
+    // Four kinds of events per row:
+    //   a(n)  the warps' pass-A partials of row n are in    -> merge, send the CTA's partial to every rank
     //   g(n)  every rank's partial of row n has arrived     -> row constants for pass B, release the consumers
-    //   b(n)  the pass-B warps' partials of row n are in -> sum, send to rank 0
+    //   b(n)  the warps' pass-B partials of row n are in    -> sum, send to rank 0
     //   f(n)  (rank 0) every rank's pass-B partial arrived  -> write the row's statistics
-    // The exchange buffers of row n are reused by row n + kClDepth. Nothing of row n + kClDepth can be produced
-    // anywhere in the cluster before this agent has sent a(n + kClDepth), so a(m) is held back until b and (on
-    // rank 0) f of row m - kClDepth + 1 are done; and a(m) waits for g(m - 2), so that no peer can overwrite
-    // lse_in of a row this agent has not combined yet.
-    RowWalk wa, wg, wb, wf;
-    wa.init(P, cluster_id, G.n_clusters);
-    wg.init(P, cluster_id, G.n_clusters);
-    wb.init(P, cluster_id, G.n_clusters);
-    wf.init(P, cluster_id, G.n_clusters);
-    bool a_row = wa.advance(), g_row = wg.advance(), b_row = wb.advance();
-    bool f_row = (rank == 0) ? wf.advance() : false;
+    // taken in the fixed order a(n), g(n), b(n-1), f(n-1), which is the order the pipelined schedule completes
+    // them in, so every wait is a blocking wait on one barrier and the agent costs the consumer warps that
+    // share its issue port next to nothing. The order also keeps the exchange buffers safe: they are
+    // kClDepth rows deep, nothing of row m can be produced anywhere in the cluster before this agent has sent
+    // a(m), and a(m) comes after g(m-1), b(m-2) and f(m-2).
     const float inv_c = 1.f / P.c;
-    unsigned idle = 0;
-    int na = 0, ng = 0, nb = 0, nf = 0;
-    while (a_row || g_row || b_row || f_row) {
-      bool progressed = false;
-      if (a_row && na - nb < kClDepth - 1 && na - ng < 2 && (rank != 0 || na - nf < kClDepth - 1)) {
-        const int d = wa.n % kClDepth;
-        if (dead || mbar_test(&ctl->a_done[d], (wa.n / kClDepth) & 1u)) {
-          // merge the pass-A warps' partials (every lane does the same arithmetic, warp order) ...
-          float4 part[kClPassWarps];
+
+    auto event_a = [&](int n) {
+      const int d = n % kClDepth;
+      wait_phase(&ctl->a_done[d], (n / kClDepth) & 1u);
+      // merge the warps' partials (every lane does the same arithmetic, warp order) ...
+      float ms = -1e30f, ml = -1e30f;
 #pragma unroll
-          for (int k = 0; k < kClPassWarps; ++k) part[k] = ctl->a_part[d][k];
-          float ms = part[0].x, ml = part[0].z;
+      for (int k = 0; k < kClPassWarps; ++k) { ms = fmaxf(ms, ctl->a_part[d][k].x); ml = fmaxf(ml, ctl->a_part[d][k].z); }
+      float ss = 0.f, sl = 0.f;
 #pragma unroll
-          for (int k = 1; k < kClPassWarps; ++k) { ms = fmaxf(ms, part[k].x); ml = fmaxf(ml, part[k].z); }
-          float ss = 0.f, sl = 0.f;
+      for (int k = 0; k < kClPassWarps; ++k) {
+        const float4 v = ctl->a_part[d][k];
+        ss = fmaf(v.y, ex2_approx(v.x - ms), ss);
+        sl = fmaf(v.w, ex2_approx(v.z - ml), sl);
+      }
+      // ... open this row's phase of the local barrier for one partial per rank, and post ours to every rank
+      if (lane == 0) mbar_arrive_expect_tx(&ctl->lse_ready[d], static_cast<unsigned>(G.cs) * 16u);
+      if (lane < G.cs)
+        remote_post_f4(map_to_rank(&ctl->lse_in[d][rank], lane), make_float4(ms, ss, ml, sl),
+                       map_to_rank(&ctl->lse_ready[d], lane));
+    };
+    auto event_g = [&](int n) {
+      const int d = n % kClDepth;
+      wait_phase(&ctl->lse_ready[d], (n / kClDepth) & 1u);
+      float ms = -INFINITY, ml = -INFINITY;
+      for (int j = 0; j < G.cs; ++j) { ms = fmaxf(ms, ctl->lse_in[d][j].x); ml = fmaxf(ml, ctl->lse_in[d][j].z); }
+      float ss = 0.f, sl = 0.f;
+      for (int j = 0; j < G.cs; ++j) {   // rank order: every CTA of the cluster gets the same bits
+        const float4 v = ctl->lse_in[d][j];
+        ss = fmaf(v.y, ex2_approx(v.x - ms), ss);
+        sl = fmaf(v.w, ex2_approx(v.z - ml), sl);
+      }
+      const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl);
+      if (lane == 0) {
+        RowConsts rc;
+        rc.off_small = ms + l2ss;
+        rc.off_large = ml + l2sl;
+        // logits below the floors give log2 p < -125; the KL variant needs true zeros and clamps nothing
+        rc.floor_small = (DIV == kDivKL) ? -INFINITY : (rc.off_small - 125.f) * inv_c;
+        rc.floor_large = (DIV == kDivKL) ? -INFINITY : (rc.off_large - 125.f) * inv_c;
+        rc.floor2_small = Pairs<T>::floor_bits(rc.floor_small);
+        rc.floor2_large = Pairs<T>::floor_bits(rc.floor_large);
+        rc.pad0 = rc.pad1 = 0u;
+        ctl->row_consts[d] = rc;
+        ctl->row_lse[d] = make_float4(ms, l2ss, ml, l2sl);
+        mbar_arrive(&ctl->b_go[d]);
+      }
+    };
+    auto event_b = [&](int n) {
+      const int d = n % kClDepth;
+      wait_phase(&ctl->b_done[d], (n / kClDepth) & 1u);
+      float js = 0.f, big = 0.f, differ = 0.f;
 #pragma unroll
-          for (int k = 0; k < kClPassWarps; ++k) {
-            ss = fmaf(part[k].y, ex2_approx(part[k].x - ms), ss);
-            sl = fmaf(part[k].w, ex2_approx(part[k].z - ml), sl);
-          }
-          // ... open this row's phase of the local barrier for one partial per rank, and post ours to every rank
-          if (lane == 0) mbar_arrive_expect_tx(&ctl->lse_ready[d], static_cast<unsigned>(G.cs) * 16u);
-          if (lane < G.cs)
-            remote_post_f4(map_to_rank(&ctl->lse_in[d][rank], lane), make_float4(ms, ss, ml, sl),
-                           map_to_rank(&ctl->lse_ready[d], lane));
-          a_row = wa.advance();
-          ++na;
-          progressed = true;
+      for (int k = 0; k < kClPassWarps; ++k) {   // warp order
+        const float4 v = ctl->b_part[d][k];
+        js += v.x; big += v.y; differ += v.z;
+      }
+      if (lane == 0) {
+        if (rank == 0) mbar_arrive_expect_tx(&ctl->fin_ready[d], static_cast<unsigned>(G.cs) * 16u);
+        remote_post_f4(map_to_rank(&ctl->fin_in[d][rank], 0), make_float4(js, big, differ, 0.f),
+                       map_to_rank(&ctl->fin_ready[d], 0));
+      }
+    };
+    auto event_f = [&](int n, int r) {   // rank 0 only
+      const int d = n % kClDepth;
+      wait_phase(&ctl->fin_ready[d], (n / kClDepth) & 1u);
+      if (lane == 0) {
+        double js = 0.0, big = 0.0, differ = 0.0;
+        for (int j = 0; j < G.cs; ++j) {   // rank order
+          const float4 v = ctl->fin_in[d][j];
+          js += v.x; big += v.y; differ += v.z;
         }
-      }
-      if (g_row && ng < na) {
-        const int d = wg.n % kClDepth;
-        if (dead || mbar_test(&ctl->lse_ready[d], (wg.n / kClDepth) & 1u)) {
-          float ms = -INFINITY, ml = -INFINITY;
-          for (int j = 0; j < G.cs; ++j) { ms = fmaxf(ms, ctl->lse_in[d][j].x); ml = fmaxf(ml, ctl->lse_in[d][j].z); }
-          float ss = 0.f, sl = 0.f;
-          for (int j = 0; j < G.cs; ++j) {   // rank order: every CTA of the cluster gets the same bits
-            const float4 v = ctl->lse_in[d][j];
-            ss = fmaf(v.y, ex2_approx(v.x - ms), ss);
-            sl = fmaf(v.w, ex2_approx(v.z - ml), sl);
-          }
-          const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl);
-          if (lane == 0) {
-            RowConsts rc;
-            rc.off_small = ms + l2ss;
-            rc.off_large = ml + l2sl;
-            // logits below the floors give log2 p < -125; the KL variant needs true zeros and clamps nothing
-            rc.floor_small = (DIV == kDivKL) ? -INFINITY : (rc.off_small - 125.f) * inv_c;
-            rc.floor_large = (DIV == kDivKL) ? -INFINITY : (rc.off_large - 125.f) * inv_c;
-            rc.floor2_small = Pairs<T>::floor_bits(rc.floor_small);
-            rc.floor2_large = Pairs<T>::floor_bits(rc.floor_large);
-            rc.pad0 = rc.pad1 = 0u;
-            ctl->row_consts[d] = rc;
-            ctl->row_lse[d] = make_float4(ms, l2ss, ml, l2sl);
-            mbar_arrive(&ctl->b_go[d]);
-          }
-          g_row = wg.advance();
-          ++ng;
-          progressed = true;
+        const float4 lse = ctl->row_lse[d];
+        RowStats st{};
+        int flags = 0;
+        if (!(fabsf(lse.x + lse.y) < INFINITY)) flags |= kFlagSmallNonfinite;   // NaN, +inf, or no finite logit
+        if (!(fabsf(lse.z + lse.w) < INFINITY)) flags |= kFlagLargeNonfinite;
+        if (flags) {
+          st.m2_small = st.l2s_small = st.m2_large = st.l2s_large = st.div = st.resid = __int_as_float(0x7fc00000);
+        } else {
+          double D;
+          const double res = big - 1.0;   // sum max(p,q) - sum q = sum max(0, p - q)
+          if (DIV == kDivJS) D = 0.5 * 0.6931471805599453 * js;   // bits -> nats, and the 1/2 of the definition
+          else if (DIV == kDivKL) D = 0.6931471805599453 * js;
+          else D = res;
+          st.m2_small = lse.x; st.l2s_small = lse.y; st.m2_large = lse.z; st.l2s_large = lse.w;
+          st.div = fmaxf(static_cast<float>(D), 0.f);
+          st.resid = fmaxf(static_cast<float>(res), 0.f);
+          if (differ == 0.0) { st.div = 0.f; st.resid = 0.f; }   // bitwise identical rows: exactly zero
         }
+        st.flags = flags;
+        P.stats[r] = st;
       }
-      if (b_row && nb < ng) {
-        const int d = wb.n % kClDepth;
-        if (dead || mbar_test(&ctl->b_done[d], (wb.n / kClDepth) & 1u)) {
-          float js = 0.f, big = 0.f, differ = 0.f;
-#pragma unroll
-          for (int k = 0; k < kClPassWarps; ++k) {   // warp order
-            const float4 v = ctl->b_part[d][k];
-            js += v.x; big += v.y; differ += v.z;
-          }
-          if (lane == 0) {
-            if (rank == 0) mbar_arrive_expect_tx(&ctl->fin_ready[d], static_cast<unsigned>(G.cs) * 16u);
-            remote_post_f4(map_to_rank(&ctl->fin_in[d][rank], 0), make_float4(js, big, differ, 0.f),
-                           map_to_rank(&ctl->fin_ready[d], 0));
-          }
-          b_row = wb.advance();
-          ++nb;
-          progressed = true;
-        }
+    };
+
+    RowWalk w;
+    w.init(P, cluster_id, G.n_clusters);
+    int prev_n = -1, prev_r = -1;
+    while (w.advance()) {
+      event_a(w.n);
+      event_g(w.n);
+      if (prev_n >= 0) {
+        event_b(prev_n);
+        if (rank == 0) event_f(prev_n, prev_r);
       }
-      if (f_row && nf < nb) {
-        const int d = wf.n % kClDepth;
-        if (dead || mbar_test(&ctl->fin_ready[d], (wf.n / kClDepth) & 1u)) {
-          if (lane == 0) {
-            double js = 0.0, big = 0.0, differ = 0.0;
-            for (int j = 0; j < G.cs; ++j) {   // rank order
-              const float4 v = ctl->fin_in[d][j];
-              js += v.x; big += v.y; differ += v.z;
-            }
-            const float4 lse = ctl->row_lse[d];
-            RowStats st{};
-            int flags = 0;
-            if (!(fabsf(lse.x + lse.y) < INFINITY)) flags |= kFlagSmallNonfinite;   // NaN, +inf, or no finite logit
-            if (!(fabsf(lse.z + lse.w) < INFINITY)) flags |= kFlagLargeNonfinite;
-            if (flags) {
-              st.m2_small = st.l2s_small = st.m2_large = st.l2s_large = st.div = st.resid = __int_as_float(0x7fc00000);
-            } else {
-              double D;
-              const double res = big - 1.0;   // sum max(p,q) - sum q = sum max(0, p - q)
-              if (DIV == kDivJS) D = 0.5 * 0.6931471805599453 * js;   // bits -> nats, and the 1/2 of the definition
-              else if (DIV == kDivKL) D = 0.6931471805599453 * js;
-              else D = res;
-              st.m2_small = lse.x; st.l2s_small = lse.y; st.m2_large = lse.z; st.l2s_large = lse.w;
-              st.div = fmaxf(static_cast<float>(D), 0.f);
-              st.resid = fmaxf(static_cast<float>(res), 0.f);
-              if (differ == 0.0) { st.div = 0.f; st.resid = 0.f; }   // bitwise identical rows: exactly zero
-            }
-            st.flags = flags;
-            P.stats[wf.r] = st;
-          }
-          f_row = wf.advance();
-          ++nf;
-          progressed = true;
-        }
-      }
-      if (progressed) idle = 0;
-      else if (!dead) {
-        if (++idle > kClSpinLimit) give_up();
-        __nanosleep(40);   // the agent shares an issue port with consumer warps: poll gently
-      }
+      prev_n = w.n;
+      prev_r = w.r;
+    }
+    if (prev_n >= 0) {
+      event_b(prev_n);
+      if (rank == 0) event_f(prev_n, prev_r);
     }
   }
   // no CTA may leave while a peer can still write into its shared memory
