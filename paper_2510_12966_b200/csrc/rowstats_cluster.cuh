@@ -407,25 +407,41 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     if (warp < kClPassWarps) {
       // ================================ pass A ================================
       LseState ls, ll;
+      bool landed = false;   // the answer of a test of the next chunk's barrier, asked one chunk early
       while (w.advance()) {
         ls.reset(); ll.reset();
         int off = 0;   // chunk offset inside the slice, in logits
         for (int cidx = 0; cidx < C; ++cidx, off += CH) {
-          wait_phase(&ctl->full[slot], par);
+          if (!landed) wait_phase(&ctl->full[slot], par);
           const unsigned char* base = my + slot * kClSlotBytes;
           uint4 us[kClVecPerLane], ul[kClVecPerLane];
           float ts[kClVecPerLane], tl[kClVecPerLane];
 #pragma unroll
           for (int i = 0; i < kClVecPerLane; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+          if (++slot == static_cast<unsigned>(R)) { slot = 0; par ^= 1u; }
+          landed = mbar_test(&ctl->full[slot], par);   // its latency hides behind this chunk's arithmetic
           const float ref_s = ls.ref, ref_l = ll.ref;
-#pragma unroll
-          for (int i = 0; i < kClVecPerLane; ++i) { ts[i] = lse_vector_sum<T>(us[i], c, ref_s); tl[i] = lse_vector_sum<T>(ul[i], c, ref_l); }
+          bool bad = false;
 #pragma unroll
           for (int i = 0; i < kClVecPerLane; ++i) {
-            lse_commit<T>(ts[i], ref_s, us[i], len[i] > off, c, ls);
-            lse_commit<T>(tl[i], ref_l, ul[i], len[i] > off, c, ll);
+            ts[i] = lse_vector_sum<T>(us[i], c, ref_s);
+            tl[i] = lse_vector_sum<T>(ul[i], c, ref_l);
+            bad |= (len[i] > off) && !(ts[i] + tl[i] < INFINITY);
           }
-          if (++slot == static_cast<unsigned>(R)) { slot = 0; par ^= 1u; }
+          // one vote per chunk: only a non-finite vector sum sends the warp through the careful commits
+          if (!__any_sync(0xffffffffu, bad)) {
+#pragma unroll
+            for (int i = 0; i < kClVecPerLane; ++i) {
+              ls.s += (len[i] > off) ? ts[i] : 0.f;
+              ll.s += (len[i] > off) ? tl[i] : 0.f;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < kClVecPerLane; ++i) {
+              lse_commit<T>(ts[i], ref_s, us[i], len[i] > off, c, ls);
+              lse_commit<T>(tl[i], ref_l, ul[i], len[i] > off, c, ll);
+            }
+          }
         }
         // row finished: the warp's partial (one reference, summed S) -> a_part, then tell the agent
         const float ss = warp_reduce<OpSum>(ls.s), sl = warp_reduce<OpSum>(ll.s);
