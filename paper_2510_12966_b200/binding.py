@@ -63,7 +63,7 @@ def load_library(path: Optional[str] = None):
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = path or LIB_PATH
+    p = path or os.environ.get("PYRAMIDSD_LIB") or LIB_PATH   # PYRAMIDSD_LIB: another build of the same library
     if not os.path.exists(p):
         raise ImportError(f"{p} is missing: build it with `python -m paper_2510_12966_b200.build` "
                           "(there is no CPU fallback for the verification path)")

@@ -27,12 +27,21 @@
 
 namespace psd {
 
-constexpr int kClPassWarps = 8;                    // warps per pass (A: 0..7, B: 8..15)
-constexpr int kClConsumerWarps = 2 * kClPassWarps;
+#ifndef PSD_A_WARPS
+#define PSD_A_WARPS 8
+#endif
+#ifndef PSD_B_WARPS
+#define PSD_B_WARPS 8
+#endif
+constexpr int kClAWarps = PSD_A_WARPS;             // warps running pass A (0 .. kClAWarps - 1)
+constexpr int kClBWarps = PSD_B_WARPS;             // warps running pass B (the next kClBWarps)
+constexpr int kClConsumerWarps = kClAWarps + kClBWarps;
 constexpr int kClConsumers = kClConsumerWarps * 32;
-constexpr int kClThreads = kClConsumers + 64;      // + loader warp + agent warp
+constexpr int kClThreads = kClConsumers + 96;      // + loader warp + two agent warps
 constexpr int kClHalfBytes = 8192;                 // one model's part of a chunk: 256 threads x 2 x 16 bytes
-constexpr int kClVecPerLane = 2;                   // 16-byte vectors per lane, chunk and model
+constexpr int kClAVec = 16 / kClAWarps;            // 16-byte vectors per lane, chunk and model in pass A
+constexpr int kClBVec = 16 / kClBWarps;            // ... and in pass B
+static_assert(kClAVec * kClAWarps == 16 && kClBVec * kClBWarps == 16, "the 512 vectors of a chunk must split evenly");
 constexpr int kClSlotBytes = 2 * kClHalfBytes;
 constexpr int kClSlots = 13;                       // ring slots
 constexpr int kClDepth = 4;                        // rows of exchange buffers in flight
@@ -60,12 +69,13 @@ struct __align__(16) ClusterCtl {
   unsigned long long full[kClSlots];
   unsigned long long empty[kClSlots];
   unsigned long long a_done[kClDepth], b_done[kClDepth], lse_ready[kClDepth], fin_ready[kClDepth], b_go[kClDepth];
-  float4 a_part[kClDepth][kClPassWarps];           // (ref_small, sum_small, ref_large, sum_large) per pass-A warp
-  float4 b_part[kClDepth][kClPassWarps];           // (divergence sum in bits, sum max(p,q), rows differ, unused) per pass-B warp
+  float4 a_part[kClDepth][kClAWarps];              // (ref_small, sum_small, ref_large, sum_large) per pass-A warp
+  float4 b_part[kClDepth][kClBWarps];              // (divergence sum in bits, sum max(p,q), rows differ, unused) per pass-B warp
   float4 row_lse[kClDepth];                        // (m2_small, l2s_small, m2_large, l2s_large) of the row
   RowConsts row_consts[kClDepth];                  // what pass B needs of the row, published by the agent
   float4 lse_in[kClDepth][kClMaxRanks];            // partials received from every rank of the cluster
   float4 fin_in[kClDepth][kClMaxRanks];            // pass-B partials received (rank 0 only)
+  int rows_closed;                                 // rows whose pass-B partials the second agent has dealt with
 };
 
 constexpr size_t kClSmemBytes = static_cast<size_t>(kClSlots) * kClSlotBytes + sizeof(ClusterCtl) + 128;
@@ -267,6 +277,18 @@ __device__ __noinline__ float lse_slow_path(uint4 u, bool live, float c, float r
   return t;
 }
 
+// Largest logit of one vector (-inf when the vector lies outside the slice), NaN ignored.
+template <typename T>
+__device__ __forceinline__ float vector_max(const uint4& u, bool live) {
+  constexpr int N = Pairs<T>::kN;
+  float2 x[N];
+  Pairs<T>::load(u, x);
+  float gm = fmaxf(x[0].x, x[0].y);
+#pragma unroll
+  for (int j = 1; j < N; ++j) gm = fmaxf(gm, fmaxf(x[j].x, x[j].y));
+  return live ? gm : -INFINITY;
+}
+
 // Add one vector sum, taken against `ref_used`, to the state; all 32 lanes call this together. When an
 // earlier vector of the same step has moved the reference the sum is taken again, so that the result
 // does not depend on how many vectors a step happened to group.
@@ -365,10 +387,11 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
   const int C = G.chunks, R = G.ring;
 
   if (tid == 0) {
-    for (int s = 0; s < kClSlots; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], kClPassWarps); }
+    ctl->rows_closed = 0;
+    for (int s = 0; s < kClSlots; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], kClBWarps); }
     for (int d = 0; d < kClDepth; ++d) {
-      mbar_init(&ctl->a_done[d], kClPassWarps);
-      mbar_init(&ctl->b_done[d], kClPassWarps);
+      mbar_init(&ctl->a_done[d], kClAWarps);
+      mbar_init(&ctl->b_done[d], kClBWarps);
       mbar_init(&ctl->lse_ready[d], 1);   // the local agent's arrive; the peers' partials count as bytes
       mbar_init(&ctl->fin_ready[d], 1);
       mbar_init(&ctl->b_go[d], 1);
@@ -393,18 +416,21 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
 
   if (warp < kClConsumerWarps) {
     const float c = P.c;
-    const int pw = warp % kClPassWarps;               // index among the warps of this pass
-    // vectors pw*32 + lane and that + 256 of every chunk; `len[i]` > chunk offset while vector i lies inside the slice
+    const bool is_a = warp < kClAWarps;
+    const int pw = is_a ? warp : warp - kClAWarps;    // index among the warps of this pass
+    const int pass_warps = is_a ? kClAWarps : kClBWarps;
+    // vectors pw*32 + lane + i * pass_warps * 32 of every chunk; `len[i]` > chunk offset while vector i lies inside the slice
     const unsigned char* my = ring + (pw * 32 + lane) * 16;
-    int len[kClVecPerLane];
+    constexpr int kMaxVec = kClAVec > kClBVec ? kClAVec : kClBVec;
+    int len[kMaxVec];
 #pragma unroll
-    for (int i = 0; i < kClVecPerLane; ++i) len[i] = slice_len - (pw * 32 + lane + i * kClPassWarps * 32) * E;
-    constexpr int kVecStride = kClPassWarps * 32 * 16;   // bytes between a lane's two vectors
+    for (int i = 0; i < kMaxVec; ++i) len[i] = slice_len - (pw * 32 + lane + i * pass_warps * 32) * E;
     RowWalk w;
     w.init(P, cluster_id, G.n_clusters);
     unsigned slot = 0, par = 0;
 
-    if (warp < kClPassWarps) {
+    if (is_a) {
+      constexpr int kVecStride = kClAWarps * 32 * 16;   // bytes between a lane's vectors
       // ================================ pass A ================================
       LseState ls, ll;
       bool landed = false;   // the answer of a test of the next chunk's barrier, asked one chunk early
@@ -414,16 +440,28 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
         for (int cidx = 0; cidx < C; ++cidx, off += CH) {
           if (!landed) wait_phase(&ctl->full[slot], par);
           const unsigned char* base = my + slot * kClSlotBytes;
-          uint4 us[kClVecPerLane], ul[kClVecPerLane];
-          float ts[kClVecPerLane], tl[kClVecPerLane];
+          uint4 us[kClAVec], ul[kClAVec];
+          float ts[kClAVec], tl[kClAVec];
 #pragma unroll
-          for (int i = 0; i < kClVecPerLane; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+          for (int i = 0; i < kClAVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
           if (++slot == static_cast<unsigned>(R)) { slot = 0; par ^= 1u; }
           landed = mbar_test(&ctl->full[slot], par);   // its latency hides behind this chunk's arithmetic
+          if (cidx == 0) {
+            // start the row at the warp's largest logit of its first vectors, so that the first chunk does
+            // not have to find its reference through the slow path (the floor keeps -inf rows at 0)
+            float gs = vector_max<T>(us[0], len[0] > 0), gl = vector_max<T>(ul[0], len[0] > 0);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              gs = fmaxf(gs, __shfl_xor_sync(0xffffffffu, gs, o));
+              gl = fmaxf(gl, __shfl_xor_sync(0xffffffffu, gl, o));
+            }
+            ls.ref = fmaxf(gs * c, -1e30f);
+            ll.ref = fmaxf(gl * c, -1e30f);
+          }
           const float ref_s = ls.ref, ref_l = ll.ref;
           bool bad = false;
 #pragma unroll
-          for (int i = 0; i < kClVecPerLane; ++i) {
+          for (int i = 0; i < kClAVec; ++i) {
             ts[i] = lse_vector_sum<T>(us[i], c, ref_s);
             tl[i] = lse_vector_sum<T>(ul[i], c, ref_l);
             bad |= (len[i] > off) && !(ts[i] + tl[i] < INFINITY);
@@ -431,13 +469,13 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
           // one vote per chunk: only a non-finite vector sum sends the warp through the careful commits
           if (!__any_sync(0xffffffffu, bad)) {
 #pragma unroll
-            for (int i = 0; i < kClVecPerLane; ++i) {
+            for (int i = 0; i < kClAVec; ++i) {
               ls.s += (len[i] > off) ? ts[i] : 0.f;
               ll.s += (len[i] > off) ? tl[i] : 0.f;
             }
           } else {
 #pragma unroll
-            for (int i = 0; i < kClVecPerLane; ++i) {
+            for (int i = 0; i < kClAVec; ++i) {
               lse_commit<T>(ts[i], ref_s, us[i], len[i] > off, c, ls);
               lse_commit<T>(tl[i], ref_l, ul[i], len[i] > off, c, ll);
             }
@@ -454,6 +492,7 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     } else {
       // ================================ pass B ================================
       constexpr int N = Pairs<T>::kN;
+      constexpr int kVecStride = kClBWarps * 32 * 16;   // bytes between a lane's vectors
       while (w.advance()) {
         const int d = w.n % kClDepth;
         wait_phase(&ctl->b_go[d], (w.n / kClDepth) & 1u);   // the row's constants are published: pass A is through
@@ -463,11 +502,11 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
         int off = 0;
         for (int cidx = 0; cidx < C; ++cidx, off += CH) {
           const unsigned char* base = my + slot * kClSlotBytes;
-          uint4 us[kClVecPerLane], ul[kClVecPerLane];
+          uint4 us[kClBVec], ul[kClBVec];
 #pragma unroll
-          for (int i = 0; i < kClVecPerLane; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+          for (int i = 0; i < kClBVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
 #pragma unroll
-          for (int i = 0; i < kClVecPerLane; ++i) {
+          for (int i = 0; i < kClBVec; ++i) {
             float2 xs[N], xl[N];
             Pairs<T>::load_clamped(us[i], rc.floor_small, rc.floor2_small, xs);
             Pairs<T>::load_clamped(ul[i], rc.floor_large, rc.floor2_large, xl);
@@ -530,11 +569,11 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     //   g(n)  every rank's partial of row n has arrived     -> row constants for pass B, release the consumers
     //   b(n)  the warps' pass-B partials of row n are in    -> sum, send to rank 0
     //   f(n)  (rank 0) every rank's pass-B partial arrived  -> write the row's statistics
-    // taken in the fixed order a(n), g(n), b(n-1), f(n-1), which is the order the pipelined schedule completes
-    // them in, so every wait is a blocking wait on one barrier and the agent costs the consumer warps that
-    // share its issue port next to nothing. The order also keeps the exchange buffers safe: they are
-    // kClDepth rows deep, nothing of row m can be produced anywhere in the cluster before this agent has sent
-    // a(m), and a(m) comes after g(m-1), b(m-2) and f(m-2).
+    // shared by two agent warps: one takes a(n), g(n) in row order (the path that releases pass B), the other
+    // b(n), f(n). Every wait is a blocking wait on one barrier, so the agents cost the consumer warps that
+    // share their issue ports next to nothing. The exchange buffers are kClDepth rows deep; nothing of row m
+    // can be produced anywhere in the cluster before a(m) has been sent, a(m) comes after g(m-1), and the
+    // first agent holds a(m) back until the second one has closed row m - kClDepth + 1.
     const float inv_c = 1.f / P.c;
 
     auto event_a = [&](int n) {
@@ -543,10 +582,10 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       // merge the warps' partials (every lane does the same arithmetic, warp order) ...
       float ms = -1e30f, ml = -1e30f;
 #pragma unroll
-      for (int k = 0; k < kClPassWarps; ++k) { ms = fmaxf(ms, ctl->a_part[d][k].x); ml = fmaxf(ml, ctl->a_part[d][k].z); }
+      for (int k = 0; k < kClAWarps; ++k) { ms = fmaxf(ms, ctl->a_part[d][k].x); ml = fmaxf(ml, ctl->a_part[d][k].z); }
       float ss = 0.f, sl = 0.f;
 #pragma unroll
-      for (int k = 0; k < kClPassWarps; ++k) {
+      for (int k = 0; k < kClAWarps; ++k) {
         const float4 v = ctl->a_part[d][k];
         ss = fmaf(v.y, ex2_approx(v.x - ms), ss);
         sl = fmaf(v.w, ex2_approx(v.z - ml), sl);
@@ -560,13 +599,24 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     auto event_g = [&](int n) {
       const int d = n % kClDepth;
       wait_phase(&ctl->lse_ready[d], (n / kClDepth) & 1u);
-      float ms = -INFINITY, ml = -INFINITY;
-      for (int j = 0; j < G.cs; ++j) { ms = fmaxf(ms, ctl->lse_in[d][j].x); ml = fmaxf(ml, ctl->lse_in[d][j].z); }
-      float ss = 0.f, sl = 0.f;
-      for (int j = 0; j < G.cs; ++j) {   // rank order: every CTA of the cluster gets the same bits
-        const float4 v = ctl->lse_in[d][j];
-        ss = fmaf(v.y, ex2_approx(v.x - ms), ss);
-        sl = fmaf(v.w, ex2_approx(v.z - ml), sl);
+      // rank order, so that every CTA of the cluster gets the same bits; four ranks at a time keeps the
+      // loads and exps of a group independent of each other (this sits on the path that releases pass B)
+      float ms = -1e30f, ml = -1e30f, ss = 0.f, sl = 0.f;
+      for (int j0 = 0; j0 < G.cs; j0 += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = (j0 + j < G.cs) ? ctl->lse_in[d][j0 + j] : make_float4(-1e30f, 0.f, -1e30f, 0.f);
+        const float gs = fmaxf(fmaxf(v[0].x, v[1].x), fmaxf(v[2].x, v[3].x));
+        const float gl = fmaxf(fmaxf(v[0].z, v[1].z), fmaxf(v[2].z, v[3].z));
+        const float ns = fmaxf(ms, gs), nl = fmaxf(ml, gl);
+        ss *= ex2_approx(ms - ns);
+        sl *= ex2_approx(ml - nl);
+        ms = ns; ml = nl;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          ss = fmaf(v[j].y, ex2_approx(v[j].x - ms), ss);
+          sl = fmaf(v[j].w, ex2_approx(v[j].z - ml), sl);
+        }
       }
       const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl);
       if (lane == 0) {
@@ -589,7 +639,7 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       wait_phase(&ctl->b_done[d], (n / kClDepth) & 1u);
       float js = 0.f, big = 0.f, differ = 0.f;
 #pragma unroll
-      for (int k = 0; k < kClPassWarps; ++k) {   // warp order
+      for (int k = 0; k < kClBWarps; ++k) {   // warp order
         const float4 v = ctl->b_part[d][k];
         js += v.x; big += v.y; differ += v.z;
       }
@@ -603,7 +653,7 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       const int d = n % kClDepth;
       wait_phase(&ctl->fin_ready[d], (n / kClDepth) & 1u);
       if (lane == 0) {
-        double js = 0.0, big = 0.0, differ = 0.0;
+        float js = 0.f, big = 0.f, differ = 0.f;
         for (int j = 0; j < G.cs; ++j) {   // rank order
           const float4 v = ctl->fin_in[d][j];
           js += v.x; big += v.y; differ += v.z;
@@ -616,15 +666,15 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
         if (flags) {
           st.m2_small = st.l2s_small = st.m2_large = st.l2s_large = st.div = st.resid = __int_as_float(0x7fc00000);
         } else {
-          double D;
-          const double res = big - 1.0;   // sum max(p,q) - sum q = sum max(0, p - q)
-          if (DIV == kDivJS) D = 0.5 * 0.6931471805599453 * js;   // bits -> nats, and the 1/2 of the definition
-          else if (DIV == kDivKL) D = 0.6931471805599453 * js;
+          float D;
+          const float res = big - 1.f;   // sum max(p,q) - sum q = sum max(0, p - q)
+          if (DIV == kDivJS) D = (0.5f * kLn2) * js;   // bits -> nats, and the 1/2 of the definition
+          else if (DIV == kDivKL) D = kLn2 * js;
           else D = res;
           st.m2_small = lse.x; st.l2s_small = lse.y; st.m2_large = lse.z; st.l2s_large = lse.w;
-          st.div = fmaxf(static_cast<float>(D), 0.f);
-          st.resid = fmaxf(static_cast<float>(res), 0.f);
-          if (differ == 0.0) { st.div = 0.f; st.resid = 0.f; }   // bitwise identical rows: exactly zero
+          st.div = fmaxf(D, 0.f);
+          st.resid = fmaxf(res, 0.f);
+          if (differ == 0.f) { st.div = 0.f; st.resid = 0.f; }   // bitwise identical rows: exactly zero
         }
         st.flags = flags;
         P.stats[r] = st;
@@ -633,20 +683,24 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
 
     RowWalk w;
     w.init(P, cluster_id, G.n_clusters);
-    int prev_n = -1, prev_r = -1;
-    while (w.advance()) {
-      event_a(w.n);
-      event_g(w.n);
-      if (prev_n >= 0) {
-        event_b(prev_n);
-        if (rank == 0) event_f(prev_n, prev_r);
+    if (warp == kClConsumerWarps + 1) {
+      // first agent: a(n), g(n) -- the path that releases pass B
+      while (w.advance()) {
+        // row n reuses the buffers of row n - kClDepth: the second agent must be through with that row
+        unsigned spins = 0;
+        while (!dead && *reinterpret_cast<volatile int*>(&ctl->rows_closed) < w.n - (kClDepth - 2))
+          if (++spins > kClSpinLimit) give_up();
+        event_a(w.n);
+        event_g(w.n);
       }
-      prev_n = w.n;
-      prev_r = w.r;
-    }
-    if (prev_n >= 0) {
-      event_b(prev_n);
-      if (rank == 0) event_f(prev_n, prev_r);
+    } else {
+      // second agent: b(n), f(n) -- off the critical path
+      while (w.advance()) {
+        event_b(w.n);
+        if (rank == 0) event_f(w.n, w.r);
+        __syncwarp();
+        if (lane == 0) *reinterpret_cast<volatile int*>(&ctl->rows_closed) = w.n + 1;
+      }
     }
   }
   // no CTA may leave while a peer can still write into its shared memory
