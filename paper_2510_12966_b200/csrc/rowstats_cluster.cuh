@@ -246,6 +246,19 @@ __device__ __forceinline__ float lse_vector_sum(const uint4& u, float c, float r
   return v.x + v.y;
 }
 
+// the same as a packed pair of partial sums (their total is the vector sum)
+template <typename T>
+__device__ __forceinline__ float2 lse_vector_sum2(const uint4& u, float c, float ref) {
+  constexpr int N = Pairs<T>::kN;
+  float2 x[N];
+  Pairs<T>::load(u, x);
+  const float2 cc = splat2(c), nref = splat2(-ref);
+  float2 v = ex2_2(__ffma2_rn(x[0], cc, nref));
+#pragma unroll
+  for (int j = 1; j < N; ++j) v = __fadd2_rn(v, ex2_2(__ffma2_rn(x[j], cc, nref)));
+  return v;
+}
+
 // Warp-wide: move the reference up to the largest logit of this vector (over the live lanes) and
 // return this lane's vector sum against the new reference.
 template <typename T>
@@ -432,23 +445,28 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
     if (is_a) {
       constexpr int kVecStride = kClAWarps * 32 * 16;   // bytes between a lane's vectors
       // ================================ pass A ================================
+      // A row is summed optimistically against one reference per model, taken from the warp's first
+      // vectors: no vote and no dependent branch per chunk, so the exps of consecutive chunks pipeline
+      // freely. Only if some lane's row sum comes out non-finite (a logit more than 2^127 above that
+      // reference, or NaN / +inf) is the row redone through the careful per-vector commits -- its chunks
+      // are all still in the ring, because pass B cannot enter the row before pass A has left it.
       LseState ls, ll;
       bool landed = false;   // the answer of a test of the next chunk's barrier, asked one chunk early
       while (w.advance()) {
         ls.reset(); ll.reset();
+        const unsigned slot0 = slot;   // where the row starts in the ring
+        float2 vs = make_float2(0.f, 0.f), vl = vs;
         int off = 0;   // chunk offset inside the slice, in logits
         for (int cidx = 0; cidx < C; ++cidx, off += CH) {
           if (!landed) wait_phase(&ctl->full[slot], par);
           const unsigned char* base = my + slot * kClSlotBytes;
           uint4 us[kClAVec], ul[kClAVec];
-          float ts[kClAVec], tl[kClAVec];
 #pragma unroll
           for (int i = 0; i < kClAVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
           if (++slot == static_cast<unsigned>(R)) { slot = 0; par ^= 1u; }
           landed = mbar_test(&ctl->full[slot], par);   // its latency hides behind this chunk's arithmetic
           if (cidx == 0) {
-            // start the row at the warp's largest logit of its first vectors, so that the first chunk does
-            // not have to find its reference through the slow path (the floor keeps -inf rows at 0)
+            // the warp's largest logit of its first vectors (the floor keeps rows that start with -inf at 0)
             float gs = vector_max<T>(us[0], len[0] > 0), gl = vector_max<T>(ul[0], len[0] > 0);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
@@ -458,27 +476,32 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
             ls.ref = fmaxf(gs * c, -1e30f);
             ll.ref = fmaxf(gl * c, -1e30f);
           }
-          const float ref_s = ls.ref, ref_l = ll.ref;
-          bool bad = false;
 #pragma unroll
           for (int i = 0; i < kClAVec; ++i) {
-            ts[i] = lse_vector_sum<T>(us[i], c, ref_s);
-            tl[i] = lse_vector_sum<T>(ul[i], c, ref_l);
-            bad |= (len[i] > off) && !(ts[i] + tl[i] < INFINITY);
+            const float2 ps = lse_vector_sum2<T>(us[i], c, ls.ref), pl = lse_vector_sum2<T>(ul[i], c, ll.ref);
+            const bool live = len[i] > off;
+            vs = __fadd2_rn(vs, live ? ps : make_float2(0.f, 0.f));
+            vl = __fadd2_rn(vl, live ? pl : make_float2(0.f, 0.f));
           }
-          // one vote per chunk: only a non-finite vector sum sends the warp through the careful commits
-          if (!__any_sync(0xffffffffu, bad)) {
-#pragma unroll
+        }
+        ls.s = vs.x + vs.y;
+        ll.s = vl.x + vl.y;
+        if (__any_sync(0xffffffffu, !(ls.s + ll.s < INFINITY))) {
+          // careful second go over the row's chunks, vector by vector, moving the references as needed
+          ls.s = 0.f; ll.s = 0.f;
+          unsigned sl2 = slot0;
+          off = 0;
+#pragma unroll 1
+          for (int cidx = 0; cidx < C; ++cidx, off += CH) {
+            const unsigned char* base = my + sl2 * kClSlotBytes;
+#pragma unroll 1
             for (int i = 0; i < kClAVec; ++i) {
-              ls.s += (len[i] > off) ? ts[i] : 0.f;
-              ll.s += (len[i] > off) ? tl[i] : 0.f;
+              const bool live = (slice_len - (pw * 32 + lane + i * kClAWarps * 32) * E) > off;
+              // a NaN "reference used" makes the commit take the vector sum afresh
+              lse_commit<T>(0.f, __int_as_float(0x7fc00000), lds128(base + i * kVecStride), live, c, ls);
+              lse_commit<T>(0.f, __int_as_float(0x7fc00000), lds128(base + kClHalfBytes + i * kVecStride), live, c, ll);
             }
-          } else {
-#pragma unroll
-            for (int i = 0; i < kClAVec; ++i) {
-              lse_commit<T>(ts[i], ref_s, us[i], len[i] > off, c, ls);
-              lse_commit<T>(tl[i], ref_l, ul[i], len[i] > off, c, ll);
-            }
+            if (++sl2 == static_cast<unsigned>(R)) sl2 = 0;
           }
         }
         // row finished: the warp's partial (one reference, summed S) -> a_part, then tell the agent
