@@ -169,6 +169,10 @@ def run_ours(args):
     n_pos = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(args.steps))
     row_bytes = 2 * w.V * es
     rs_bytes = n_pos * row_bytes   # the statistics kernel streams each verified row pair once
+    timed_cap = 4096               # launches the library's event timing holds; beyond it only the first ones are timed
+    if 4 * args.steps > timed_cap:
+        steps_timed = timed_cap // 4
+        rs_bytes = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(steps_timed)) * row_bytes
 
     # ---- end to end through the host-pointer entry point: H2D of the step's inputs + D2H of its results ----
     e2e = None
