@@ -3,8 +3,8 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2] [--impl ours|reference]
 
-A step is one pass of the whole hot path — pyramidsd_verify: stage-1 statistics + finalisation, window
-build, stage-2 statistics + finalisation — over one batch of seeded synthetic logits (the BASELINE
+A step is one pass of the whole hot path — pyramidsd_verify: the statistics of both stages' rows in one
+launch, then stage-1 finalisation, window build and stage-2 finalisation in another — over one batch of seeded synthetic logits (the BASELINE
 "batched serving" configuration by default: B=64, V=128256, bf16, K_draft=16, K_qual=8). Metric: verified
 positions per second (a position = one row pair actually verified: all B*K_d stage-1 rows plus the
 stage-2 rows inside each sequence's window). Prints ONE JSON line on rank 0.
@@ -170,8 +170,9 @@ def run_ours(args):
     row_bytes = 2 * w.V * es
     rs_bytes = n_pos * row_bytes   # the statistics kernel streams each verified row pair once
     timed_cap = 4096               # launches the library's event timing holds; beyond it only the first ones are timed
-    if 4 * args.steps > timed_cap:
-        steps_timed = timed_cap // 4
+    launches_per_step = 2          # one statistics launch (both stages' rows) and one finalisation launch
+    if launches_per_step * args.steps > timed_cap:
+        steps_timed = timed_cap // launches_per_step
         rs_bytes = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(steps_timed)) * row_bytes
 
     # ---- end to end through the host-pointer entry point: H2D of the step's inputs + D2H of its results ----

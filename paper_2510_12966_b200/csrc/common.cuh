@@ -54,6 +54,13 @@ struct StageParams {
   int32_t* n_window;
   int K_window;
   int* status;        // device status word (bounded-wait timeouts)
+  // Second row set of the statistics pass (two-stage wrapper): rows [B*K, B*K + B*K2) of the launch are
+  // the stage-2 pairs (qualifier as the small model, target as the large one). K2 == 0: none.
+  const void* small2;
+  const void* large2;
+  long long seq_stride_small2, seq_stride_large2;
+  int K2;
+  RowStats* stats2;
 };
 
 // ---- special functions (single MUFU instruction each) -------------------------------------------------

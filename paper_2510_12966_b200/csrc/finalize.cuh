@@ -14,6 +14,7 @@ constexpr int kFinThreads = 1024;
 constexpr int kFinElemsPerThread = 8;                      // consecutive vocabulary indices per thread and tile
 constexpr int kFinTile = kFinThreads * kFinElemsPerThread;  // 8192 indices per tile
 constexpr int kFinMaxTiles = 1024;                          // V <= 8,388,608
+constexpr int kFinBatch = 32;                               // tiles summed between two CTA-wide barriers
 
 template <typename T>
 struct RowView {
@@ -51,15 +52,24 @@ struct RowView {
   }
 };
 
-template <typename T>
-__global__ void __launch_bounds__(kFinThreads) finalize_kernel(const StageParams P) {
-  __shared__ double tile_total[kFinMaxTiles];
-  __shared__ float warp_total[32];
-  __shared__ double scratch[32];
-  __shared__ int sh_L, sh_nv, sh_flags, sh_tile, sh_warp, sh_token;
-  __shared__ float sh_u2, sh_m2l, sh_l2sl, sh_m2s, sh_l2ss, sh_resid, sh_target;
+struct FinShared {
+  double tile_total[kFinMaxTiles];
+  float warp_total[32];
+  float warp_tile[kFinBatch][32];   // per-warp sums of a batch of tiles
+  int sh_L, sh_nv, sh_flags, sh_tile, sh_warp, sh_token;
+  float sh_u2, sh_m2l, sh_l2sl, sh_m2s, sh_l2ss, sh_resid, sh_target;
+};
 
-  const int b = blockIdx.x;
+// One stage's finalisation of sequence b; every thread of the CTA calls it.
+template <typename T>
+__device__ __forceinline__ void finalize_sequence(const StageParams& P, const int b, FinShared& S) {
+  double (&tile_total)[kFinMaxTiles] = S.tile_total;
+  float (&warp_total)[32] = S.warp_total;
+  float (&warp_tile)[kFinBatch][32] = S.warp_tile;
+  int &sh_L = S.sh_L, &sh_nv = S.sh_nv, &sh_flags = S.sh_flags, &sh_tile = S.sh_tile, &sh_warp = S.sh_warp, &sh_token = S.sh_token;
+  float &sh_u2 = S.sh_u2, &sh_m2l = S.sh_m2l, &sh_l2sl = S.sh_l2sl, &sh_m2s = S.sh_m2s, &sh_l2ss = S.sh_l2ss,
+        &sh_resid = S.sh_resid, &sh_target = S.sh_target;
+
   const int K = P.K, V = P.V;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const T* large_seq = static_cast<const T*>(P.large) + b * P.seq_stride_large;
@@ -144,16 +154,27 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(const StageParams
 
     const int n_tiles = (V + kFinTile - 1) / kFinTile;
     float w[kFinElemsPerThread];
-    // level 0: total weight of every tile
-    for (int j = 0; j < n_tiles; ++j) {
-      row.weights(j * kFinTile + tid * kFinElemsPerThread, w);
-      float ts = 0.f;
+    // level 0: total weight of every tile. The tiles of a batch are independent (their loads overlap);
+    // each warp leaves its sum per tile, then one thread per tile adds the 32 warp sums in warp order.
+    for (int j0 = 0; j0 < n_tiles; j0 += kFinBatch) {
+      const int nb = min(kFinBatch, n_tiles - j0);
+#pragma unroll 4
+      for (int j = 0; j < nb; ++j) {
+        row.weights((j0 + j) * kFinTile + tid * kFinElemsPerThread, w);
+        float ts = 0.f;
 #pragma unroll
-      for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
-      const double tt = block_reduce<OpSum>(static_cast<double>(ts), scratch, 0.0);
-      if (tid == 0) tile_total[j] = tt;
+        for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
+        ts = warp_reduce<OpSum>(ts);
+        if (lane == 0) warp_tile[j][warp] = ts;
+      }
+      __syncthreads();
+      if (tid < nb) {
+        double tt = 0.0;
+        for (int k = 0; k < 32; ++k) tt += static_cast<double>(warp_tile[tid][k]);
+        tile_total[j0 + tid] = tt;
+      }
+      __syncthreads();
     }
-    __syncthreads();
     if (tid == 0) {
       double total = 0.0;
       for (int j = 0; j < n_tiles; ++j) total += tile_total[j];
@@ -246,6 +267,24 @@ __global__ void __launch_bounds__(kFinThreads) finalize_kernel(const StageParams
         P.window[b * P.K_window + j] = (j < n2) ? ((j < L) ? P.tokens[b * K + j] : next) : 0;
     }
   }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads) finalize_kernel(const StageParams P) {
+  __shared__ FinShared S;
+  finalize_sequence<T>(P, blockIdx.x, S);
+}
+
+// Both stages of the two-stage wrapper for one sequence: stage 1 (draft against qualifier) writes the
+// window and its length, stage 2 (window against target) reads them back. The statistics of every
+// stage-2 row were computed beforehand, whatever the window turned out to be.
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads) finalize_pyramid_kernel(const StageParams P1, const StageParams P2) {
+  __shared__ FinShared S;
+  finalize_sequence<T>(P1, blockIdx.x, S);
+  __threadfence_block();
+  __syncthreads();   // the window and its length, written by thread 0, are visible to the whole CTA
+  finalize_sequence<T>(P2, blockIdx.x, S);
 }
 
 }  // namespace psd

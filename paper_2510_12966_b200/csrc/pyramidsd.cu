@@ -145,7 +145,7 @@ int check_launch() {
 // Statistics pass for one stage: picks the kernel variant and launches it.
 int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_size, cudaStream_t stream) {
   const long long rows = static_cast<long long>(P.B) * P.K;
-  if (rows == 0) return PSD_OK;
+  if (rows == 0 && P.K2 == 0) return PSD_OK;
   bool use_cluster = false;
   psd::ClusterGeom geom{};
   if (variant == PSD_KERNEL_CLUSTER || variant == PSD_KERNEL_AUTO) {
@@ -160,9 +160,22 @@ int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_si
       return PSD_ERR_CUDA;
     }
   } else {
-    const dim3 grid(static_cast<unsigned>(rows)), block(1024);
-    if (dtype == PSD_F32) psd::rowstats_baseline_kernel<float><<<grid, block, 0, stream>>>(P);
-    else psd::rowstats_baseline_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(P);
+    const dim3 block(1024);
+    if (rows > 0) {
+      const dim3 grid(static_cast<unsigned>(rows));
+      if (dtype == PSD_F32) psd::rowstats_baseline_kernel<float><<<grid, block, 0, stream>>>(P);
+      else psd::rowstats_baseline_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(P);
+    }
+    if (P.K2 > 0) {   // the second row set as a launch of its own
+      StageParams Q = P;
+      Q.small = P.small2; Q.large = P.large2;
+      Q.seq_stride_small = P.seq_stride_small2; Q.seq_stride_large = P.seq_stride_large2;
+      Q.K = P.K2; Q.K2 = 0; Q.stats = P.stats2; Q.n_valid = nullptr;
+      const dim3 grid(static_cast<unsigned>(static_cast<long long>(P.B) * P.K2));
+      if (dtype == PSD_F32) psd::rowstats_baseline_kernel<float><<<grid, block, 0, stream>>>(Q);
+      else psd::rowstats_baseline_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(Q);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
   }
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return check_launch();
@@ -313,9 +326,6 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   s1.stream = stream;
   s1.use_stream_field = 1;
   s1.kernel_variant = variant;
-  rc = run_stage(&s1, window, n_window, K_q);
-  if (rc != PSD_OK) return rc;
-
   psd_stage_args s2 = s1;
   s2.logits_small = logits_qual;   // P_MQ takes the place of P_MD in the target comparison (Fig. 1)
   s2.logits_large = logits_target;
@@ -330,7 +340,40 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   s2.out_next_token = out_next_token;
   s2.workspace = base + ws1;
   s2.workspace_bytes = ws2;
-  return run_stage(&s2, nullptr, nullptr, 0);
+  rc = validate_stage(&s1);
+  if (rc == PSD_OK) rc = validate_stage(&s2);
+  if (rc != PSD_OK) return rc;
+  {
+    std::lock_guard<std::mutex> lock(ds->mu);
+    rc = ensure_status(ds);
+    if (rc != PSD_OK) return rc;
+  }
+  // Two launches for the whole pyramid. The statistics of both stages are independent of the stage-1
+  // outcome (only the token looked up in a row and the window length depend on it), so one launch of
+  // the statistics kernel covers the B*K_d stage-1 rows and the B*K_q stage-2 rows; one finalisation
+  // kernel then runs stage 1, builds the window, and runs stage 2 per sequence.
+  StageParams P1 = make_params(&s1, s1.workspace, ds->status);
+  P1.window = window;
+  P1.n_window = n_window;
+  P1.K_window = K_q;
+  const StageParams P2 = make_params(&s2, s2.workspace, ds->status);
+  StageParams PS = P1;
+  PS.small2 = P2.small;
+  PS.large2 = P2.large;
+  PS.seq_stride_small2 = P2.seq_stride_small;
+  PS.seq_stride_large2 = P2.seq_stride_large;
+  PS.K2 = K_q;
+  PS.stats2 = P2.stats;
+  rc = launch_rowstats(PS, dtype, variant, 0, stream);
+  if (rc != PSD_OK) return rc;
+  {
+    const dim3 grid(static_cast<unsigned>(B)), block(psd::kFinThreads);
+    TimedLaunch timed(stream, 1);
+    if (dtype == PSD_F32) psd::finalize_pyramid_kernel<float><<<grid, block, 0, stream>>>(P1, P2);
+    else psd::finalize_pyramid_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(P1, P2);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+  }
+  return check_launch();
 }
 
 }  // namespace

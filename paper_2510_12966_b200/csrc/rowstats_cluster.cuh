@@ -140,18 +140,19 @@ __device__ __forceinline__ uint4 lds128(const void* p) {
 // Every role of every CTA of a cluster walks the same list: rows q, q + n_clusters, ... of the [B*K]
 // grid, skipping positions at or beyond the sequence's n_valid. `n` counts the rows taken so far.
 struct RowWalk {
-  int next_r, stride, rows, K;
+  int next_r, stride, rows, rows1, K;
   const int32_t* n_valid;
   int n;     // ordinal of the current row among the rows this cluster takes
   int r;     // current row index (valid after advance() returned true)
   __device__ void init(const StageParams& P, int cluster_id, int n_clusters) {
-    next_r = cluster_id; stride = n_clusters; rows = P.B * P.K; K = P.K; n_valid = P.n_valid; n = -1; r = -1;
+    next_r = cluster_id; stride = n_clusters; rows = P.B * (P.K + P.K2); rows1 = P.B * P.K; K = P.K;
+    n_valid = P.n_valid; n = -1; r = -1;
   }
   __device__ bool advance() {
     while (next_r < rows) {
       const int cand = next_r;
       next_r += stride;
-      if (n_valid != nullptr) {
+      if (n_valid != nullptr && cand < rows1) {   // n_valid speaks of the first row set only
         const int b = cand / K, k = cand - b * K;
         if (k >= n_valid[b]) continue;
       }
@@ -563,8 +564,12 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       w.init(P, cluster_id, G.n_clusters);
       unsigned slot = 0, fills = 0;   // ring position; how often the ring has wrapped
       while (w.advance()) {
-        const T* rs = row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V) + slice_begin;
-        const T* rl = row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V) + slice_begin;
+        const int rows1 = P.B * K;
+        const bool second = w.r >= rows1;   // a row of the second set (stage 2 of the two-stage wrapper)
+        const T* rs = (second ? row_ptr<T>(P.small2, P.seq_stride_small2, w.r - rows1, P.K2, V)
+                              : row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V)) + slice_begin;
+        const T* rl = (second ? row_ptr<T>(P.large2, P.seq_stride_large2, w.r - rows1, P.K2, V)
+                              : row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V)) + slice_begin;
         for (int cidx = 0; cidx < C; ++cidx) {
           if (fills > 0) {
             wait_phase(&ctl->empty[slot], (fills - 1u) & 1u);
@@ -700,7 +705,8 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
           if (differ == 0.f) { st.div = 0.f; st.resid = 0.f; }   // bitwise identical rows: exactly zero
         }
         st.flags = flags;
-        P.stats[r] = st;
+        if (r < P.B * P.K) P.stats[r] = st;
+        else P.stats2[r - P.B * P.K] = st;
       }
     };
 
@@ -830,6 +836,10 @@ inline bool cluster_shape_ok(const StageParams& P, int dtype) {
   if (P.V < 2048 || (P.V % vec) != 0) return false;
   if ((P.seq_stride_small % vec) != 0 || (P.seq_stride_large % vec) != 0) return false;
   if (((reinterpret_cast<uintptr_t>(P.small) | reinterpret_cast<uintptr_t>(P.large)) & 15u) != 0) return false;
+  if (P.K2 > 0) {
+    if ((P.seq_stride_small2 % vec) != 0 || (P.seq_stride_large2 % vec) != 0) return false;
+    if (((reinterpret_cast<uintptr_t>(P.small2) | reinterpret_cast<uintptr_t>(P.large2)) & 15u) != 0) return false;
+  }
   return true;
 }
 
@@ -838,7 +848,7 @@ inline bool cluster_shape_ok(const StageParams& P, int dtype) {
 inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, ClusterGeom* g) {
   if (!cluster_shape_ok(P, dtype)) return false;
   const int es = dtype == 0 ? 4 : 2;
-  const long long rows = static_cast<long long>(P.B) * P.K;
+  const long long rows = static_cast<long long>(P.B) * (P.K + P.K2);
   int cs = 0, slice = 0, chunks = 0;
   if (forced_cs <= 0) {
     // tuning aid: PYRAMIDSD_CLUSTER_SIZE=<power of two> overrides the library's choice for every call
