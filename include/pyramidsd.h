@@ -172,6 +172,24 @@ int pyramidsd_verify_stage_noalloc(const void* logits_small, const void* logits_
                                    int32_t* out_accept_len, int32_t* out_next_token,
                                    int32_t* out_wait_timeout, void* cuda_stream);
 
+/* One verification stage whose LARGE-model logits are produced inside the call: z_large = hidden x W^T
+ * (the model's LM head), by a tensor-core GEMM whose epilogue does the softmax / divergence / residual
+ * arithmetic of Sec. 3.1-3.2, so the large model's logits are never written to memory. Not in the paper
+ * (it verifies logits the models have already produced); the rest of the stage is pyramidsd_verify_stage.
+ *   hidden        [B*K, d_model] bf16, row-major (the large model's final hidden states), device
+ *   w_t           [V, d_model]  bf16, row-major: the LM-head weight as checkpoints store it (out x in), device
+ *   logits_small  [B, K, V] bf16, device; tokens [B, K] int32
+ *   out_div, out_resid_mass  [B, K] float32 or NULL
+ * Requires B*K <= 256 and d_model a multiple of 64 (else PSD_ERR_UNSUPPORTED); hidden and w_t 16-byte aligned.
+ * Jensen-Shannon divergence, temperature 1. Runs the GEMM twice (the divergence needs the large model's
+ * normaliser first). Scratch (partial sums per row and 128-column tile) is library-owned, grown with
+ * cudaMalloc on first use. Asynchronous on `cuda_stream`; device-side timeouts via pyramidsd_last_status(). */
+int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const void* logits_small,
+                                  const int32_t* tokens, int B, int K, int d_model, int V, float threshold,
+                                  psd_mode mode, uint64_t philox_seed, uint64_t offset,
+                                  int32_t* out_accept_len, int32_t* out_next_token,
+                                  float* out_div, float* out_resid_mass, void* cuda_stream);
+
 /* The Philox uniforms the verification draws for rows 0..n_rows-1 with this seed and offset (see the
  * header comment for the counter layout): out_u[r] decides the strict coin flip of row r, out_u2[r]
  * drives its inverse CDF. Device pointers, float32 [n_rows]; either may be NULL. Lets a caller replay

@@ -22,7 +22,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, 
 
 EXPORTS = (
     "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_host",
-    "pyramidsd_verify_stage_noalloc",
+    "pyramidsd_verify_stage_noalloc", "pyramidsd_verify_fused_lmhead",
     "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
     "pyramidsd_kernel_timing_begin", "pyramidsd_kernel_timing_end",
     "pyramidsd_cluster_occupancy", "pyramidsd_version", "pyramidsd_status_string",
@@ -73,6 +73,8 @@ def load_library(path: Optional[str] = None):
     lib.pyramidsd_verify_stage.restype = i32
     lib.pyramidsd_verify_stage_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, f32, i32, u64, u64, vp, vp, vp, vp]
     lib.pyramidsd_verify_stage_noalloc.restype = i32
+    lib.pyramidsd_verify_fused_lmhead.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, u64, u64, vp, vp, vp, vp, vp]
+    lib.pyramidsd_verify_fused_lmhead.restype = i32
     lib.pyramidsd_verify_stage_ex.argtypes = [C.POINTER(StageArgs)]
     lib.pyramidsd_verify_stage_ex.restype = i32
     pyr = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, u64, u64, vp, vp, vp, vp]
@@ -200,6 +202,33 @@ def verify_stage(logits_small, logits_large, draft_tokens, threshold, mode=FUZZY
         int(philox_seed), int(offset), _dev_ptr(out_accept_len, torch.int32), _dev_ptr(out_next_token, torch.int32))
     _check(rc, "pyramidsd_verify_stage")
     return out_accept_len, out_next_token
+
+
+def verify_fused_lmhead(hidden, w_t, logits_small, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
+                        want_rows=True, stream=None, raise_on_error=True):
+    """``pyramidsd_verify_fused_lmhead``: hidden [B*K, d] bf16, w_t [V, d] bf16 (LM-head weight, out x in),
+    logits_small [B, K, V] bf16, tokens [B, K]. Returns a dict of device tensors (+ "status")."""
+    B, K, V = logits_small.shape
+    d = hidden.shape[1]
+    assert hidden.shape[0] == B * K and w_t.shape == (V, d)
+    dev = hidden.device
+    out = {"accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+           "next_token": torch.empty(B, dtype=torch.int32, device=dev)}
+    if want_rows:
+        out["div"] = torch.empty((B, K), dtype=torch.float32, device=dev)
+        out["resid_mass"] = torch.empty((B, K), dtype=torch.float32, device=dev)
+    s = torch.cuda.current_stream() if stream is None else stream
+    rc = load_library().pyramidsd_verify_fused_lmhead(
+        _dev_ptr(hidden, torch.bfloat16, "hidden"), _dev_ptr(w_t, torch.bfloat16, "w_t"),
+        _dev_ptr(logits_small, torch.bfloat16, "logits_small"), _dev_ptr(tokens, torch.int32, "tokens"),
+        B, K, d, V, float(threshold), int(mode), int(philox_seed), int(offset),
+        out["accept_len"].data_ptr(), out["next_token"].data_ptr(),
+        out["div"].data_ptr() if want_rows else None, out["resid_mass"].data_ptr() if want_rows else None,
+        C.c_void_p(s.cuda_stream))
+    out["status"] = rc
+    if raise_on_error:
+        _check(rc, "pyramidsd_verify_fused_lmhead")
+    return out
 
 
 NOALLOC_MAX_ROWS = 8192

@@ -13,6 +13,7 @@
 #include "finalize.cuh"
 #include "rowstats_baseline.cuh"
 #include "rowstats_cluster.cuh"
+#include "lmhead_fused.cuh"
 
 namespace {
 
@@ -48,6 +49,8 @@ struct DeviceState {
   size_t stage_bytes[4] = {0, 0, 0, 0};
   int32_t* out4 = nullptr;  // 4 x [B] results of the host entry point
   size_t out4_elems = 0;
+  void* lm_ws = nullptr;    // partial sums of the fused LM-head path
+  size_t lm_ws_bytes = 0;
 };
 DeviceState g_dev[kMaxDevices];
 
@@ -529,6 +532,112 @@ int pyramidsd_verify_stage_noalloc(const void* logits_small, const void* logits_
       cudaMemcpyAsync(out_wait_timeout, flag, sizeof(int), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
     return PSD_ERR_CUDA;
   return PSD_OK;
+}
+
+int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const void* logits_small,
+                                  const int32_t* tokens, int B, int K, int d_model, int V, float threshold,
+                                  psd_mode mode, uint64_t philox_seed, uint64_t offset, int32_t* out_accept_len,
+                                  int32_t* out_next_token, float* out_div, float* out_resid_mass, void* cuda_stream) {
+  if (!valid_mode(mode) || B < 0 || K < 0 || K > 32 || V < 1 || d_model < 1 || std::isnan(threshold)) return PSD_ERR_INVALID_ARG;
+  const long long M = static_cast<long long>(B) * K;
+  if (M > psd::kLmM || (d_model % psd::kLmK) != 0) return PSD_ERR_UNSUPPORTED;
+  if (B == 0) return PSD_OK;
+  if (!out_accept_len || !out_next_token) return PSD_ERR_INVALID_ARG;
+  if (K > 0 && (!hidden || !w_t || !logits_small || !tokens)) return PSD_ERR_INVALID_ARG;
+  if (((reinterpret_cast<uintptr_t>(hidden) | reinterpret_cast<uintptr_t>(w_t)) & 15u) != 0) return PSD_ERR_UNSUPPORTED;
+  const cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (K == 0) {
+    // nothing to verify: every sequence accepts its empty window
+    if (cudaMemsetAsync(out_accept_len, 0, static_cast<size_t>(B) * 4, stream) != cudaSuccess) return PSD_ERR_CUDA;
+    if (cudaMemsetAsync(out_next_token, 0xff, static_cast<size_t>(B) * 4, stream) != cudaSuccess) return PSD_ERR_CUDA;
+    return PSD_OK;
+  }
+  DeviceState* ds = nullptr;
+  int rc = current_device_state(&ds);
+  if (rc != PSD_OK) return rc;
+  const int n_tiles = (V + psd::kLmN - 1) / psd::kLmN;
+  const size_t per = static_cast<size_t>(M) * n_tiles;
+  const size_t bytes = align_up(per * sizeof(float2)) * 2 + align_up(per * sizeof(float4)) + align_up(static_cast<size_t>(M) * sizeof(float4));
+  {
+    std::lock_guard<std::mutex> lock(ds->mu);
+    rc = ensure_status(ds);
+    if (rc != PSD_OK) return rc;
+    rc = grow(&ds->lm_ws, &ds->lm_ws_bytes, bytes);
+    if (rc != PSD_OK) return rc;
+  }
+  // tensor maps: hidden [M, d] and W^T [V, d], bf16, K innermost, boxes of 64 x 256 / 64 x 128, 128-byte swizzle
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) fn = nullptr;
+    return reinterpret_cast<EncodeFn>(fn);
+  }();
+  if (encode == nullptr) return PSD_ERR_CUDA;
+  CUtensorMap map_a, map_b;
+  {
+    const cuuint64_t dims_a[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(M)};
+    const cuuint64_t dims_b[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(V)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(d_model) * 2};
+    const cuuint32_t box_a[2] = {psd::kLmK, psd::kLmM}, box_b[2] = {psd::kLmK, psd::kLmN}, estr[2] = {1, 1};
+    if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(hidden), dims_a, strides, box_a, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
+    if (encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w_t), dims_b, strides, box_b, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
+  }
+  char* ws = static_cast<char*>(ds->lm_ws);
+  psd::LmParams L{};
+  L.small = static_cast<const __nv_bfloat16*>(logits_small);
+  L.tokens = tokens;
+  L.M = static_cast<int>(M); L.d = d_model; L.V = V; L.n_tiles = n_tiles;
+  L.c = 1.4426950408889634f;
+  L.part_large = reinterpret_cast<float2*>(ws); ws += align_up(per * sizeof(float2));
+  L.part_small = reinterpret_cast<float2*>(ws); ws += align_up(per * sizeof(float2));
+  L.part_div = reinterpret_cast<float4*>(ws); ws += align_up(per * sizeof(float4));
+  L.row_lse = reinterpret_cast<float4*>(ws);
+  L.status = ds->status;
+  static bool attr_set[kMaxDevices] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_set[dev]) {
+    if (cudaFuncSetAttribute(psd::lmhead_sweep_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLmSmemBytes)) != cudaSuccess ||
+        cudaFuncSetAttribute(psd::lmhead_sweep_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLmSmemBytes)) != cudaSuccess) {
+      cudaGetLastError();
+      return PSD_ERR_CUDA;
+    }
+    attr_set[dev] = true;
+  }
+  int sms = psd::cluster_sm_count();
+  if (sms <= 0) sms = 1;
+  const unsigned grid = static_cast<unsigned>(n_tiles < sms ? n_tiles : sms);
+  {
+    TimedLaunch timed(stream, 0);
+    psd::lmhead_sweep_kernel<1><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
+    psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);
+    psd::lmhead_sweep_kernel<2><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
+  }
+  psd::LmFinalParams F{};
+  F.lm = L;
+  F.hidden = static_cast<const __nv_bfloat16*>(hidden);
+  F.w_t = static_cast<const __nv_bfloat16*>(w_t);
+  F.B = B; F.K = K;
+  F.threshold = threshold;
+  F.mode = mode;
+  F.seed = philox_seed; F.offset = offset;
+  F.out_accept_len = out_accept_len;
+  F.out_next_token = out_next_token;
+  F.out_div = out_div;
+  F.out_resid = out_resid_mass;
+  {
+    TimedLaunch timed(stream, 1);
+    psd::lmhead_final_kernel<<<static_cast<unsigned>(B), 256, 0, stream>>>(F);
+  }
+  g_launches.fetch_add(4, std::memory_order_relaxed);
+  return check_launch();
 }
 
 int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, float* out_u, float* out_u2) {

@@ -1,0 +1,91 @@
+"""GPU parity of the fused LM-head path: logits = hidden x W^T computed by the tensor-core kernel and
+consumed in its epilogue, against the oracle's double-precision GEMM followed by the ordinary stage."""
+import numpy as np
+import pytest
+import torch
+
+from parity_utils import host_bits
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def psd():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2510_12966_b200 import binding
+    binding.load_library()
+    torch.cuda.set_device(0)
+    return binding
+
+
+def make_case(B, K, d, V, seed, sigma_q=0.7, w_scale=0.02):
+    g = torch.Generator().manual_seed(seed)
+    h = torch.randn((B * K, d), generator=g).to(torch.bfloat16)
+    w_t = (torch.randn((V, d), generator=g) * w_scale).to(torch.bfloat16)     # LM-head weight, out x in
+    z = h.float() @ w_t.float().T
+    z_q = (z + torch.randn((B * K, V), generator=g) * sigma_q).to(torch.bfloat16).reshape(B, K, V).contiguous()
+    tok = torch.multinomial(torch.softmax(z_q.float().reshape(B * K, V), -1), 1, generator=g).reshape(B, K).to(torch.int32)
+    return h.contiguous(), w_t.contiguous(), z_q, tok.contiguous()
+
+
+def run_both(psd, oracle, h, w_t, z_q, tok, tau, mode, seed=3, offset=5):
+    dev = torch.device("cuda:0")
+    out = psd.verify_fused_lmhead(h.to(dev), w_t.to(dev), z_q.to(dev), tok.to(dev), tau, mode, seed, offset)
+    torch.cuda.synchronize()
+    assert psd.last_status() == 0
+    gpu = {k: v.cpu().numpy() for k, v in out.items() if isinstance(v, torch.Tensor)}
+    B, K, V = z_q.shape
+    z = oracle.lmhead_logits(host_bits(h), host_bits(w_t.T.contiguous()), n_threads=16).reshape(B, K, V)
+    orc = oracle.verify_stage_mixed(host_bits(z_q), z, tok.numpy(), np.float32(tau), mode, seed, offset, n_threads=16)
+    return gpu, orc
+
+
+def check(gpu, orc, tau, mode, max_token_ties=1):
+    assert np.abs(gpu["div"] - orc["div"]).max() < 2e-3, np.abs(gpu["div"] - orc["div"]).max()
+    assert np.abs(gpu["resid_mass"] - orc["resid_mass"]).max() < 2e-3
+    ties = 0
+    for b in range(len(orc["accept_len"])):
+        Lg, Lo = int(gpu["accept_len"][b]), int(orc["accept_len"][b])
+        if Lg != Lo:
+            k = min(Lg, Lo)
+            assert mode in (0, 2) and abs(orc["div"][b, k] - tau) < 1e-4, (b, Lg, Lo, orc["div"][b, k], tau)
+            ties += 1
+            continue
+        if int(gpu["next_token"][b]) != int(orc["next_token"][b]):
+            ties += 1       # an inverse-CDF pick on a prefix-sum boundary; must stay rare
+            assert gpu["next_token"][b] >= 0 and orc["next_token"][b] >= 0
+    assert ties <= max_token_ties, ties
+    return ties
+
+
+@pytest.mark.parametrize("B,K,d,V", [(2, 4, 128, 1000), (3, 5, 256, 4099), (32, 8, 512, 2048)])
+def test_fused_lmhead_small_shapes(psd, oracle, B, K, d, V):
+    """Ragged last tile (V not a multiple of 128), fewer rows than the 256-row tile, several K steps."""
+    h, w_t, z_q, tok = make_case(B, K, d, V, seed=50 + V, w_scale=0.08)
+    for tau, mode in ((0.05, 0), (0.2, 0), (0.0, 1)):
+        gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, tau, mode)
+        check(gpu, orc, tau, mode)
+        assert 0 <= orc["accept_len"].sum() <= B * K
+
+
+def test_fused_lmhead_reduced_cfg5(psd, oracle):
+    """BASELINE config 5 recipe (B=32, K=8, d=4096, W ~ N(0, 0.02^2), qualifier noise 0.7) at V=4096."""
+    h, w_t, z_q, tok = make_case(32, 8, 4096, 4096, seed=5000)
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.2, 0)
+    check(gpu, orc, 0.2, 0, max_token_ties=2)
+    assert 0 < orc["accept_len"].sum() < 32 * 8
+
+
+def test_fused_lmhead_rejects_unsupported_shapes(psd):
+    dev = torch.device("cuda:0")
+    h = torch.zeros((264, 128), dtype=torch.bfloat16, device=dev)
+    w = torch.zeros((512, 128), dtype=torch.bfloat16, device=dev)
+    z = torch.zeros((33, 8, 512), dtype=torch.bfloat16, device=dev)
+    t = torch.zeros((33, 8), dtype=torch.int32, device=dev)
+    assert psd.verify_fused_lmhead(h, w, z, t, 0.1, raise_on_error=False)["status"] == psd.ERR_UNSUPPORTED   # 264 rows
+    h2 = torch.zeros((8, 96), dtype=torch.bfloat16, device=dev)
+    w2 = torch.zeros((512, 96), dtype=torch.bfloat16, device=dev)
+    z2 = torch.zeros((1, 8, 512), dtype=torch.bfloat16, device=dev)
+    t2 = torch.zeros((1, 8), dtype=torch.int32, device=dev)
+    assert psd.verify_fused_lmhead(h2, w2, z2, t2, 0.1, raise_on_error=False)["status"] == psd.ERR_UNSUPPORTED  # d % 64
