@@ -249,6 +249,102 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_fused(args):
+    """Config 5: the fused LM-head + target verify. A step = one pyramidsd_verify_fused_lmhead call (two GEMM
+    sweeps with the statistics in their epilogues, a row reduction, the finalisation). The bound is the
+    tensor pipe: achieved = 2 sweeps x 2*M*d*V flops / device time of the sweep kernels."""
+    from paper_2510_12966_b200 import binding, workloads
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1 and int(os.environ.get("RANK", "0")) != 0:
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the verification path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    binding.load_library()
+    binding.set_stream()
+    w = workloads.CONFIGS[5]
+    M = w.B * w.K_d
+    h, w_t, z_q, tok = workloads.make_fused_inputs(w.B, w.K_d, w.V, w.d_model, seed=5000, sigma_q=w.sigma_q, device=dev)
+    hs = [h, h.clone()]          # the weight (1.05 GB) stays resident like a model's; activations alternate
+    zs = [z_q, z_q.clone()]
+
+    def step(i):
+        return binding.verify_fused_lmhead(hs[i % 2], w_t, zs[i % 2], tok, w.tau_t, binding.FUZZY, 0, i, want_rows=False)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches0 = binding.launch_count()
+    binding.kernel_timing_begin()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        out = step(args.warmup + i)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms_total = ev0.elapsed_time(ev1)
+    ms_sweeps, n_sw, ms_fin, n_fin = binding.kernel_timing_end()
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop()
+    if binding.last_status() != 0:
+        raise SystemExit("bench.py: library status != 0")
+    peaks, peak_kind = load_peaks()
+    flops = 2 * 2.0 * M * w.d_model * w.V
+    achieved = flops * n_sw / (ms_sweeps * 1e-3) / 1e12 if ms_sweeps > 0 else 0.0
+    # end to end: activations and qualifier logits come from pinned host memory every step, results go back
+    e2e = None
+    if not args.no_e2e:
+        hh, zh, th = h.cpu().pin_memory(), z_q.cpu().pin_memory(), tok.cpu().pin_memory()
+        res = torch.empty((2, w.B), dtype=torch.int32).pin_memory()
+        n = max(2, min(args.steps, 8))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for it in range(n + 2):
+            if it == 2:
+                torch.cuda.synchronize()
+                e0.record()
+            hs[0].copy_(hh, non_blocking=True); zs[0].copy_(zh, non_blocking=True); tok.copy_(th, non_blocking=True)
+            o = binding.verify_fused_lmhead(hs[0], w_t, zs[0], tok, w.tau_t, binding.FUZZY, 0, it, want_rows=False)
+            res[0].copy_(o["accept_len"], non_blocking=True); res[1].copy_(o["next_token"], non_blocking=True)
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        e2e = {"value": M * n / (e0.elapsed_time(e1) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": hh.numel() * 2 + zh.numel() * 2 + th.numel() * 4, "d2h_bytes_per_step": 8 * w.B,
+               "ms_per_step": e0.elapsed_time(e1) / n, "steps": n}
+    line = {
+        "metric": METRIC, "value": M * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 x bf16 -> f32 (GEMM), f32 (epilogue)", "data": "synthetic",
+        "config": {"workload": f"{w.name}: B={w.B}, K={w.K_d} (M={M}), d={w.d_model}, V={w.V}, LM-head weight bf16 [V, d], "
+                               f"qualifier logits bf16, tau_t={w.tau_t}, fuzzy mode, Philox seed 0",
+                   "l2_policy": "the weight (1.05 GB) is larger than L2 and is streamed twice per step"},
+        "roofline": {"bound": "tensor", "kernel": "lmhead_sweep (two tcgen05 GEMM sweeps + row reduction)",
+                     "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                     "peak_kind": f"of {peak_kind} (burst)", "traffic": None, "launches": n_sw,
+                     "avg_launch_ms": ms_sweeps / max(n_sw, 1), "finalize_ms_per_launch": ms_fin / max(n_fin, 1),
+                     "weight_gb_per_s": 2 * w.V * w.d_model * 2 * n_sw / (ms_sweeps * 1e-3) / 1e9 if ms_sweeps > 0 else 0.0},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        cores = os.cpu_count() or 1
+        nb = 2                     # sequences in the sample (16 rows, full vocabulary)
+        t0 = time.perf_counter()
+        zl = oracle.lmhead_logits(workloads.to_host_bits(h[:nb * w.K_d]), workloads.to_host_bits(w_t.T.contiguous()),
+                                  n_threads=cores).reshape(nb, w.K_d, w.V)
+        oracle.verify_stage_mixed(workloads.to_host_bits(z_q[:nb]), zl, tok[:nb].cpu().numpy(), np.float32(w.tau_t),
+                                  oracle.FUZZY, 0, 0, n_threads=cores)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": nb * w.K_d / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"first {nb} sequences ({nb * w.K_d} rows, full vocabulary: double-precision GEMM + stage), {dt:.1f} s wall"}
+    print(json.dumps(line))
+
+
 def read_profile_traffic(w):
     """DRAM bytes per full-size rowstats launch from the committed ncu summary, if present."""
     path = os.path.join(ROOT, "profiles", "rowstats_traffic.json")
@@ -326,7 +422,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences per step of the CPU-oracle reference arm")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (small profiling cases)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -336,6 +432,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "cfg5":
+        run_fused(args)
     else:
         run_ours(args)
 

@@ -105,17 +105,18 @@ def make_pyramid_inputs(B, K_d, K_q, V, dtype="bf16", seed=0, boost=(8.0, 8.0), 
 
 
 def make_fused_inputs(B, K, V, d_model, seed=0, sigma_q=0.7, device="cpu"):
-    """Fused-LM-head inputs: hidden [B*K, d] bf16 ~ N(0,1), W [d, V] bf16 ~ N(0, 0.02^2), qualifier logits
-    [B, K, V] bf16 = hidden x W + N(0, sigma_q^2) (a library matmul builds this input, nothing more), and
-    window tokens drawn from the qualifier's softmax."""
+    """Fused-LM-head inputs: hidden [B*K, d] bf16 ~ N(0,1); the LM-head weight ~ N(0, 0.02^2) bf16 in the
+    layout checkpoints keep it in, w_t [V, d] (out x in; the [d, V] matrix of the config is its transpose);
+    qualifier logits [B, K, V] bf16 = hidden x W + N(0, sigma_q^2) (a library matmul builds this input,
+    nothing more); window tokens drawn from the qualifier's softmax."""
     g = _gen(seed, device)
     h = torch.randn((B * K, d_model), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
-    W = (torch.randn((d_model, V), generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
-    z = h.float() @ W.float()
+    w_t = (torch.randn((V, d_model), generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    z = h.float() @ w_t.float().T
     z_q = (z + torch.randn((B * K, V), generator=g, device=device, dtype=torch.float32) * sigma_q)
     z_q = z_q.to(torch.bfloat16).reshape(B, K, V).contiguous()
     tok = _sample_tokens(z_q, g)
-    return h.contiguous(), W.contiguous(), z_q, tok.contiguous()
+    return h.contiguous(), w_t.contiguous(), z_q, tok.contiguous()
 
 
 def workload_inputs(cfg: int, round_idx: int = 0, device="cpu", B: Optional[int] = None,

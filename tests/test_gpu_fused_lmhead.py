@@ -72,9 +72,44 @@ def test_fused_lmhead_small_shapes(psd, oracle, B, K, d, V):
 def test_fused_lmhead_reduced_cfg5(psd, oracle):
     """BASELINE config 5 recipe (B=32, K=8, d=4096, W ~ N(0, 0.02^2), qualifier noise 0.7) at V=4096."""
     h, w_t, z_q, tok = make_case(32, 8, 4096, 4096, seed=5000)
-    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.2, 0)
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.2, 0)       # the config's threshold: accepts everything here
     check(gpu, orc, 0.2, 0, max_token_ties=2)
+    tau = float(np.float32(np.median(orc["div"])))                    # a threshold that splits the rows
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, tau, 0)
+    check(gpu, orc, tau, 0, max_token_ties=3)
     assert 0 < orc["accept_len"].sum() < 32 * 8
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.0, 1)        # strict mode: coin flips on token probabilities
+    check(gpu, orc, 0.0, 1, max_token_ties=3)
+
+
+def test_fused_lmhead_full_size_cfg5_sampled(psd, oracle):
+    """BASELINE config 5 at full size (M=256, d=4096, V=128256) in the launch configuration bench.py times;
+    the oracle recomputes two sampled sequences (its double-precision GEMM is far too slow for all 256 rows)."""
+    from paper_2510_12966_b200 import workloads
+    dev = torch.device("cuda:0")
+    w = workloads.CONFIGS[5]
+    h, w_t, z_q, tok = workloads.make_fused_inputs(w.B, w.K_d, w.V, w.d_model, seed=5000, sigma_q=w.sigma_q, device=dev)
+    out = psd.verify_fused_lmhead(h, w_t, z_q, tok, w.tau_t, psd.FUZZY, 0, 0)
+    torch.cuda.synchronize()
+    assert psd.last_status() == 0
+    div = out["div"].cpu().numpy()
+    al, nt = out["accept_len"].cpu().numpy(), out["next_token"].cpu().numpy()
+    assert np.all(np.isfinite(div)) and np.all((div >= 0) & (div <= 0.6932))
+    assert np.all((0 <= al) & (al <= w.K_d)) and np.all((nt >= 0) == (al < w.K_d)) and np.all(nt < w.V)
+    w_host = host_bits(w_t.T.contiguous())
+    for b in (0, 17):
+        rows = slice(b * w.K_d, (b + 1) * w.K_d)
+        z = oracle.lmhead_logits(host_bits(h[rows]), w_host, n_threads=16).reshape(1, w.K_d, w.V)
+        # the Philox block of a row is indexed by its position in the full batch: shift the offset-free
+        # counter by asking the oracle for sequence b through a batch of one with the same row indices
+        orc = oracle.verify_stage_mixed(host_bits(z_q[b:b + 1]), z, tok[b:b + 1].cpu().numpy(), np.float32(w.tau_t),
+                                        oracle.FUZZY, 0, 0, n_threads=16)
+        assert np.abs(div[b] - orc["div"][0]).max() < 2e-3
+        assert np.abs(out["resid_mass"].cpu().numpy()[b] - orc["resid_mass"][0]).max() < 2e-3
+        near = np.abs(orc["div"][0] - w.tau_t).min() < 1e-4
+        assert near or al[b] == orc["accept_len"][0]
+        if b == 0 and al[b] == orc["accept_len"][0] and al[b] < w.K_d:
+            assert nt[b] == orc["next_token"][0]     # sequence 0 has batch row indices 0..K-1: same Philox blocks
 
 
 def test_fused_lmhead_rejects_unsupported_shapes(psd):
