@@ -190,6 +190,17 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
                                   int32_t* out_accept_len, int32_t* out_next_token,
                                   float* out_div, float* out_resid_mass, void* cuda_stream);
 
+/* Analytic throughput model of Sec. 3.3 (host arithmetic, no GPU): tokens per second of standard or
+ * fuzzy speculative decoding with speculative length ell and acceptance rate beta between a small model
+ * of speed v_small and a large one of speed v_large (tokens/s each),
+ *     V = beta * (ell + 1) / (ell / v_small + 1 / v_large),
+ * and of the pyramid: the draft/qualifier pair first (beta_qd, ell_d, v_draft, v_qual), whose result takes
+ * the place of the small model's speed against the target (beta_tq, ell_q, v_target).
+ * Return NaN on non-positive speeds or lengths, or acceptance rates outside [0, 1]. */
+double pyramidsd_model_sd_throughput(double beta, double ell, double v_small, double v_large);
+double pyramidsd_model_psd_throughput(double beta_qd, double ell_d, double v_draft, double v_qual,
+                                      double beta_tq, double ell_q, double v_target);
+
 /* The Philox uniforms the verification draws for rows 0..n_rows-1 with this seed and offset (see the
  * header comment for the counter layout): out_u[r] decides the strict coin flip of row r, out_u2[r]
  * drives its inverse CDF. Device pointers, float32 [n_rows]; either may be NULL. Lets a caller replay

@@ -23,6 +23,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, 
 EXPORTS = (
     "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_host",
     "pyramidsd_verify_stage_noalloc", "pyramidsd_verify_fused_lmhead",
+    "pyramidsd_model_sd_throughput", "pyramidsd_model_psd_throughput",
     "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
     "pyramidsd_kernel_timing_begin", "pyramidsd_kernel_timing_end",
     "pyramidsd_cluster_occupancy", "pyramidsd_version", "pyramidsd_status_string",
@@ -75,6 +76,10 @@ def load_library(path: Optional[str] = None):
     lib.pyramidsd_verify_stage_noalloc.restype = i32
     lib.pyramidsd_verify_fused_lmhead.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, u64, u64, vp, vp, vp, vp, vp]
     lib.pyramidsd_verify_fused_lmhead.restype = i32
+    lib.pyramidsd_model_sd_throughput.argtypes = [C.c_double] * 4
+    lib.pyramidsd_model_sd_throughput.restype = C.c_double
+    lib.pyramidsd_model_psd_throughput.argtypes = [C.c_double] * 7
+    lib.pyramidsd_model_psd_throughput.restype = C.c_double
     lib.pyramidsd_verify_stage_ex.argtypes = [C.POINTER(StageArgs)]
     lib.pyramidsd_verify_stage_ex.restype = i32
     pyr = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, u64, u64, vp, vp, vp, vp]
@@ -229,6 +234,16 @@ def verify_fused_lmhead(hidden, w_t, logits_small, tokens, threshold, mode=FUZZY
     if raise_on_error:
         _check(rc, "pyramidsd_verify_fused_lmhead")
     return out
+
+
+def model_sd_throughput(beta, ell, v_small, v_large) -> float:
+    """Sec. 3.3: tokens/s of (fuzzy) speculative decoding for one model pair."""
+    return load_library().pyramidsd_model_sd_throughput(beta, ell, v_small, v_large)
+
+
+def model_psd_throughput(beta_qd, ell_d, v_draft, v_qual, beta_tq, ell_q, v_target) -> float:
+    """Sec. 3.3: tokens/s of the three-model pyramid."""
+    return load_library().pyramidsd_model_psd_throughput(beta_qd, ell_d, v_draft, v_qual, beta_tq, ell_q, v_target)
 
 
 NOALLOC_MAX_ROWS = 8192

@@ -640,6 +640,18 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
   return check_launch();
 }
 
+double pyramidsd_model_sd_throughput(double beta, double ell, double v_small, double v_large) {
+  if (!(beta >= 0.0 && beta <= 1.0) || !(ell > 0.0) || !(v_small > 0.0) || !(v_large > 0.0)) return std::nan("");
+  return beta * (ell + 1.0) / (ell / v_small + 1.0 / v_large);
+}
+
+double pyramidsd_model_psd_throughput(double beta_qd, double ell_d, double v_draft, double v_qual, double beta_tq,
+                                      double ell_q, double v_target) {
+  const double v_fsd = pyramidsd_model_sd_throughput(beta_qd, ell_d, v_draft, v_qual);
+  if (!(v_fsd > 0.0)) return std::nan("");
+  return pyramidsd_model_sd_throughput(beta_tq, ell_q, v_fsd, v_target);
+}
+
 int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, float* out_u, float* out_u2) {
   if (n_rows < 0) return PSD_ERR_INVALID_ARG;
   if (n_rows == 0 || (!out_u && !out_u2)) return PSD_OK;

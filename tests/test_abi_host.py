@@ -92,3 +92,23 @@ def test_product_path_does_not_touch_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower() or f == "workloads.py", f
+
+
+def test_analytic_throughput_model(lib):
+    """Sec. 3.3 formulas against values worked out by hand and their limiting cases."""
+    import math
+    from paper_2510_12966_b200 import binding
+    # beta = 1, ell = 4, draft 100 tok/s, target 20 tok/s: 5 / (0.04 + 0.05) = 55.555...
+    assert abs(binding.model_sd_throughput(1.0, 4, 100.0, 20.0) - 5 / 0.09) < 1e-12
+    # a draft as slow as the target and always accepted still gains the one free token: (ell+1)/(ell+1) * v
+    assert abs(binding.model_sd_throughput(1.0, 7, 30.0, 30.0) - 30.0) < 1e-12
+    # nothing accepted: no throughput; the rate is linear in beta
+    assert binding.model_sd_throughput(0.0, 4, 100.0, 20.0) == 0.0
+    assert abs(binding.model_sd_throughput(0.5, 4, 100.0, 20.0) - 0.5 * 5 / 0.09) < 1e-12
+    # pyramid = the pair formula applied twice: inner (0.8, 5, 200, 80) -> 0.8*6/(5/200+1/80) = 128
+    inner = binding.model_sd_throughput(0.8, 5, 200.0, 80.0)
+    assert abs(inner - 128.0) < 1e-9
+    outer = binding.model_psd_throughput(0.8, 5, 200.0, 80.0, 0.9, 10, 25.0)
+    assert abs(outer - 0.9 * 11 / (10 / 128.0 + 1 / 25.0)) < 1e-9
+    assert math.isnan(binding.model_sd_throughput(1.2, 4, 100.0, 20.0))
+    assert math.isnan(binding.model_psd_throughput(0.8, 0, 200.0, 80.0, 0.9, 10, 25.0))
