@@ -117,6 +117,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     binding.load_library()
     binding.set_stream()
+    binding.set_two_stage_policy(binding.TWO_STAGE_SEPARATE if args.two_stage == "separate" else binding.TWO_STAGE_FUSED)
     cfg, w = workload_from_name(args.workload)
     if args.batch > 0:
         import dataclasses
@@ -170,7 +171,7 @@ def run_ours(args):
     row_bytes = 2 * w.V * es
     rs_bytes = n_pos * row_bytes   # the statistics kernel streams each verified row pair once
     timed_cap = 4096               # launches the library's event timing holds; beyond it only the first ones are timed
-    launches_per_step = 2          # one statistics launch (both stages' rows) and one finalisation launch
+    launches_per_step = 2 if args.two_stage == "fused" else 4
     if launches_per_step * args.steps > timed_cap:
         steps_timed = timed_cap // launches_per_step
         rs_bytes = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(steps_timed)) * row_bytes
@@ -220,7 +221,7 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"{w.name}: B={w.B} per GPU, V={w.V}, {w.dtype} logits, K_draft={w.K_d}, "
-                                   f"K_qual={w.K_q}, tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0",
+                                   f"K_qual={w.K_q}, tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0, two-stage schedule {args.two_stage}",
                        "logits_dtype": w.dtype, "positions_per_step": n_pos / args.steps,
                        "l2_policy": "inputs larger than L2 (one round = %.0f MB), two rounds alternate" %
                                     ((2 * w.K_d + w.K_q) * w.B * w.V * es / 1e6),
@@ -425,6 +426,8 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences per step of the CPU-oracle reference arm")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (small profiling cases)")
+    ap.add_argument("--two-stage", choices=["fused", "separate"], default="fused",
+                    help="schedule of the two stages (same results): one statistics launch for both, or stage by stage")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -23,7 +23,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, 
 EXPORTS = (
     "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_host",
     "pyramidsd_verify_stage_noalloc", "pyramidsd_verify_fused_lmhead",
-    "pyramidsd_model_sd_throughput", "pyramidsd_model_psd_throughput",
+    "pyramidsd_model_sd_throughput", "pyramidsd_model_psd_throughput", "pyramidsd_set_two_stage_policy",
     "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
     "pyramidsd_kernel_timing_begin", "pyramidsd_kernel_timing_end",
     "pyramidsd_cluster_occupancy", "pyramidsd_version", "pyramidsd_status_string",
@@ -91,6 +91,8 @@ def load_library(path: Optional[str] = None):
     lib.pyramidsd_row_uniforms.restype = i32
     lib.pyramidsd_workspace_bytes.argtypes = [i32, i32, i32, i32]
     lib.pyramidsd_workspace_bytes.restype = C.c_size_t
+    lib.pyramidsd_set_two_stage_policy.argtypes = [i32]
+    lib.pyramidsd_set_two_stage_policy.restype = i32
     lib.pyramidsd_set_stream.argtypes = [vp]
     lib.pyramidsd_set_stream.restype = i32
     lib.pyramidsd_last_status.argtypes = []
@@ -148,6 +150,14 @@ def set_stream(stream: Optional[torch.cuda.Stream] = None) -> None:
     """Use ``stream`` (default: torch's current stream) for the entry points without a stream argument."""
     s = torch.cuda.current_stream() if stream is None else stream
     _check(load_library().pyramidsd_set_stream(C.c_void_p(s.cuda_stream)), "pyramidsd_set_stream")
+
+
+TWO_STAGE_FUSED, TWO_STAGE_SEPARATE = 0, 1
+
+
+def set_two_stage_policy(policy: int) -> None:
+    """``pyramidsd_set_two_stage_policy``: one statistics launch for both stages, or stage by stage."""
+    _check(load_library().pyramidsd_set_two_stage_policy(int(policy)), "pyramidsd_set_two_stage_policy")
 
 
 def last_status() -> int:

@@ -22,6 +22,7 @@ using psd::StageParams;
 
 std::atomic<uint64_t> g_launches{0};
 thread_local cudaStream_t t_stream = nullptr;
+thread_local int t_two_stage_policy = PSD_TWO_STAGE_FUSED;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
@@ -346,6 +347,12 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   rc = validate_stage(&s1);
   if (rc == PSD_OK) rc = validate_stage(&s2);
   if (rc != PSD_OK) return rc;
+  if (t_two_stage_policy == PSD_TWO_STAGE_SEPARATE) {
+    // stage by stage: stage 2's statistics run after stage 1 has fixed the windows and skip the rows beyond them
+    rc = run_stage(&s1, window, n_window, K_q);
+    if (rc != PSD_OK) return rc;
+    return run_stage(&s2, nullptr, nullptr, 0);
+  }
   {
     std::lock_guard<std::mutex> lock(ds->mu);
     rc = ensure_status(ds);
@@ -663,6 +670,12 @@ int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, fl
 size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype) {
   if (B < 0 || K < 0 || K > 32 || V < 1 || !valid_dtype(dtype)) return 0;
   return stage_workspace_bytes(B, K);
+}
+
+int pyramidsd_set_two_stage_policy(int policy) {
+  if (policy != PSD_TWO_STAGE_FUSED && policy != PSD_TWO_STAGE_SEPARATE) return PSD_ERR_INVALID_ARG;
+  t_two_stage_policy = policy;
+  return PSD_OK;
 }
 
 int pyramidsd_set_stream(void* cuda_stream) {

@@ -360,6 +360,23 @@ def test_pyramid_small_vocab_all_paths(psd, oracle, wl):
         assert len(lens) >= 2
 
 
+def test_two_stage_policies_give_the_same_results(psd, wl):
+    dev = torch.device("cuda:0")
+    zd, zq, zt, tok = [t.to(dev) for t in wl.make_pyramid_inputs(9, 8, 4, 8192, "bf16", seed=23, sigma_q=0.6, sigma_d=1.2)]
+    try:
+        psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+        a = psd.verify(zd, zq, zt, tok, 0.3, 0.15, 2, 3, 4)
+        torch.cuda.synchronize()
+        psd.set_two_stage_policy(psd.TWO_STAGE_SEPARATE)
+        b = psd.verify(zd, zq, zt, tok, 0.3, 0.15, 2, 3, 4)
+        torch.cuda.synchronize()
+    finally:
+        psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+    for k in a:
+        assert torch.equal(a[k], b[k]), k
+    assert 0 < int(a["accept_len_q"].sum()) < 9 * 8
+
+
 def test_host_entry_point_equals_device_entry_point(psd, wl):
     dev = torch.device("cuda:0")
     zd, zq, zt, tok = wl.make_pyramid_inputs(5, 8, 4, 9000, "bf16", seed=22)
