@@ -264,6 +264,9 @@ def run_fused(args):
     binding.load_library()
     binding.set_stream()
     w = workloads.CONFIGS[5]
+    if args.vocab > 0:
+        import dataclasses
+        w = dataclasses.replace(w, V=args.vocab, name=f"{w.name}[V={args.vocab}]")
     M = w.B * w.K_d
     h, w_t, z_q, tok = workloads.make_fused_inputs(w.B, w.K_d, w.V, w.d_model, seed=5000, sigma_q=w.sigma_q, device=dev)
     hs = [h, h.clone()]          # the weight (1.05 GB) stays resident like a model's; activations alternate
@@ -426,6 +429,7 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences per step of the CPU-oracle reference arm")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (small profiling cases)")
+    ap.add_argument("--vocab", type=int, default=0, help="override the vocabulary size V of cfg5 (small profiling cases)")
     ap.add_argument("--two-stage", choices=["fused", "separate"], default="fused",
                     help="schedule of the two stages (same results): one statistics launch for both, or stage by stage")
     ap.add_argument("--no-e2e", action="store_true")
