@@ -146,6 +146,67 @@ __device__ __forceinline__ void load_small32(const __nv_bfloat16* p, bool aligne
   }
 }
 
+// What one thread (= one row) leaves per 128-column tile.
+struct LmTilePartial {
+  float2 large, small;   // sweep 1: (max, sum) of both models
+  float4 div;            // sweep 2: (js bits, sum max(p,q), residual mass, mass of p)
+};
+
+// The epilogue of one 128-column tile for this thread's row: reads the accumulator from tensor memory 32
+// columns at a time (all 32 lanes execute the loads, whatever row_ok says) and the small model's logits
+// from global memory.
+template <int SWEEP>
+__device__ __forceinline__ void lm_epilogue_tile(unsigned tacc, int n0, bool row_ok, const __nv_bfloat16* small_row, float c,
+                                                 float off_l, float off_s, int V, LmTilePartial& out) {
+  OnlineLse ol, os;
+  ol.init(); os.init();
+  float js = 0.f, big = 0.f, resid = 0.f, pmass = 0.f;
+#pragma unroll 1
+  for (int cb = 0; cb < kLmN / 32; ++cb) {
+    float z[32], x[32];
+    tmem_ld32(tacc + static_cast<unsigned>(cb * 32), z);
+    const int col0 = n0 + cb * 32;
+    const int nv = min(32, V - col0);   // columns of this group inside the vocabulary (<= 0: none)
+    if (row_ok && nv > 0) {
+      const __nv_bfloat16* sp = small_row + col0;
+      load_small32(sp, (reinterpret_cast<uintptr_t>(sp) & 15u) == 0, nv, x);
+      if (SWEEP == 1) {
+        ol.add<32>(z, c, nv);
+        os.add<32>(x, c, nv);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (i < nv) {
+            const float a = fmaxf(fmaf(z[i], c, -off_l), -125.f), b = fmaxf(fmaf(x[i], c, -off_s), -125.f);   // log2 p, log2 q
+            const float E = ex2_approx(fmaxf(a, b));
+            const float dd = a - b;
+            const float u = ex2_approx(-fabsf(dd));
+            const float2 ps = psi_poly(make_float2(u, u));
+            js = fmaf(E, fmaf(u, -fabsf(dd), ps.x), js);
+            big += E;
+            const float lo = E * u;                       // min(p, q)
+            resid += (dd > 0.f) ? E - lo : 0.f;           // max(0, p - q)
+            pmass += (dd >= 0.f) ? E : lo;                // p
+          }
+        }
+      }
+    }
+  }
+  out.large = make_float2(ol.m, ol.s);
+  out.small = make_float2(os.m, os.s);
+  out.div = make_float4(js, big, resid, pmass);
+}
+
+template <int SWEEP>
+__device__ __forceinline__ void lm_store_partial(const LmParams& P, size_t idx, const LmTilePartial& part) {
+  if (SWEEP == 1) {
+    P.part_large[idx] = part.large;
+    P.part_small[idx] = part.small;
+  } else {
+    P.part_div[idx] = part.div;
+  }
+}
+
 template <int SWEEP>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const LmParams P) {
@@ -237,52 +298,12 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const unsigned tacc = tmem_base + static_cast<unsigned>(buf) * 256u + static_cast<unsigned>(half) * 128u +
                             (static_cast<unsigned>(quarter * 32) << 16);
       const int n0 = tile * kLmN;
-      OnlineLse ol, os;
-      ol.init(); os.init();
-      float js = 0.f, big = 0.f, resid = 0.f, pmass = 0.f;
-#pragma unroll 1
-      for (int cb = 0; cb < kLmN / 32; ++cb) {
-        float z[32], x[32];
-        tmem_ld32(tacc + static_cast<unsigned>(cb * 32), z);
-        const int col0 = n0 + cb * 32;
-        const int nv = min(32, P.V - col0);   // columns of this group inside the vocabulary (<= 0: none)
-        if (row_ok && nv > 0) {
-          const __nv_bfloat16* sp = small_row + col0;
-          load_small32(sp, (reinterpret_cast<uintptr_t>(sp) & 15u) == 0, nv, x);
-          if (SWEEP == 1) {
-            ol.add<32>(z, c, nv);
-            os.add<32>(x, c, nv);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              if (i < nv) {
-                const float a = fmaxf(fmaf(z[i], c, -off_l), -125.f), b = fmaxf(fmaf(x[i], c, -off_s), -125.f);   // log2 p, log2 q
-                const float E = ex2_approx(fmaxf(a, b));
-                const float dd = a - b;
-                const float u = ex2_approx(-fabsf(dd));
-                const float2 ps = psi_poly(make_float2(u, u));
-                js = fmaf(E, fmaf(u, -fabsf(dd), ps.x), js);
-                big += E;
-                const float lo = E * u;                       // min(p, q)
-                resid += (dd > 0.f) ? E - lo : 0.f;           // max(0, p - q)
-                pmass += (dd >= 0.f) ? E : lo;                // p
-              }
-            }
-          }
-        }
-      }
+      LmTilePartial part;
+      lm_epilogue_tile<SWEEP>(tacc, n0, row_ok, small_row, c, off_l, off_s, P.V, part);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);   // this warp has read its part of the accumulator
-      if (row_ok) {
-        const size_t idx = static_cast<size_t>(row) * P.n_tiles + tile;
-        if (SWEEP == 1) {
-          P.part_large[idx] = make_float2(ol.m, ol.s);
-          P.part_small[idx] = make_float2(os.m, os.s);
-        } else {
-          P.part_div[idx] = make_float4(js, big, resid, pmass);
-        }
-      }
+      if (row_ok) lm_store_partial<SWEEP>(P, static_cast<size_t>(row) * P.n_tiles + tile, part);
     }
   }
   tc_fence_before();
@@ -290,6 +311,163 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---- two-SM variant -------------------------------------------------------------------------------------
+// A pair of CTAs (cluster of 2) shares one 256 x 256 tile: tcgen05.mma.cta_group::2 with M = 256 takes rows
+// 0..127 of A from the even CTA's shared memory and rows 128..255 from the odd one's, and the two halves of
+// the 256 B rows likewise; each CTA keeps its 128 rows of the fp32 accumulator in its own tensor memory
+// (256 columns, two buffers). Per K step a CTA stages 16 KB of A and 16 KB of B (six stages), so the hidden
+// matrix crosses L2 -> SM once per 256 columns instead of once per 128, and the ring holds 1.5x the K steps.
+// The even CTA issues the MMAs; both CTAs' TMA loads count their bytes on the even CTA's "full" barrier,
+// tcgen05.commit (multicast to both CTAs) frees the stages and publishes the accumulators, and the odd CTA's
+// epilogue warps arrive remotely on the even CTA's "accumulator drained" barrier.
+constexpr int kLm2N = 256;
+constexpr int kLm2Stages = 6;
+constexpr int kLm2HalfBytes = 128 * kLmK * 2;              // 16 KB: 128 rows x 64 bf16
+constexpr int kLm2StageBytes = 2 * kLm2HalfBytes;          // A half + B half
+constexpr size_t kLm2SmemBytes = static_cast<size_t>(kLm2Stages) * kLm2StageBytes + 1024 + 256;
+
+struct Lm2Barriers {
+  unsigned long long full[kLm2Stages], empty[kLm2Stages], tmem_full[2], tmem_empty[2];
+  unsigned tmem_base;
+};
+
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
+  // the barrier address with the peer bit cleared names the even CTA's barrier at the same offset
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar) & 0xFEFFFFFFu), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(unsigned* smem_result, unsigned ncols) {   // same warp index in both CTAs
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(unsigned taddr, unsigned ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(unsigned long long* bar) {   // arrives on this barrier in both CTAs
+  const unsigned short mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(unsigned tmem_d, unsigned long long desc_a, unsigned long long desc_b, unsigned idesc,
+                                                 unsigned accumulate) {
+  const unsigned z = 0;
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+               " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n}"
+               ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(z) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote_release(unsigned cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+template <int SWEEP>
+__global__ void __launch_bounds__(kLmThreads, 1)
+lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const LmParams P) {
+  extern __shared__ unsigned char lm_smem_raw[];
+  unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(lm_smem_raw) + 1023) & ~uintptr_t(1023));
+  Lm2Barriers* bars = reinterpret_cast<Lm2Barriers*>(tiles + static_cast<size_t>(kLm2Stages) * kLm2StageBytes);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const unsigned rank = cluster_rank();          // 0: issues the MMAs; 1: its peer
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int k_steps = P.d / kLmK;
+  const int n_tiles2 = (P.n_tiles + 1) / 2;      // 256-column tiles
+
+  if (tid == 0) {
+    for (int s = 0; s < kLm2Stages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&bars->tmem_full[b], 1); mbar_init(&bars->tmem_empty[b], 2 * kLmEpiWarps); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc_pair(&bars->tmem_base, 512);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();        // both CTAs' barriers and allocations exist before either signals the other
+  tc_fence_after();
+  const unsigned tmem_base = bars->tmem_base;
+
+  bool dead = false;
+  auto wait_phase = [&](unsigned long long* bar, unsigned parity) {
+    if (mbar_test(bar, parity)) return;
+    unsigned spins = 0;
+    while (!dead && !mbar_try(bar, parity))
+      if (++spins > kLmSpinLimit) { dead = true; atomicExch(P.status, 1); }
+  };
+
+  if (warp == 0) {
+    // ================================ TMA producer (both CTAs) ================================
+    if (lane == 0) {
+      unsigned stage = 0, fills = 0;
+      for (int tile = pair; tile < n_tiles2; tile += n_pairs) {
+        for (int ks = 0; ks < k_steps; ++ks) {
+          if (fills > 0) wait_phase(&bars->empty[stage], (fills - 1u) & 1u);
+          unsigned char* sa = tiles + static_cast<size_t>(stage) * kLm2StageBytes;
+          // the even CTA's barrier counts the bytes of both CTAs
+          if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2u * kLm2StageBytes);
+          tma_load_2d_pair(sa, &map_a, ks * kLmK, static_cast<int>(rank) * 128, &bars->full[stage]);
+          tma_load_2d_pair(sa + kLm2HalfBytes, &map_b, ks * kLmK, tile * kLm2N + static_cast<int>(rank) * 128, &bars->full[stage]);
+          if (++stage == kLm2Stages) { stage = 0; ++fills; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer (even CTA only) ================================
+    if (lane == 0 && rank == 0) {
+      constexpr unsigned idesc = umma_idesc_bf16(256, kLm2N);
+      unsigned stage = 0, par = 0;
+      int it = 0;
+      for (int tile = pair; tile < n_tiles2; tile += n_pairs, ++it) {
+        const int buf = it & 1;
+        if (it >= 2) wait_phase(&bars->tmem_empty[buf], ((it >> 1) - 1) & 1u);   // both CTAs' epilogues have drained this buffer
+        tc_fence_after();
+        const unsigned acc = tmem_base + static_cast<unsigned>(buf) * 256u;
+        for (int ks = 0; ks < k_steps; ++ks) {
+          wait_phase(&bars->full[stage], par);
+          tc_fence_after();
+          const unsigned sa = smem_u32(tiles + static_cast<size_t>(stage) * kLm2StageBytes);
+          const unsigned long long da = umma_desc_k128(sa), db = umma_desc_k128(sa + kLm2HalfBytes);
+#pragma unroll
+          for (int kk = 0; kk < kLmK / 16; ++kk)
+            tc_mma_bf16_pair(acc, da + 2ull * kk, db + 2ull * kk, idesc, (ks | kk) != 0 ? 1u : 0u);
+          tc_commit_pair(&bars->empty[stage]);   // frees the stage in both CTAs once these MMAs have read it
+          if (++stage == kLm2Stages) { stage = 0; par ^= 1u; }
+        }
+        tc_commit_pair(&bars->tmem_full[buf]);   // the accumulators of this tile are complete, in both CTAs
+      }
+    }
+  } else {
+    // ================================ epilogue (both CTAs) ================================
+    const int quarter = warp & 3, half = (warp - 2) >> 2;          // TMEM lanes 32*quarter.., columns 128*half..
+    const int row = static_cast<int>(rank) * 128 + quarter * 32 + lane;
+    const bool row_ok = row < P.M;
+    const float c = P.c;
+    const __nv_bfloat16* small_row = P.small + static_cast<size_t>(row_ok ? row : 0) * P.V;
+    float4 lse = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (SWEEP == 2 && row_ok) lse = P.row_lse[row];
+    const float off_s = lse.x + lse.y, off_l = lse.z + lse.w;
+    const unsigned drained = map_to_rank(&bars->tmem_empty[0], 0);   // the even CTA's barriers
+    int it = 0;
+    for (int tile = pair; tile < n_tiles2; tile += n_pairs, ++it) {
+      const int buf = it & 1;
+      wait_phase(&bars->tmem_full[buf], (it >> 1) & 1u);
+      tc_fence_after();
+      const unsigned tacc = tmem_base + static_cast<unsigned>(buf) * 256u + static_cast<unsigned>(half) * 128u +
+                            (static_cast<unsigned>(quarter * 32) << 16);
+      const int tile128 = tile * 2 + half;
+      LmTilePartial part;
+      lm_epilogue_tile<SWEEP>(tacc, tile128 * kLmN, row_ok, small_row, c, off_l, off_s, P.V, part);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote_release(drained + static_cast<unsigned>(buf) * 8u);
+      if (row_ok && tile128 < P.n_tiles) lm_store_partial<SWEEP>(P, static_cast<size_t>(row) * P.n_tiles + tile128, part);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();        // nobody frees tensor memory or leaves while the peer can still touch it
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
   }
 }
 

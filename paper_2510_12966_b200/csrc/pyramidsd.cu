@@ -620,8 +620,50 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
   }
   int sms = psd::cluster_sm_count();
   if (sms <= 0) sms = 1;
-  const unsigned grid = static_cast<unsigned>(n_tiles < sms ? n_tiles : sms);
-  {
+  // the two-SM (cta_group::2) sweeps are the default; PYRAMIDSD_LMHEAD_PAIR=0 selects the one-SM variant
+  static const bool use_pair = [] { const char* e = std::getenv("PYRAMIDSD_LMHEAD_PAIR"); return !(e && std::atoi(e) == 0); }();
+  if (use_pair) {
+    static bool pair_attr[kMaxDevices] = {};
+    if (!pair_attr[dev]) {
+      if (cudaFuncSetAttribute(psd::lmhead_sweep2sm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLm2SmemBytes)) != cudaSuccess ||
+          cudaFuncSetAttribute(psd::lmhead_sweep2sm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLm2SmemBytes)) != cudaSuccess) {
+        cudaGetLastError();
+        return PSD_ERR_CUDA;
+      }
+      pair_attr[dev] = true;
+    }
+    // the pair's A / B boxes are 64 x 128
+    CUtensorMap map_a2, map_b2;
+    {
+      const cuuint64_t dims_a[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(M)};
+      const cuuint64_t dims_b[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(V)};
+      const cuuint64_t strides[1] = {static_cast<cuuint64_t>(d_model) * 2};
+      const cuuint32_t box[2] = {psd::kLmK, 128}, estr[2] = {1, 1};
+      if (encode(&map_a2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(hidden), dims_a, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
+      if (encode(&map_b2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w_t), dims_b, strides, box, estr,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
+    }
+    const int n_tiles2 = (n_tiles + 1) / 2;
+    const int pairs = n_tiles2 < sms / 2 ? n_tiles2 : sms / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * (pairs > 0 ? pairs : 1)));
+    cfg.blockDim = dim3(psd::kLmThreads);
+    cfg.dynamicSmemBytes = psd::kLm2SmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    TimedLaunch timed(stream, 0);
+    if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<1>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+    psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);
+    if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<2>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+  } else {
+    const unsigned grid = static_cast<unsigned>(n_tiles < sms ? n_tiles : sms);
     TimedLaunch timed(stream, 0);
     psd::lmhead_sweep_kernel<1><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
     psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);

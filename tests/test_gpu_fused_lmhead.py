@@ -112,6 +112,27 @@ def test_fused_lmhead_full_size_cfg5_sampled(psd, oracle):
             assert nt[b] == orc["next_token"][0]     # sequence 0 has batch row indices 0..K-1: same Philox blocks
 
 
+def test_fused_lmhead_one_sm_variant_agrees(psd, oracle):
+    """The one-SM sweeps (PYRAMIDSD_LMHEAD_PAIR=0, read when the library first runs the fused path) in a fresh
+    process against the oracle, so that both variants stay covered."""
+    import os, subprocess, sys, textwrap
+    code = textwrap.dedent("""
+        import sys, numpy as np, torch
+        sys.path.insert(0, %r); sys.path.insert(0, %r)
+        import oracle
+        from paper_2510_12966_b200 import binding
+        from test_gpu_fused_lmhead import make_case, run_both, check
+        binding.load_library(); torch.cuda.set_device(0)
+        h, w_t, z_q, tok = make_case(32, 8, 512, 2048, seed=61, w_scale=0.08)
+        gpu, orc = run_both(binding, oracle, h, w_t, z_q, tok, 0.1, 0)
+        check(gpu, orc, 0.1, 0)
+        print("ok")
+    """) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, PYRAMIDSD_LMHEAD_PAIR="0")
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
+
+
 def test_fused_lmhead_rejects_unsupported_shapes(psd):
     dev = torch.device("cuda:0")
     h = torch.zeros((264, 128), dtype=torch.bfloat16, device=dev)
