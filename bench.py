@@ -122,13 +122,17 @@ def run_ours(args):
     if args.batch > 0:
         import dataclasses
         w = dataclasses.replace(w, B=args.batch, name=f"{w.name}[B={args.batch}]")
+    if args.logits_dtype and args.logits_dtype != w.dtype:
+        import dataclasses
+        w = dataclasses.replace(w, dtype=args.logits_dtype, name=f"{w.name}[{args.logits_dtype}]")
     es = 2 if w.dtype == "bf16" else 4
 
     # Each rank owns its own batch of B sequences (weak scaling; sequences are independent, no collective
     # on the data path). Two distinct rounds alternate so that a step never re-reads a buffer it just used;
     # one round (788 MB for cfg3) already exceeds the 126 MB L2.
     n_bufs = 2
-    rounds = [workloads.workload_inputs(cfg, 100 * rank + i, device=dev, B=w.B) for i in range(n_bufs)]
+    rounds = [workloads.make_pyramid_inputs(w.B, w.K_d, w.K_q, w.V, w.dtype, 1000 * cfg + 100 * rank + i, w.boost, w.sigma_q,
+                                            w.sigma_d, device=dev) for i in range(n_bufs)]
     outs = [{k: torch.empty(w.B, dtype=torch.int32, device=dev)
              for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")} for _ in range(n_bufs)]
     mode, seed = binding.FUZZY, 0
@@ -248,6 +252,62 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def run_single_stage(args):
+    """Config 1: the tiny fp32 single-stage check (B=1, K=4, V=32000). A step = one fuzzy (tau=0.3) and one
+    strict pyramidsd_verify_stage call on one round of inputs; 1 MB per step, so this line is a latency figure."""
+    from paper_2510_12966_b200 import binding, workloads
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1 and int(os.environ.get("RANK", "0")) != 0:
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the verification path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    binding.load_library()
+    binding.set_stream()
+    w = workloads.CONFIGS[1]
+    rounds = [workloads.workload_inputs(1, i, device=dev) for i in range(64)]
+    outs = (torch.empty(w.B, dtype=torch.int32, device=dev), torch.empty(w.B, dtype=torch.int32, device=dev))
+
+    def step(i):
+        zs, zl, tok = rounds[i % 64]
+        binding.verify_stage(zs, zl, tok, w.tau_q, binding.FUZZY, 0, i, *outs)
+        binding.verify_stage(zs, zl, tok, w.tau_q, binding.STRICT, 0, i, *outs)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches0 = binding.launch_count()
+    binding.kernel_timing_begin()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms_total = ev0.elapsed_time(ev1)
+    ms_rs, n_rs, ms_fin, n_fin = binding.kernel_timing_end()
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop()
+    peaks, peak_kind = load_peaks()
+    pos = 2 * w.B * w.K_d * args.steps
+    row_bytes = 2 * w.V * 4
+    achieved = (n_rs * w.B * w.K_d * row_bytes) / (ms_rs * 1e-3) / 1e9 if ms_rs > 0 else 0.0
+    print(json.dumps({
+        "metric": METRIC, "value": pos / (ms_total * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": f"{w.name}: B=1, K=4, V=32000, fp32 logits, one fuzzy (tau=0.3) and one strict call per step, 64 rounds",
+                   "l2_policy": "64 rounds of 1 MB stay in L2: this is a latency figure, not a bandwidth one",
+                   "us_per_call": ms_total / args.steps / 2 * 1e3},
+        "roofline": {"bound": "hbm", "kernel": "rowstats (4 row pairs per launch: launch-latency-bound)", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
+                     "traffic": None, "launches": n_rs, "avg_launch_ms": ms_rs / max(n_rs, 1),
+                     "finalize_ms_per_launch": ms_fin / max(n_fin, 1)},
+        "gpu_launches": launches, "clocks": clocks}))
 
 
 def run_fused(args):
@@ -426,7 +486,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--logits-dtype", choices=["bf16", "f32"], default=None, help="override the workload's logits dtype (cfg4's fp32 run)")
     ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences per step of the CPU-oracle reference arm")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (small profiling cases)")
     ap.add_argument("--vocab", type=int, default=0, help="override the vocabulary size V of cfg5 (small profiling cases)")
@@ -441,6 +502,8 @@ def main():
         run_reference(args)
     elif args.workload == "cfg5":
         run_fused(args)
+    elif args.workload == "cfg1":
+        run_single_stage(args)
     else:
         run_ours(args)
 

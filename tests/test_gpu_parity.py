@@ -360,6 +360,38 @@ def test_pyramid_small_vocab_all_paths(psd, oracle, wl):
         assert len(lens) >= 2
 
 
+@pytest.mark.parametrize("K", [4, 8, 16, 32])
+def test_cfg4_sweep_cells(psd, oracle, wl, K):
+    """BASELINE config 4 recipe (V=152064 bf16, qualifier noise 0.5, draft noise 2.0, boost 8) at B=2: every
+    (K, tau) cell of the sweep, as the stage-1 pairing, the stage-2 pairing and the two-stage wrapper."""
+    w = wl.CONFIGS[4]
+    zd, zq, zt, tok = wl.make_pyramid_inputs(2, K, K, w.V, "bf16", seed=4000 + K, boost=w.boost, sigma_q=w.sigma_q,
+                                             sigma_d=w.sigma_d)
+    ties = 0
+    for tau in wl.CFG4_TAU:
+        _, o1, r1 = run_stage_both(psd, oracle, zd, zq, tok, tau, seed=0, offset=K)          # draft -> qualifier
+        _, o2, r2 = run_stage_both(psd, oracle, zq, zt, tok, tau, seed=0, offset=K + 1)      # qualifier -> target
+        ties += sum(r[k] for r in (r1, r2) for k in ("tie_div", "tie_cdf"))
+        if tau >= 1.0:
+            assert np.all(o1["accept_len"] == K) and np.all(o2["accept_len"] == K)   # tau >= max JS: all accepted
+        Kq = max(K // 2, 1)
+        gpu, orc, hosts = run_pyramid_both(psd, oracle, zd, zq, zt[:, :Kq].contiguous(), tok, tau, tau, 0, 0, 2 * K)
+        t, _ = check_pyramid(oracle, gpu, orc, hosts, "bf16", 0, tau, tau, 0, 2 * K, tok.numpy())
+        ties += t
+    assert ties <= 2
+
+
+def test_cfg4_fp32_k8(psd, oracle, wl):
+    """Config 4's fp32 run at K=8 (B=2): the 1e-5 tolerance class on the large vocabulary."""
+    w = wl.CONFIGS[4]
+    zd, zq, zt, tok = wl.make_pyramid_inputs(2, 8, 8, w.V, "f32", seed=4999, boost=w.boost, sigma_q=w.sigma_q, sigma_d=w.sigma_d)
+    for tau in (0.05, 0.5):
+        _, _, rep = run_stage_both(psd, oracle, zq, zt, tok, tau, seed=0, offset=3)
+        assert rep["max_err_div"] < 1e-5 and rep["max_err_prob"] < 1e-5
+        _, _, rep = run_stage_both(psd, oracle, zd, zq, tok, tau, mode=1, seed=0, offset=4)
+        assert rep["max_err_div"] < 1e-5
+
+
 def test_two_stage_policies_give_the_same_results(psd, wl):
     dev = torch.device("cuda:0")
     zd, zq, zt, tok = [t.to(dev) for t in wl.make_pyramid_inputs(9, 8, 4, 8192, "bf16", seed=23, sigma_q=0.6, sigma_d=1.2)]
