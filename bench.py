@@ -245,7 +245,7 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, rounds)
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
-        traffic = read_profile_traffic(w)
+        traffic = read_profile_traffic(w) if args.two_stage == "fused" else None
         if traffic is not None:
             line["roofline"]["traffic"] = traffic
         print(json.dumps(line))
@@ -417,7 +417,7 @@ def read_profile_traffic(w):
     with open(path) as f:
         t = json.load(f)
     per_row = t.get("dram_bytes_per_row", {}).get(f"V{w.V}_{w.dtype}")
-    return None if per_row is None else per_row * w.B * w.K_d
+    return None if per_row is None else per_row * w.B * (w.K_d + w.K_q)   # rows of the fused statistics launch
 
 
 def cpu_baseline(w, rounds):
