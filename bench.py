@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2] [--impl ours|reference]
 
 A step is one pass of the whole hot path — pyramidsd_verify: the statistics of both stages' rows in one
-launch, then stage-1 finalisation, window build and stage-2 finalisation in another — over one batch of seeded synthetic logits (the BASELINE
-"batched serving" configuration by default: B=64, V=128256, bf16, K_draft=16, K_qual=8). Metric: verified
+launch, then stage-1 finalisation, window build and stage-2 finalisation in another — over one batch of
+seeded synthetic logits (workload configuration 3, "batched serving", by default: B=64, V=128256, bf16,
+K_draft=16, K_qual=8). Metric: verified
 positions per second (a position = one row pair actually verified: all B*K_d stage-1 rows plus the
 stage-2 rows inside each sequence's window). Prints ONE JSON line on rank 0.
 

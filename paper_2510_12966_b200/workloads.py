@@ -121,7 +121,7 @@ def make_fused_inputs(B, K, V, d_model, seed=0, sigma_q=0.7, device="cpu"):
 
 def workload_inputs(cfg: int, round_idx: int = 0, device="cpu", B: Optional[int] = None,
                     K_d: Optional[int] = None, K_q: Optional[int] = None, V: Optional[int] = None):
-    """Inputs of BASELINE config ``cfg`` for one round; B / K / V can be overridden for reduced test cases."""
+    """Inputs of workload configuration ``cfg`` for one round; B / K / V can be overridden for reduced test cases."""
     w = CONFIGS[cfg]
     B = w.B if B is None else B
     K_d = w.K_d if K_d is None else K_d

@@ -70,7 +70,7 @@ def test_fused_lmhead_small_shapes(psd, oracle, B, K, d, V):
 
 
 def test_fused_lmhead_reduced_cfg5(psd, oracle):
-    """BASELINE config 5 recipe (B=32, K=8, d=4096, W ~ N(0, 0.02^2), qualifier noise 0.7) at V=4096."""
+    """workload configuration 5 recipe (B=32, K=8, d=4096, W ~ N(0, 0.02^2), qualifier noise 0.7) at V=4096."""
     h, w_t, z_q, tok = make_case(32, 8, 4096, 4096, seed=5000)
     gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.2, 0)       # the config's threshold: accepts everything here
     check(gpu, orc, 0.2, 0, max_token_ties=2)
@@ -83,7 +83,7 @@ def test_fused_lmhead_reduced_cfg5(psd, oracle):
 
 
 def test_fused_lmhead_full_size_cfg5_sampled(psd, oracle):
-    """BASELINE config 5 at full size (M=256, d=4096, V=128256) in the launch configuration bench.py times;
+    """workload configuration 5 at full size (M=256, d=4096, V=128256) in the launch configuration bench.py times;
     the oracle recomputes two sampled sequences (its double-precision GEMM is far too slow for all 256 rows)."""
     from paper_2510_12966_b200 import workloads
     dev = torch.device("cuda:0")

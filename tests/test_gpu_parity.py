@@ -1,6 +1,6 @@
 """GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded
 inputs and the same Philox stream. Sizes span several tiles and ragged tails; reduced versions of the
-BASELINE workloads run element by element, and the full-size bench configuration is checked on sampled
+benchmark workloads run element by element, and the full-size bench configuration is checked on sampled
 sequences."""
 import math
 
@@ -101,7 +101,7 @@ def test_temperature(psd, oracle, wl):
 
 
 def test_cfg1_tiny_fp32(psd, oracle, wl):
-    """BASELINE config 1: B=1, K=4, V=32000 fp32, fuzzy tau=0.3 and strict, Philox seed 0, several rounds."""
+    """workload configuration 1: B=1, K=4, V=32000 fp32, fuzzy tau=0.3 and strict, Philox seed 0, several rounds."""
     ties = 0
     for rnd in range(8):
         zs, zl, tok = wl.workload_inputs(1, rnd)
@@ -327,7 +327,7 @@ def check_pyramid(oracle, gpu, orc, hosts, dtype, mode, tau_q, tau_t, seed, offs
 
 @pytest.mark.parametrize("mode", [0, 1])
 def test_pyramid_reduced_cfg2(psd, oracle, wl, mode):
-    """BASELINE config 2 (single stream, V=128256 bf16, K_d=8, K_q=4), a few rounds."""
+    """workload configuration 2 (single stream, V=128256 bf16, K_d=8, K_q=4), a few rounds."""
     ties = 0
     for rnd in range(3):
         zd, zq, zt, tok = wl.workload_inputs(2, rnd)
@@ -338,7 +338,7 @@ def test_pyramid_reduced_cfg2(psd, oracle, wl, mode):
 
 
 def test_pyramid_reduced_cfg3(psd, oracle, wl):
-    """BASELINE config 3 recipe at B=6 (V=128256 bf16, K_d=16, K_q=8, per-sequence boost U[4,12])."""
+    """workload configuration 3 recipe at B=6 (V=128256 bf16, K_d=16, K_q=8, per-sequence boost U[4,12])."""
     zd, zq, zt, tok = wl.workload_inputs(3, 0, B=6)
     ties = 0
     for tau_q, tau_t in ((0.4, 0.2), (0.69, 0.5)):
@@ -362,7 +362,7 @@ def test_pyramid_small_vocab_all_paths(psd, oracle, wl):
 
 @pytest.mark.parametrize("K", [4, 8, 16, 32])
 def test_cfg4_sweep_cells(psd, oracle, wl, K):
-    """BASELINE config 4 recipe (V=152064 bf16, qualifier noise 0.5, draft noise 2.0, boost 8) at B=2: every
+    """workload configuration 4 recipe (V=152064 bf16, qualifier noise 0.5, draft noise 2.0, boost 8) at B=2: every
     (K, tau) cell of the sweep, as the stage-1 pairing, the stage-2 pairing and the two-stage wrapper."""
     w = wl.CONFIGS[4]
     zd, zq, zt, tok = wl.make_pyramid_inputs(2, K, K, w.V, "bf16", seed=4000 + K, boost=w.boost, sigma_q=w.sigma_q,
