@@ -14,7 +14,23 @@ constexpr int kFinThreads = 1024;
 constexpr int kFinElemsPerThread = 8;                      // consecutive vocabulary indices per thread and tile
 constexpr int kFinTile = kFinThreads * kFinElemsPerThread;  // 8192 indices per tile
 constexpr int kFinMaxTiles = 1024;                          // V <= 8,388,608
-constexpr int kFinBatch = 32;                               // tiles summed between two CTA-wide barriers
+constexpr int kFinBatch = 32;
+constexpr int kFinCluster = 4;                              // CTAs that share the tile sums of one draw
+
+__device__ __forceinline__ unsigned fin_cluster_rank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void fin_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// one double into the same shared-memory variable of another CTA of the cluster
+__device__ __forceinline__ void fin_remote_store(double* local, unsigned rank, double v) {
+  unsigned addr;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(addr) : "r"(static_cast<unsigned>(__cvta_generic_to_shared(local))), "r"(rank));
+  asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
+}                               // tiles summed between two CTA-wide barriers
 
 template <typename T>
 struct RowView {
@@ -60,9 +76,16 @@ struct FinShared {
   float sh_u2, sh_m2l, sh_l2sl, sh_m2s, sh_l2ss, sh_resid, sh_target;
 };
 
-// One stage's finalisation of sequence b; every thread of the CTA calls it.
-template <typename T>
-__device__ __forceinline__ void finalize_sequence(const StageParams& P, const int b, FinShared& S) {
+// One stage's finalisation of sequence b; every thread of the CTA calls it. With CL > 1 the CTAs of a
+// cluster all call it for the same sequence: each repeats the (cheap) accept scan, the tile sums of the draw
+// are split between them and exchanged through distributed shared memory, and the CTA that owns the chosen
+// tile finishes the draw and writes the results. `nv_given` >= 0 replaces P.n_valid[b], and `tokens_given`
+// (with `n_given` entries; positions beyond it count as token 0) replaces P.tokens for this sequence: that
+// is how stage 2 of a fuzzy pyramid runs without waiting for stage 1's draw.
+template <typename T, int CL>
+__device__ __forceinline__ void finalize_sequence(const StageParams& P, const int b, FinShared& S, const int nv_given = -1,
+                                                  const int32_t* tokens_given = nullptr, const int n_given = 0) {
+  const unsigned cl_rank = (CL > 1) ? fin_cluster_rank() : 0u;
   double (&tile_total)[kFinMaxTiles] = S.tile_total;
   float (&warp_total)[32] = S.warp_total;
   float (&warp_tile)[kFinBatch][32] = S.warp_tile;
@@ -76,7 +99,8 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
   const T* small_seq = static_cast<const T*>(P.small) + b * P.seq_stride_small;
 
   int nv = K;
-  if (P.n_valid != nullptr) nv = min(max(P.n_valid[b], 0), K);
+  if (nv_given >= 0) nv = min(nv_given, K);
+  else if (P.n_valid != nullptr) nv = min(max(P.n_valid[b], 0), K);
 
   // ---- accept bits and prefix length: lane k of warp 0 owns position k (K <= 32) ----
   if (warp == 0) {
@@ -87,7 +111,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
     if (lane < nv) {
       const int r = b * K + lane;
       st = P.stats[r];
-      const int x = P.tokens[r];
+      const int x = (tokens_given != nullptr) ? (lane < n_given ? tokens_given[lane] : 0) : P.tokens[r];
       flags = st.flags | ((x < 0 || x >= V) ? kFlagTokenRange : 0);
       row_uniforms(P.seed, P.offset, static_cast<unsigned>(r), &u, &u2);
       const float nanf_ = __int_as_float(0x7fc00000);
@@ -106,12 +130,14 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
       else if (P.mode == kModeStrict || P.mode == kModeAssisted) acc = coin_ok;
       else acc = fuzzy_ok || coin_ok;
       if (flags) acc = false;
-      if (P.out_div) P.out_div[r] = st.div;
-      if (P.out_resid_mass) P.out_resid_mass[r] = st.resid;
-      if (P.out_p_small_tok) P.out_p_small_tok[r] = qx;
-      if (P.out_p_large_tok) P.out_p_large_tok[r] = px;
-      if (P.out_row_flags) P.out_row_flags[r] = flags;
-    } else if (lane < K) {
+      if (cl_rank == 0) {
+        if (P.out_div) P.out_div[r] = st.div;
+        if (P.out_resid_mass) P.out_resid_mass[r] = st.resid;
+        if (P.out_p_small_tok) P.out_p_small_tok[r] = qx;
+        if (P.out_p_large_tok) P.out_p_large_tok[r] = px;
+        if (P.out_row_flags) P.out_row_flags[r] = flags;
+      }
+    } else if (lane < K && cl_rank == 0) {
       const int r = b * K + lane;
       if (P.out_div) P.out_div[r] = 0.f;
       if (P.out_resid_mass) P.out_resid_mass[r] = 0.f;
@@ -134,6 +160,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
   __syncthreads();
   const int L = sh_L;
   int next = -1;
+  unsigned writer = 0;   // the CTA of the cluster that writes the sequence's results
   bool need_draw = false;
   if (L < sh_nv) {
     if (sh_flags & (kFlagSmallNonfinite | kFlagLargeNonfinite)) next = -2;  // no distribution to draw from
@@ -154,27 +181,37 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
 
     const int n_tiles = (V + kFinTile - 1) / kFinTile;
     float w[kFinElemsPerThread];
-    // level 0: total weight of every tile. The tiles of a batch are independent (their loads overlap);
-    // each warp leaves its sum per tile, then one thread per tile adds the 32 warp sums in warp order.
-    for (int j0 = 0; j0 < n_tiles; j0 += kFinBatch) {
-      const int nb = min(kFinBatch, n_tiles - j0);
+    // level 0: total weight of every tile. CTA `cl_rank` of the cluster takes tiles cl_rank, cl_rank + CL, ...;
+    // the tiles of a batch are independent (their loads overlap); each warp leaves its sum per tile, then one
+    // thread per tile adds the 32 warp sums in warp order and hands the total to every CTA of the cluster.
+    const int my_tiles = (n_tiles - static_cast<int>(cl_rank) + CL - 1) / CL;
+    for (int m0 = 0; m0 < my_tiles; m0 += kFinBatch) {
+      const int nb = min(kFinBatch, my_tiles - m0);
 #pragma unroll 4
-      for (int j = 0; j < nb; ++j) {
-        row.weights((j0 + j) * kFinTile + tid * kFinElemsPerThread, w);
+      for (int m = 0; m < nb; ++m) {
+        const int j = (m0 + m) * CL + static_cast<int>(cl_rank);
+        row.weights(j * kFinTile + tid * kFinElemsPerThread, w);
         float ts = 0.f;
 #pragma unroll
         for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
         ts = warp_reduce<OpSum>(ts);
-        if (lane == 0) warp_tile[j][warp] = ts;
+        if (lane == 0) warp_tile[m][warp] = ts;
       }
       __syncthreads();
       if (tid < nb) {
         double tt = 0.0;
         for (int k = 0; k < 32; ++k) tt += static_cast<double>(warp_tile[tid][k]);
-        tile_total[j0 + tid] = tt;
+        const int j = (m0 + tid) * CL + static_cast<int>(cl_rank);
+        tile_total[j] = tt;
+        if (CL > 1) {
+#pragma unroll
+          for (int p = 0; p < CL; ++p)
+            if (p != static_cast<int>(cl_rank)) fin_remote_store(&tile_total[j], static_cast<unsigned>(p), tt);
+        }
       }
       __syncthreads();
     }
+    if (CL > 1) fin_cluster_sync();   // every CTA now holds every tile's total
     if (tid == 0) {
       double total = 0.0;
       for (int j = 0; j < n_tiles; ++j) total += tile_total[j];
@@ -195,7 +232,8 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
     }
     __syncthreads();
     const int tile = sh_tile;
-    if (tile >= 0) {
+    writer = (CL > 1 && tile >= 0) ? static_cast<unsigned>(tile % CL) : 0u;   // the CTA that summed the chosen tile goes on
+    if (tile >= 0 && cl_rank == writer) {
       // level 1: warps of the chosen tile
       const int i0 = tile * kFinTile + tid * kFinElemsPerThread;
       row.weights(i0, w);
@@ -255,7 +293,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
     }
   }
 
-  if (tid == 0) {
+  if (tid == 0 && cl_rank == writer) {
     P.out_accept_len[b] = L;
     P.out_next_token[b] = next;
     if (P.window != nullptr) {
@@ -269,22 +307,61 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
   }
 }
 
-template <typename T>
+template <typename T, int CL>
 __global__ void __launch_bounds__(kFinThreads) finalize_kernel(const StageParams P) {
   __shared__ FinShared S;
-  finalize_sequence<T>(P, blockIdx.x, S);
+  finalize_sequence<T, CL>(P, blockIdx.x / CL, S);
+  if (CL > 1) fin_cluster_sync();   // nobody leaves while a peer may still post tile sums into its shared memory
 }
 
 // Both stages of the two-stage wrapper for one sequence: stage 1 (draft against qualifier) writes the
 // window and its length, stage 2 (window against target) reads them back. The statistics of every
 // stage-2 row were computed beforehand, whatever the window turned out to be.
-template <typename T>
+template <typename T, int CL>
 __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_kernel(const StageParams P1, const StageParams P2) {
   __shared__ FinShared S;
-  finalize_sequence<T>(P1, blockIdx.x, S);
-  __threadfence_block();
-  __syncthreads();   // the window and its length, written by thread 0, are visible to the whole CTA
-  finalize_sequence<T>(P2, blockIdx.x, S);
+  finalize_sequence<T, CL>(P1, blockIdx.x / CL, S);
+  __threadfence();
+  __syncthreads();
+  if (CL > 1) fin_cluster_sync();   // the window and its length, written by one thread of the cluster, are visible to all of it
+  finalize_sequence<T, CL>(P2, blockIdx.x / CL, S);
+  if (CL > 1) fin_cluster_sync();
+}
+
+// Fuzzy mode only: the stage-2 half of the pyramid does not need stage 1's drawn token -- the accept bits
+// depend on the divergences alone, and the window length follows from stage 1's accept scan -- so the two
+// stages of a sequence run side by side, one cluster each. Cluster 2b is stage 1 (it also writes the
+// window); cluster 2b+1 repeats stage 1's cheap scan to get the window length, then runs stage 2 on the
+// accepted draft prefix.
+template <typename T, int CL>
+__global__ void __launch_bounds__(kFinThreads) finalize_pyramid_split_kernel(const StageParams P1, const StageParams P2) {
+  __shared__ FinShared S;
+  __shared__ int sh_L1, sh_n2;
+  const int unit = blockIdx.x / CL, b = unit >> 1;
+  if ((unit & 1) == 0) {
+    finalize_sequence<T, CL>(P1, b, S);
+  } else {
+    if (threadIdx.x < 32) {
+      const int lane = threadIdx.x, K = P1.K;
+      bool acc = true;
+      int flags = 0;
+      if (lane < K) {
+        const RowStats st = P1.stats[b * K + lane];
+        const int x = P1.tokens[b * K + lane];
+        flags = st.flags | ((x < 0 || x >= P1.V) ? kFlagTokenRange : 0);
+        acc = (st.div <= P1.threshold) && !flags;
+      }
+      const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
+      const int L1 = rejected ? (__ffs(rejected) - 1) : K;
+      const int flags_L = __shfl_sync(0xffffffffu, flags, min(L1, 31));
+      // a correction token follows the accepted prefix unless everything was accepted or the rejected row has no distribution
+      const int has_next = (L1 < K && !(flags_L & (kFlagSmallNonfinite | kFlagLargeNonfinite))) ? 1 : 0;
+      if (lane == 0) { sh_L1 = L1; sh_n2 = min(L1 + has_next, P2.K); }
+    }
+    __syncthreads();
+    finalize_sequence<T, CL>(P2, b, S, sh_n2, P1.tokens + b * P1.K, sh_L1);
+  }
+  if (CL > 1) fin_cluster_sync();
 }
 
 }  // namespace psd

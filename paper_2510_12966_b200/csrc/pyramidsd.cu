@@ -185,13 +185,32 @@ int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_si
   return check_launch();
 }
 
+// The finalisation kernels run as clusters of kFinCluster CTAs per sequence (per stage in the split form).
+template <typename Kernel, typename... Args>
+cudaError_t launch_fin_clusters(Kernel kernel, unsigned units, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(units * psd::kFinCluster);
+  cfg.blockDim = dim3(psd::kFinThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = psd::kFinCluster;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 int launch_finalize(const StageParams& P, int dtype, cudaStream_t stream) {
   if (P.B == 0) return PSD_OK;
-  const dim3 grid(static_cast<unsigned>(P.B)), block(psd::kFinThreads);
   TimedLaunch timed(stream, 1);
-  if (dtype == PSD_F32) psd::finalize_kernel<float><<<grid, block, 0, stream>>>(P);
-  else psd::finalize_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(P);
+  cudaError_t e;
+  if (dtype == PSD_F32) e = launch_fin_clusters(psd::finalize_kernel<float, psd::kFinCluster>, static_cast<unsigned>(P.B), stream, P);
+  else e = launch_fin_clusters(psd::finalize_kernel<__nv_bfloat16, psd::kFinCluster>, static_cast<unsigned>(P.B), stream, P);
   g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (e != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
   return check_launch();
 }
 
@@ -377,11 +396,19 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   rc = launch_rowstats(PS, dtype, variant, 0, stream);
   if (rc != PSD_OK) return rc;
   {
-    const dim3 grid(static_cast<unsigned>(B)), block(psd::kFinThreads);
     TimedLaunch timed(stream, 1);
-    if (dtype == PSD_F32) psd::finalize_pyramid_kernel<float><<<grid, block, 0, stream>>>(P1, P2);
-    else psd::finalize_pyramid_kernel<__nv_bfloat16><<<grid, block, 0, stream>>>(P1, P2);
+    cudaError_t e;
+    constexpr int CL = psd::kFinCluster;
+    if (mode == PSD_FUZZY) {
+      // threshold-only acceptance: stage 2 does not depend on stage 1's drawn token, the stages run side by side
+      if (dtype == PSD_F32) e = launch_fin_clusters(psd::finalize_pyramid_split_kernel<float, CL>, 2u * B, stream, P1, P2);
+      else e = launch_fin_clusters(psd::finalize_pyramid_split_kernel<__nv_bfloat16, CL>, 2u * B, stream, P1, P2);
+    } else {
+      if (dtype == PSD_F32) e = launch_fin_clusters(psd::finalize_pyramid_kernel<float, CL>, static_cast<unsigned>(B), stream, P1, P2);
+      else e = launch_fin_clusters(psd::finalize_pyramid_kernel<__nv_bfloat16, CL>, static_cast<unsigned>(B), stream, P1, P2);
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
   }
   return check_launch();
 }
