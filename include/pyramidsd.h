@@ -180,7 +180,8 @@ int pyramidsd_verify_stage_noalloc(const void* logits_small, const void* logits_
  *   w_t           [V, d_model]  bf16, row-major: the LM-head weight as checkpoints store it (out x in), device
  *   logits_small  [B, K, V] bf16, device; tokens [B, K] int32
  *   out_div, out_resid_mass  [B, K] float32 or NULL
- * Requires B*K <= 256 and d_model a multiple of 64 (else PSD_ERR_UNSUPPORTED); hidden and w_t 16-byte aligned.
+ * Requires d_model a multiple of 64 (else PSD_ERR_UNSUPPORTED); hidden and w_t 16-byte aligned. Rows are
+ * processed in blocks of 256 (B*K <= 256 is the intended case: one block, the weight streamed twice).
  * Jensen-Shannon divergence, temperature 1. Runs the GEMM twice (the divergence needs the large model's
  * normaliser first). Scratch (partial sums per row and 128-column tile) is library-owned, grown with
  * cudaMalloc on first use. Asynchronous on `cuda_stream`; device-side timeouts via pyramidsd_last_status(). */

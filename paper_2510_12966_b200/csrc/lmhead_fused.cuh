@@ -43,6 +43,7 @@ struct LmParams {
   const __nv_bfloat16* small;     // [M, V] bf16 logits of the small model
   const int32_t* tokens;          // [M]
   int M, d, V, n_tiles;
+  int row0;                       // first row of the 256-row block this launch works on
   float c;                        // log2(e) / T
   float2* part_large;             // sweep 1: [M][n_tiles] (max in scaled base-2 domain, sum)
   float2* part_small;
@@ -244,7 +245,7 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (fills > 0) wait_phase(&bars->empty[stage], (fills - 1u) & 1u);
           unsigned char* sa = tiles + static_cast<size_t>(stage) * kLmStageBytes;
           mbar_arrive_expect_tx(&bars->full[stage], kLmStageBytes);
-          tma_load_2d(sa, &map_a, ks * kLmK, 0, &bars->full[stage]);                      // hidden rows 0..255
+          tma_load_2d(sa, &map_a, ks * kLmK, P.row0, &bars->full[stage]);                 // 256 hidden rows of the block
           tma_load_2d(sa + kLmABytes, &map_b, ks * kLmK, tile * kLmN, &bars->full[stage]);  // W^T rows tile*128..
           if (++stage == kLmStages) { stage = 0; ++fills; }
         }
@@ -283,7 +284,7 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ================================ epilogue ================================
     // a warp reads the TMEM lanes 32 * (its index in the CTA mod 4) ..; warps 2..5 take accumulator 0, 6..9 accumulator 1
     const int quarter = warp & 3, half = (warp - 2) >> 2;
-    const int row = half * 128 + quarter * 32 + lane;            // this thread's row of the tile (= TMEM lane + 128*half)
+    const int row = P.row0 + half * 128 + quarter * 32 + lane;   // this thread's row (TMEM lane + 128*half of the block)
     const bool row_ok = row < P.M;
     const float c = P.c;
     const __nv_bfloat16* small_row = P.small + static_cast<size_t>(row_ok ? row : 0) * P.V;
@@ -404,7 +405,7 @@ lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
           unsigned char* sa = tiles + static_cast<size_t>(stage) * kLm2StageBytes;
           // the even CTA's barrier counts the bytes of both CTAs
           if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2u * kLm2StageBytes);
-          tma_load_2d_pair(sa, &map_a, ks * kLmK, static_cast<int>(rank) * 128, &bars->full[stage]);
+          tma_load_2d_pair(sa, &map_a, ks * kLmK, P.row0 + static_cast<int>(rank) * 128, &bars->full[stage]);
           tma_load_2d_pair(sa + kLm2HalfBytes, &map_b, ks * kLmK, tile * kLm2N + static_cast<int>(rank) * 128, &bars->full[stage]);
           if (++stage == kLm2Stages) { stage = 0; ++fills; }
         }
@@ -438,7 +439,7 @@ lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   } else {
     // ================================ epilogue (both CTAs) ================================
     const int quarter = warp & 3, half = (warp - 2) >> 2;          // TMEM lanes 32*quarter.., columns 128*half..
-    const int row = static_cast<int>(rank) * 128 + quarter * 32 + lane;
+    const int row = P.row0 + static_cast<int>(rank) * 128 + quarter * 32 + lane;
     const bool row_ok = row < P.M;
     const float c = P.c;
     const __nv_bfloat16* small_row = P.small + static_cast<size_t>(row_ok ? row : 0) * P.V;
@@ -554,8 +555,9 @@ __global__ void __launch_bounds__(256) lmhead_final_kernel(const LmFinalParams F
       sh_res[k] = fmaxf(static_cast<float>(res), 0.f);
       sh_pm[k] = static_cast<float>(pm);
       sh_px[k] = px; sh_qx[k] = qx; sh_flag[k] = flags;
-      if (F.out_div) F.out_div[r] = flags ? __int_as_float(0x7fc00000) : sh_div[k];
-      if (F.out_resid) F.out_resid[r] = flags ? __int_as_float(0x7fc00000) : sh_res[k];
+      const bool no_dist = (flags & (kFlagSmallNonfinite | kFlagLargeNonfinite)) != 0;   // a bad token leaves D and R intact
+      if (F.out_div) F.out_div[r] = no_dist ? __int_as_float(0x7fc00000) : sh_div[k];
+      if (F.out_resid) F.out_resid[r] = no_dist ? __int_as_float(0x7fc00000) : sh_res[k];
     }
   }
   __syncthreads();

@@ -574,7 +574,7 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
                                   int32_t* out_next_token, float* out_div, float* out_resid_mass, void* cuda_stream) {
   if (!valid_mode(mode) || B < 0 || K < 0 || K > 32 || V < 1 || d_model < 1 || std::isnan(threshold)) return PSD_ERR_INVALID_ARG;
   const long long M = static_cast<long long>(B) * K;
-  if (M > psd::kLmM || (d_model % psd::kLmK) != 0) return PSD_ERR_UNSUPPORTED;
+  if ((d_model % psd::kLmK) != 0) return PSD_ERR_UNSUPPORTED;
   if (B == 0) return PSD_OK;
   if (!out_accept_len || !out_next_token) return PSD_ERR_INVALID_ARG;
   if (K > 0 && (!hidden || !w_t || !logits_small || !tokens)) return PSD_ERR_INVALID_ARG;
@@ -686,15 +686,30 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
     cfg.attrs = at;
     cfg.numAttrs = 1;
     TimedLaunch timed(stream, 0);
-    if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<1>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+    // more than 256 rows: one pair of sweeps per block of 256 rows (the weight is streamed once per block and sweep)
+    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
+      L.row0 = r0;
+      if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<1>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+    }
     psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);
-    if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<2>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
+      L.row0 = r0;
+      if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<2>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+    }
+    L.row0 = 0;
   } else {
     const unsigned grid = static_cast<unsigned>(n_tiles < sms ? n_tiles : sms);
     TimedLaunch timed(stream, 0);
-    psd::lmhead_sweep_kernel<1><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
+    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
+      L.row0 = r0;
+      psd::lmhead_sweep_kernel<1><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
+    }
     psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);
-    psd::lmhead_sweep_kernel<2><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
+    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
+      L.row0 = r0;
+      psd::lmhead_sweep_kernel<2><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
+    }
+    L.row0 = 0;
   }
   psd::LmFinalParams F{};
   F.lm = L;
@@ -712,7 +727,7 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
     TimedLaunch timed(stream, 1);
     psd::lmhead_final_kernel<<<static_cast<unsigned>(B), 256, 0, stream>>>(F);
   }
-  g_launches.fetch_add(4, std::memory_order_relaxed);
+  g_launches.fetch_add(2 + 2 * static_cast<uint64_t>((M + psd::kLmM - 1) / psd::kLmM), std::memory_order_relaxed);
   return check_launch();
 }
 

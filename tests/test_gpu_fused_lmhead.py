@@ -133,13 +133,33 @@ def test_fused_lmhead_one_sm_variant_agrees(psd, oracle):
     assert out.returncode == 0 and "ok" in out.stdout, out.stderr[-2000:]
 
 
+def test_fused_lmhead_more_than_one_row_block(psd, oracle):
+    """B*K = 40*8 = 320 rows: two blocks of 256 rows (the second one partial)."""
+    h, w_t, z_q, tok = make_case(40, 8, 256, 1536, seed=77, w_scale=0.08)
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.08, 0)
+    check(gpu, orc, 0.08, 0, max_token_ties=2)
+    tau = float(np.float32(np.median(orc["div"])))      # a threshold that splits the rows, in both blocks
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, tau, 0)
+    check(gpu, orc, tau, 0, max_token_ties=3)
+    assert 0 < orc["accept_len"][:32].sum() < 32 * 8 and 0 < orc["accept_len"][32:].sum() < 8 * 8
+
+
+def test_fused_lmhead_masked_and_poisoned_rows(psd, oracle):
+    """-inf in the small logits (masked vocabulary), a NaN in a hidden row, a token out of range."""
+    h, w_t, z_q, tok = make_case(4, 4, 128, 1000, seed=78, w_scale=0.08)
+    z_q[0, 1, 100:700] = -float("inf")
+    h[2 * 4 + 1, 5] = float("nan")            # sequence 2, position 1: the large model's row is poisoned
+    tok[3, 2] = 1000                           # out of range
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 1.0, 0)
+    assert gpu["accept_len"][2] == 1 and gpu["next_token"][2] == -2
+    assert gpu["accept_len"][3] == 2 and gpu["next_token"][3] >= 0
+    assert np.array_equal(gpu["accept_len"], orc["accept_len"])
+    ok = np.isfinite(orc["div"])
+    assert np.abs(gpu["div"][ok] - orc["div"][ok]).max() < 2e-3
+
+
 def test_fused_lmhead_rejects_unsupported_shapes(psd):
     dev = torch.device("cuda:0")
-    h = torch.zeros((264, 128), dtype=torch.bfloat16, device=dev)
-    w = torch.zeros((512, 128), dtype=torch.bfloat16, device=dev)
-    z = torch.zeros((33, 8, 512), dtype=torch.bfloat16, device=dev)
-    t = torch.zeros((33, 8), dtype=torch.int32, device=dev)
-    assert psd.verify_fused_lmhead(h, w, z, t, 0.1, raise_on_error=False)["status"] == psd.ERR_UNSUPPORTED   # 264 rows
     h2 = torch.zeros((8, 96), dtype=torch.bfloat16, device=dev)
     w2 = torch.zeros((512, 96), dtype=torch.bfloat16, device=dev)
     z2 = torch.zeros((1, 8, 512), dtype=torch.bfloat16, device=dev)
