@@ -105,7 +105,7 @@ typedef struct psd_stage_args {
   void* stream;                  /* cudaStream_t, or NULL for the stream set by pyramidsd_set_stream */
   int32_t use_stream_field;      /* non-zero: take `stream` even when it is NULL (the legacy default stream) */
   int32_t kernel_variant;        /* psd_kernel_variant */
-  int32_t cluster_size;          /* CTAs per cluster for the cluster kernel (power of two <= 16); 0 = chosen by the library */
+  int32_t cluster_size;          /* CTAs per cluster for the cluster kernel (1..16); 0 = chosen by the library */
 } psd_stage_args;
 
 /* One verification stage (Sec. 3.1 for one model pair; Sec. 3.2 applies it twice). Jensen-Shannon

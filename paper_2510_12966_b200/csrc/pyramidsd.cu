@@ -821,9 +821,7 @@ int pyramidsd_cluster_occupancy(int B, int K, int V, psd_dtype dtype, int* out_c
   const bool ok = B > 0 && K > 0 && psd::cluster_geometry(P, dtype, 0, &g);
   if (out_cluster_size) *out_cluster_size = ok ? g.cs : 0;
   if (out_max_active_clusters) {
-    int log2cs = 0;
-    while (ok && (1 << log2cs) < g.cs) ++log2cs;
-    *out_max_active_clusters = ok ? psd::cluster_max_active_any(dtype, PSD_DIV_JS, log2cs) : 0;
+    *out_max_active_clusters = ok ? psd::cluster_max_active_any(dtype, PSD_DIV_JS, g.cs) : 0;
   }
   return PSD_OK;
 }

@@ -772,7 +772,7 @@ inline int cluster_max_active(int cs) {
 constexpr int kClMaxDevices = 64;
 struct ClusterDeviceCache {
   bool prepared[2][3];
-  int max_active[2][3][5];   // 0 = not queried yet, -1 = none fit
+  int max_active[2][3][kClMaxRanks + 1];   // by cluster size; 0 = not queried yet, -1 = none fit
   int sm_count;
 };
 inline ClusterDeviceCache* cluster_cache() {
@@ -783,30 +783,30 @@ inline ClusterDeviceCache* cluster_cache() {
 }
 
 template <typename T, int DIV>
-inline int cluster_max_active_cached(int dtype, int log2cs) {
+inline int cluster_max_active_cached(int dtype, int cs) {
   ClusterDeviceCache* cc = cluster_cache();
   if (cc == nullptr) return 0;
   if (!cc->prepared[dtype][DIV]) {
     if (cluster_prepare<T, DIV>() != cudaSuccess) { cudaGetLastError(); return 0; }
     cc->prepared[dtype][DIV] = true;
   }
-  int& slot = cc->max_active[dtype][DIV][log2cs];
+  int& slot = cc->max_active[dtype][DIV][cs];
   if (slot == 0) {
-    const int n = cluster_max_active<T, DIV>(1 << log2cs);
+    const int n = cluster_max_active<T, DIV>(cs);
     slot = n > 0 ? n : -1;
   }
   return slot > 0 ? slot : 0;
 }
 
-inline int cluster_max_active_any(int dtype, int div_kind, int log2cs) {
+inline int cluster_max_active_any(int dtype, int div_kind, int cs) {
   if (dtype == 0) {
-    if (div_kind == kDivJS) return cluster_max_active_cached<float, kDivJS>(0, log2cs);
-    if (div_kind == kDivTV) return cluster_max_active_cached<float, kDivTV>(0, log2cs);
-    return cluster_max_active_cached<float, kDivKL>(0, log2cs);
+    if (div_kind == kDivJS) return cluster_max_active_cached<float, kDivJS>(0, cs);
+    if (div_kind == kDivTV) return cluster_max_active_cached<float, kDivTV>(0, cs);
+    return cluster_max_active_cached<float, kDivKL>(0, cs);
   }
-  if (div_kind == kDivJS) return cluster_max_active_cached<__nv_bfloat16, kDivJS>(1, log2cs);
-  if (div_kind == kDivTV) return cluster_max_active_cached<__nv_bfloat16, kDivTV>(1, log2cs);
-  return cluster_max_active_cached<__nv_bfloat16, kDivKL>(1, log2cs);
+  if (div_kind == kDivJS) return cluster_max_active_cached<__nv_bfloat16, kDivJS>(1, cs);
+  if (div_kind == kDivTV) return cluster_max_active_cached<__nv_bfloat16, kDivTV>(1, cs);
+  return cluster_max_active_cached<__nv_bfloat16, kDivKL>(1, cs);
 }
 
 inline int cluster_sm_count() {
@@ -856,7 +856,7 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
     if (env_cs > 0) forced_cs = env_cs;
   }
   if (forced_cs > 0) {
-    if (forced_cs > kClMaxRanks || (forced_cs & (forced_cs - 1)) != 0) return false;
+    if (forced_cs > kClMaxRanks) return false;
     cs = forced_cs;
     cluster_slices(P.V, es, cs, &slice, &chunks);
     if (chunks > kClSlots - 1) return false;
@@ -873,9 +873,7 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
       cluster_slices(P.V, es, cs, &slice, &chunks);
     }
   }
-  int log2cs = 0;
-  while ((1 << log2cs) < cs) ++log2cs;
-  const int max_active = cluster_max_active_any(dtype, P.div_kind, log2cs);
+  const int max_active = cluster_max_active_any(dtype, P.div_kind, cs);
   if (max_active <= 0) return false;
   g->cs = cs;
   g->slice = slice;

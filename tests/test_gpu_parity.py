@@ -204,7 +204,7 @@ def test_results_are_bit_identical_run_to_run(psd, wl):
 
 # -------------------------------------------------------------------------------------------------- cluster kernel
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("cs", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("cs", [1, 2, 3, 4, 6, 8, 16])
 @pytest.mark.parametrize("V", [2048, 8200, 32000, 128256])
 def test_cluster_kernel_every_cluster_size(psd, oracle, wl, dtype, cs, V):
     """The cluster kernel with the cluster size forced: slices with ragged tails, empty slices (small V
