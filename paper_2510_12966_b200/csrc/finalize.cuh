@@ -15,7 +15,6 @@ constexpr int kFinElemsPerThread = 8;                      // consecutive vocabu
 constexpr int kFinTile = kFinThreads * kFinElemsPerThread;  // 8192 indices per tile
 constexpr int kFinMaxTiles = 1024;                          // V <= 8,388,608
 constexpr int kFinBatch = 32;
-constexpr int kFinCluster = 4;                              // CTAs that share the tile sums of one draw
 
 __device__ __forceinline__ unsigned fin_cluster_rank() {
   unsigned r;

@@ -185,17 +185,18 @@ int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_si
   return check_launch();
 }
 
-// The finalisation kernels run as clusters of kFinCluster CTAs per sequence (per stage in the split form).
+// The finalisation kernels run as clusters of CL CTAs per sequence (per stage in the split form): four while
+// that still leaves SMs to spare, fewer for large batches, where one CTA per sequence already fills the GPU.
 template <typename Kernel, typename... Args>
-cudaError_t launch_fin_clusters(Kernel kernel, unsigned units, cudaStream_t stream, Args... args) {
+cudaError_t launch_fin_clusters(Kernel kernel, int cl, unsigned units, cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(units * psd::kFinCluster);
+  cfg.gridDim = dim3(units * static_cast<unsigned>(cl));
   cfg.blockDim = dim3(psd::kFinThreads);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = psd::kFinCluster;
+  at[0].val.clusterDim.x = static_cast<unsigned>(cl);
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   cfg.attrs = at;
@@ -203,12 +204,27 @@ cudaError_t launch_fin_clusters(Kernel kernel, unsigned units, cudaStream_t stre
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+int fin_cluster_size(long long units) {
+  int sms = psd::cluster_sm_count();
+  if (sms <= 0) sms = 148;
+  if (units * 4 <= 2ll * sms) return 4;
+  if (units * 2 <= 2ll * sms) return 2;
+  return 1;
+}
+
+#define PSD_FIN_DISPATCH(KERNEL, T, cl, units, stream, ...)                                              \
+  ((cl) == 4 ? launch_fin_clusters(psd::KERNEL<T, 4>, 4, units, stream, __VA_ARGS__)                        \
+   : (cl) == 2 ? launch_fin_clusters(psd::KERNEL<T, 2>, 2, units, stream, __VA_ARGS__)                      \
+               : launch_fin_clusters(psd::KERNEL<T, 1>, 1, units, stream, __VA_ARGS__))
+
 int launch_finalize(const StageParams& P, int dtype, cudaStream_t stream) {
   if (P.B == 0) return PSD_OK;
   TimedLaunch timed(stream, 1);
+  const int cl = fin_cluster_size(P.B);
+  const unsigned units = static_cast<unsigned>(P.B);
   cudaError_t e;
-  if (dtype == PSD_F32) e = launch_fin_clusters(psd::finalize_kernel<float, psd::kFinCluster>, static_cast<unsigned>(P.B), stream, P);
-  else e = launch_fin_clusters(psd::finalize_kernel<__nv_bfloat16, psd::kFinCluster>, static_cast<unsigned>(P.B), stream, P);
+  if (dtype == PSD_F32) e = PSD_FIN_DISPATCH(finalize_kernel, float, cl, units, stream, P);
+  else e = PSD_FIN_DISPATCH(finalize_kernel, __nv_bfloat16, cl, units, stream, P);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   if (e != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
   return check_launch();
@@ -398,14 +414,15 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   {
     TimedLaunch timed(stream, 1);
     cudaError_t e;
-    constexpr int CL = psd::kFinCluster;
     if (mode == PSD_FUZZY) {
       // threshold-only acceptance: stage 2 does not depend on stage 1's drawn token, the stages run side by side
-      if (dtype == PSD_F32) e = launch_fin_clusters(psd::finalize_pyramid_split_kernel<float, CL>, 2u * B, stream, P1, P2);
-      else e = launch_fin_clusters(psd::finalize_pyramid_split_kernel<__nv_bfloat16, CL>, 2u * B, stream, P1, P2);
+      const int cl = fin_cluster_size(2ll * B);
+      if (dtype == PSD_F32) e = PSD_FIN_DISPATCH(finalize_pyramid_split_kernel, float, cl, 2u * B, stream, P1, P2);
+      else e = PSD_FIN_DISPATCH(finalize_pyramid_split_kernel, __nv_bfloat16, cl, 2u * B, stream, P1, P2);
     } else {
-      if (dtype == PSD_F32) e = launch_fin_clusters(psd::finalize_pyramid_kernel<float, CL>, static_cast<unsigned>(B), stream, P1, P2);
-      else e = launch_fin_clusters(psd::finalize_pyramid_kernel<__nv_bfloat16, CL>, static_cast<unsigned>(B), stream, P1, P2);
+      const int cl = fin_cluster_size(B);
+      if (dtype == PSD_F32) e = PSD_FIN_DISPATCH(finalize_pyramid_kernel, float, cl, static_cast<unsigned>(B), stream, P1, P2);
+      else e = PSD_FIN_DISPATCH(finalize_pyramid_kernel, __nv_bfloat16, cl, static_cast<unsigned>(B), stream, P1, P2);
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }

@@ -140,12 +140,12 @@ __device__ __forceinline__ uint4 lds128(const void* p) {
 // Every role of every CTA of a cluster walks the same list: rows q, q + n_clusters, ... of the [B*K]
 // grid, skipping positions at or beyond the sequence's n_valid. `n` counts the rows taken so far.
 struct RowWalk {
-  int next_r, stride, rows, rows1, K;
+  int next_r, stride, rows, rows1, K, B;
   const int32_t* n_valid;
   int n;     // ordinal of the current row among the rows this cluster takes
   int r;     // current row index (valid after advance() returned true)
   __device__ void init(const StageParams& P, int cluster_id, int n_clusters) {
-    next_r = cluster_id; stride = n_clusters; rows = P.B * (P.K + P.K2); rows1 = P.B * P.K; K = P.K;
+    next_r = cluster_id; stride = n_clusters; rows = P.B * (P.K + P.K2); rows1 = P.B * P.K; K = P.K; B = P.B;
     n_valid = P.n_valid; n = -1; r = -1;
   }
   __device__ bool advance() {
@@ -153,8 +153,13 @@ struct RowWalk {
       const int cand = next_r;
       next_r += stride;
       if (n_valid != nullptr && cand < rows1) {   // n_valid speaks of the first row set only
-        const int b = cand / K, k = cand - b * K;
+        // candidates are taken position-major (all sequences' position 0, then position 1, ...): the early
+        // positions, which are the ones that are usually valid, then spread evenly over the clusters
+        // whatever the number of clusters and K have in common
+        const int k = cand / B, b = cand - k * B;
         if (k >= n_valid[b]) continue;
+        r = b * K + k; ++n;
+        return true;
       }
       r = cand; ++n;
       return true;
@@ -861,11 +866,16 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
     cluster_slices(P.V, es, cs, &slice, &chunks);
     if (chunks > kClSlots - 1) return false;
   } else {
-    for (cs = 1; cs <= kClMaxRanks; cs *= 2) {
-      cluster_slices(P.V, es, cs, &slice, &chunks);
-      if (chunks <= kClSlots - 3) break;
-    }
-    if (cs > kClMaxRanks) return false;
+    // the smallest cluster whose slice leaves at least five ring slots beyond a row (measured: 4 CTAs for
+    // V = 128256 bf16, 5 for V = 152064 bf16); failing that, three slots
+    const int wanted[2] = {kClSlots - 5, kClSlots - 3};
+    bool found = false;
+    for (int pass = 0; pass < 2 && !found; ++pass)
+      for (cs = 1; cs <= (pass == 0 ? 8 : kClMaxRanks); ++cs) {   // sizes above 8 place few clusters: last resort
+        cluster_slices(P.V, es, cs, &slice, &chunks);
+        if (chunks <= wanted[pass] && cluster_max_active_any(dtype, P.div_kind, cs) > 0) { found = true; break; }
+      }
+    if (!found) return false;
     // few rows: spread each row over more CTAs so that more SMs pull on HBM
     const int sms = cluster_sm_count();
     while (cs < 8 && chunks >= 2 && rows * cs * 2 <= sms) {

@@ -280,6 +280,8 @@ def test_cluster_kernel_other_divergences(psd, oracle, wl, div_kind):
 def test_cluster_occupancy_query(psd):
     cs, n = psd.cluster_occupancy(64, 16, 128256, psd.BF16)
     assert cs == 4 and n >= 16
+    cs, n = psd.cluster_occupancy(256, 8, 152064, psd.BF16)
+    assert cs == 5 and n >= 16
     cs, n = psd.cluster_occupancy(1, 4, 32000, psd.F32)
     assert cs >= 2 and n >= 1
     assert psd.cluster_occupancy(4, 4, 1001, psd.F32) == (0, 0)
