@@ -383,7 +383,18 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   if (rc == PSD_OK) rc = validate_stage(&s2);
   if (rc != PSD_OK) return rc;
   if (t_two_stage_policy == PSD_TWO_STAGE_SEPARATE) {
-    // stage by stage: stage 2's statistics run after stage 1 has fixed the windows and skip the rows beyond them
+    // stage by stage: stage 2's statistics run after stage 1 has fixed the windows and skip the rows beyond them.
+    // Both launches take the cluster size the single-launch schedule would pick, so a row's vocabulary is
+    // cut into the same slices and its statistics come out bit-identical under either policy.
+    {
+      StageParams PS = make_params(&s1, s1.workspace, nullptr);
+      const StageParams Q = make_params(&s2, s2.workspace, nullptr);
+      PS.small2 = Q.small; PS.large2 = Q.large;
+      PS.seq_stride_small2 = Q.seq_stride_small; PS.seq_stride_large2 = Q.seq_stride_large;
+      PS.K2 = K_q;
+      psd::ClusterGeom g{};
+      if (variant != PSD_KERNEL_BASELINE && psd::cluster_geometry(PS, dtype, 0, &g)) s1.cluster_size = s2.cluster_size = g.cs;
+    }
     rc = run_stage(&s1, window, n_window, K_q);
     if (rc != PSD_OK) return rc;
     return run_stage(&s2, nullptr, nullptr, 0);
