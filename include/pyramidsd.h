@@ -212,8 +212,8 @@ int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, fl
  * wrapper). Pure host arithmetic; 0 on invalid arguments. */
 size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype);
 
-/* How pyramidsd_verify / pyramidsd_verify_host schedule the two stages (per host thread; results are the
- * same either way). PSD_TWO_STAGE_FUSED (default): two launches -- one statistics launch over the stage-1 rows
+/* How pyramidsd_verify / pyramidsd_verify_host schedule the two stages (per host thread; results are
+ * bit-identical either way: both use the same split of a row over CTAs). PSD_TWO_STAGE_FUSED (default): two launches -- one statistics launch over the stage-1 rows
  * and all B*K_q stage-2 rows, one finalisation launch for both stages; best when windows are (nearly) full,
  * as in the paper's pipeline, which keeps drafting until the window holds K_q tokens (Fig. 1).
  * PSD_TWO_STAGE_SEPARATE: four launches, stage by stage; stage 2 then skips the rows beyond each window,

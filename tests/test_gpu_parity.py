@@ -394,9 +394,13 @@ def test_cfg4_fp32_k8(psd, oracle, wl):
         assert rep["max_err_div"] < 1e-5
 
 
-def test_two_stage_policies_give_the_same_results(psd, wl):
+@pytest.mark.parametrize("B,K_d,K_q,V,dtype", [(9, 8, 4, 8192, "bf16"), (2, 8, 4, 65536, "bf16"), (3, 16, 8, 128256, "bf16"),
+                                              (5, 5, 2, 32000, "f32")])
+def test_two_stage_policies_give_the_same_results(psd, wl, B, K_d, K_q, V, dtype):
+    """Few rows make the library widen its clusters; the stage-by-stage schedule sees fewer rows per launch than
+    the single-launch one, and must still cut every row the same way."""
     dev = torch.device("cuda:0")
-    zd, zq, zt, tok = [t.to(dev) for t in wl.make_pyramid_inputs(9, 8, 4, 8192, "bf16", seed=23, sigma_q=0.6, sigma_d=1.2)]
+    zd, zq, zt, tok = [t.to(dev) for t in wl.make_pyramid_inputs(B, K_d, K_q, V, dtype, seed=23, sigma_q=0.6, sigma_d=1.2)]
     try:
         psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
         a = psd.verify(zd, zq, zt, tok, 0.3, 0.15, 2, 3, 4)
@@ -408,7 +412,8 @@ def test_two_stage_policies_give_the_same_results(psd, wl):
         psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
     for k in a:
         assert torch.equal(a[k], b[k]), k
-    assert 0 < int(a["accept_len_q"].sum()) < 9 * 8
+    if B >= 9:
+        assert 0 < int(a["accept_len_q"].sum()) < B * K_d
 
 
 def test_host_entry_point_equals_device_entry_point(psd, wl):
