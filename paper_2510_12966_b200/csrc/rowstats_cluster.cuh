@@ -38,6 +38,7 @@ constexpr int kClBWarps = PSD_B_WARPS;             // warps running pass B (the 
 constexpr int kClConsumerWarps = kClAWarps + kClBWarps;
 constexpr int kClConsumers = kClConsumerWarps * 32;
 constexpr int kClThreads = kClConsumers + 96;      // + loader warp + two agent warps
+constexpr int kClThreadsRS = kClThreads + 32;      // the streamed-twice variant has a loader warp per pass
 constexpr int kClHalfBytes = 8192;                 // one model's part of a chunk: 256 threads x 2 x 16 bytes
 constexpr int kClAVec = 16 / kClAWarps;            // 16-byte vectors per lane, chunk and model in pass A
 constexpr int kClBVec = 16 / kClBWarps;            // ... and in pass B
@@ -54,6 +55,8 @@ struct ClusterGeom {
   int chunks;    // chunks per slice
   int ring;      // ring slots in use: min(kClSlots, 3 * chunks - 1), at least chunks + 1
   int n_clusters;
+  int ra;        // 0: a slice stays in the ring from pass A to pass B. > 0 (slice larger than the ring): the
+                 // slice is streamed twice, slots [0, ra) feed pass A and slots [ra, ring) feed pass B
 };
 
 // Per-row constants of pass B: -log2 of the normalisers in the scaled base-2 domain and the clamp floors.
@@ -389,8 +392,11 @@ template <typename V>
 __device__ __forceinline__ V warp_sum(V v) { return warp_reduce<OpSum>(v); }
 
 // ---- the kernel -------------------------------------------------------------------------------------
-template <typename T, int DIV>
-__global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const StageParams P, const ClusterGeom G) {
+// RS = false: a CTA's slice of a row fits the ring and is copied in once. RS = true ("re-stream"): the slice is
+// larger than the ring (small clusters, which is what fills every SM of the device), so it is copied in
+// twice -- once for each pass, the second copy coming out of L2 -- through two rings of their own.
+template <typename T, int DIV, bool RS>
+__global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cluster_kernel(const StageParams P, const ClusterGeom G) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   ClusterCtl* ctl = reinterpret_cast<ClusterCtl*>(ring + static_cast<size_t>(kClSlots) * kClSlotBytes);
@@ -404,10 +410,15 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
   const int slice_begin = static_cast<int>(rank) * G.slice;
   const int slice_len = max(0, min(G.slice, V - slice_begin));   // logits this CTA owns
   const int C = G.chunks, R = G.ring;
+  const int RA = RS ? G.ra : R;        // slots pass A cycles through
+  const int RB0 = RS ? G.ra : 0;       // first slot of pass B
 
   if (tid == 0) {
     ctl->rows_closed = 0;
-    for (int s = 0; s < kClSlots; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], kClBWarps); }
+    for (int s = 0; s < kClSlots; ++s) {
+      mbar_init(&ctl->full[s], 1);
+      mbar_init(&ctl->empty[s], (RS && s < RA) ? kClAWarps : kClBWarps);   // the warps that hand the slot back
+    }
     for (int d = 0; d < kClDepth; ++d) {
       mbar_init(&ctl->a_done[d], kClAWarps);
       mbar_init(&ctl->b_done[d], kClBWarps);
@@ -469,7 +480,8 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
           uint4 us[kClAVec], ul[kClAVec];
 #pragma unroll
           for (int i = 0; i < kClAVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
-          if (++slot == static_cast<unsigned>(R)) { slot = 0; par ^= 1u; }
+          const unsigned used = slot;
+          if (++slot == static_cast<unsigned>(RA)) { slot = 0; par ^= 1u; }
           landed = mbar_test(&ctl->full[slot], par);   // its latency hides behind this chunk's arithmetic
           if (cidx == 0) {
             // the warp's largest logit of its first vectors (the floor keeps rows that start with -inf at 0)
@@ -489,6 +501,10 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
             vs = __fadd2_rn(vs, live ? ps : make_float2(0.f, 0.f));
             vl = __fadd2_rn(vl, live ? pl : make_float2(0.f, 0.f));
           }
+          if (RS) {   // pass A is this slot's only reader: hand it back
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->empty[used]);
+          }
         }
         ls.s = vs.x + vs.y;
         ll.s = vl.x + vl.y;
@@ -497,15 +513,30 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
           ls.s = 0.f; ll.s = 0.f;
           unsigned sl2 = slot0;
           off = 0;
+          // when the slice is streamed twice its chunks have left the ring: take the vectors from global memory
+          const int rows1 = P.B * K;
+          const bool second = w.r >= rows1;
+          const T* gs = (second ? row_ptr<T>(P.small2, P.seq_stride_small2, w.r - rows1, P.K2, V)
+                                : row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V)) + slice_begin;
+          const T* gl = (second ? row_ptr<T>(P.large2, P.seq_stride_large2, w.r - rows1, P.K2, V)
+                                : row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V)) + slice_begin;
 #pragma unroll 1
           for (int cidx = 0; cidx < C; ++cidx, off += CH) {
             const unsigned char* base = my + sl2 * kClSlotBytes;
 #pragma unroll 1
             for (int i = 0; i < kClAVec; ++i) {
-              const bool live = (slice_len - (pw * 32 + lane + i * kClAWarps * 32) * E) > off;
+              const int e = off + (pw * 32 + lane + i * kClAWarps * 32) * E;   // first logit of the vector, in the slice
+              const bool live = e < slice_len;
+              uint4 vs4 = make_uint4(0u, 0u, 0u, 0u), vl4 = vs4;
+              if (RS) {
+                if (live) { vs4 = *reinterpret_cast<const uint4*>(gs + e); vl4 = *reinterpret_cast<const uint4*>(gl + e); }
+              } else {
+                vs4 = lds128(base + i * kVecStride);
+                vl4 = lds128(base + kClHalfBytes + i * kVecStride);
+              }
               // a NaN "reference used" makes the commit take the vector sum afresh
-              lse_commit<T>(0.f, __int_as_float(0x7fc00000), lds128(base + i * kVecStride), live, c, ls);
-              lse_commit<T>(0.f, __int_as_float(0x7fc00000), lds128(base + kClHalfBytes + i * kVecStride), live, c, ll);
+              lse_commit<T>(0.f, __int_as_float(0x7fc00000), vs4, live, c, ls);
+              lse_commit<T>(0.f, __int_as_float(0x7fc00000), vl4, live, c, ll);
             }
             if (++sl2 == static_cast<unsigned>(R)) sl2 = 0;
           }
@@ -513,6 +544,11 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
         // row finished: the warp's partial (one reference, summed S) -> a_part, then tell the agent
         const float ss = warp_reduce<OpSum>(ls.s), sl = warp_reduce<OpSum>(ll.s);
         const int d = w.n % kClDepth;
+        // With a ring of its own pass A could run rows ahead of pass B and of the agents (a resident slice
+        // cannot: its slots come back from pass B). The exchange buffers are kClDepth rows deep, so row n is
+        // handed over only once row n - kClDepth has been released to pass B, which is after the agent has
+        // read that row's partials out of this buffer.
+        if (RS && w.n >= kClDepth) wait_phase(&ctl->b_go[d], ((w.n / kClDepth) - 1) & 1u);
         if (lane == 0) {
           ctl->a_part[d][pw] = make_float4(ls.ref, ss, ll.ref, sl);
           mbar_arrive(&ctl->a_done[d]);
@@ -522,6 +558,8 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
       // ================================ pass B ================================
       constexpr int N = Pairs<T>::kN;
       constexpr int kVecStride = kClBWarps * 32 * 16;   // bytes between a lane's vectors
+      if (RS) slot = static_cast<unsigned>(RB0);
+      bool landed = false;   // as in pass A: the next chunk's barrier is tested one chunk early
       while (w.advance()) {
         const int d = w.n % kClDepth;
         wait_phase(&ctl->b_go[d], (w.n / kClDepth) & 1u);   // the row's constants are published: pass A is through
@@ -530,10 +568,16 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
         acc.reset();
         int off = 0;
         for (int cidx = 0; cidx < C; ++cidx, off += CH) {
+          if (RS && !landed) wait_phase(&ctl->full[slot], par);   // pass B's own copy of the chunk
           const unsigned char* base = my + slot * kClSlotBytes;
           uint4 us[kClBVec], ul[kClBVec];
 #pragma unroll
           for (int i = 0; i < kClBVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+          if (RS) {
+            unsigned nslot = slot + 1u, npar = par;
+            if (nslot == static_cast<unsigned>(R)) { nslot = static_cast<unsigned>(RB0); npar ^= 1u; }
+            landed = mbar_test(&ctl->full[nslot], npar);
+          }
 #pragma unroll
           for (int i = 0; i < kClBVec; ++i) {
             float2 xs[N], xl[N];
@@ -551,7 +595,7 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&ctl->empty[slot]);   // this warp is done with the slot
-          if (++slot == static_cast<unsigned>(R)) slot = 0;
+          if (++slot == static_cast<unsigned>(R)) { slot = static_cast<unsigned>(RB0); par ^= 1u; }
         }
         const float js = warp_reduce<OpSum>(acc.js.x + acc.js.y);
         const float big = warp_reduce<OpSum>(acc.big.x + acc.big.y);
@@ -562,38 +606,50 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
         }
       }
     }
-  } else if (warp == kClConsumerWarps) {
+  } else if (warp == kClConsumerWarps || warp == kClConsumerWarps + 3) {
     // ================================ loader ================================
+    // One thread per ring: the whole ring, or (slice streamed twice) pass A's slots [0, RA) from this warp and
+    // pass B's slots [RA, R) from the last warp. The two streams run freely; pass B's copy of a chunk is
+    // asked for about one row slice after pass A's and is served by L2.
+    const bool for_b = warp != kClConsumerWarps;
+    const unsigned lo = for_b ? static_cast<unsigned>(RB0) : 0u, hi = static_cast<unsigned>(for_b ? R : RA);
     if (lane == 0) {
       RowWalk w;
       w.init(P, cluster_id, G.n_clusters);
-      unsigned slot = 0, fills = 0;   // ring position; how often the ring has wrapped
+      const int rows1 = P.B * K;
+      auto row_small = [&](int r) {
+        return (r >= rows1 ? row_ptr<T>(P.small2, P.seq_stride_small2, r - rows1, P.K2, V)   // second set: stage 2 of the wrapper
+                           : row_ptr<T>(P.small, P.seq_stride_small, r, K, V)) + slice_begin;
+      };
+      auto row_large = [&](int r) {
+        return (r >= rows1 ? row_ptr<T>(P.large2, P.seq_stride_large2, r - rows1, P.K2, V)
+                           : row_ptr<T>(P.large, P.seq_stride_large, r, K, V)) + slice_begin;
+      };
+      // chunk `cidx` of a row slice into `slot`, once the slot's readers of `fills` ring turns ago are through
+      auto fill = [&](const T* rs, const T* rl, int cidx, unsigned slot, unsigned fills) {
+        if (fills > 0) wait_phase(&ctl->empty[slot], (fills - 1u) & 1u);
+        const int e0 = cidx * CH;
+        const int n = min(CH, slice_len - e0);
+        if (n > 0) {
+          const unsigned bytes = static_cast<unsigned>(n) * sizeof(T);
+          unsigned char* dst = ring + static_cast<size_t>(slot) * kClSlotBytes;
+          mbar_arrive_expect_tx(&ctl->full[slot], 2u * bytes);
+          bulk_load(dst, rs + e0, bytes, &ctl->full[slot]);
+          bulk_load(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot]);
+        } else {
+          mbar_arrive(&ctl->full[slot]);   // nothing of this chunk falls into this CTA's slice
+        }
+      };
+      unsigned slot = lo, fills = 0;   // ring position; how often the ring has wrapped
       while (w.advance()) {
-        const int rows1 = P.B * K;
-        const bool second = w.r >= rows1;   // a row of the second set (stage 2 of the two-stage wrapper)
-        const T* rs = (second ? row_ptr<T>(P.small2, P.seq_stride_small2, w.r - rows1, P.K2, V)
-                              : row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V)) + slice_begin;
-        const T* rl = (second ? row_ptr<T>(P.large2, P.seq_stride_large2, w.r - rows1, P.K2, V)
-                              : row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V)) + slice_begin;
+        const T* rs = row_small(w.r);
+        const T* rl = row_large(w.r);
         for (int cidx = 0; cidx < C; ++cidx) {
-          if (fills > 0) {
-            wait_phase(&ctl->empty[slot], (fills - 1u) & 1u);
-          }
-          const int e0 = cidx * CH;
-          const int n = min(CH, slice_len - e0);
-          if (n > 0) {
-            const unsigned bytes = static_cast<unsigned>(n) * sizeof(T);
-            unsigned char* dst = ring + static_cast<size_t>(slot) * kClSlotBytes;
-            mbar_arrive_expect_tx(&ctl->full[slot], 2u * bytes);
-            bulk_load(dst, rs + e0, bytes, &ctl->full[slot]);
-            bulk_load(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot]);
-          } else {
-            mbar_arrive(&ctl->full[slot]);   // nothing of this chunk falls into this CTA's slice
-          }
-          if (++slot == static_cast<unsigned>(R)) { slot = 0; ++fills; }
+          fill(rs, rl, cidx, slot, fills);
+          if (++slot == hi) { slot = lo; ++fills; }
         }
       }
-      // every copy issued above is waited for by pass A of the consumers before they leave
+      // every copy issued above is waited for by its consumers before they leave
     }
   } else {
     // ================================ agent ================================
@@ -743,19 +799,26 @@ __global__ void __launch_bounds__(kClThreads, 1) rowstats_cluster_kernel(const S
 }
 
 // ---- host side --------------------------------------------------------------------------------------
-template <typename T, int DIV>
-inline cudaError_t cluster_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <typename T, int DIV, bool RS>
+inline cudaError_t cluster_prepare_one() {
+  cudaError_t e = cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV, RS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kClSmemBytes));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  return cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV, RS>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+}
+template <typename T, int DIV>
+inline cudaError_t cluster_prepare() {
+  const cudaError_t e = cluster_prepare_one<T, DIV, false>();
+  return e != cudaSuccess ? e : cluster_prepare_one<T, DIV, true>();
 }
 
-template <typename T, int DIV>
-inline int cluster_max_active(int cs) {
+// Co-resident clusters of this size. Both variants of the kernel have the same block size and shared memory;
+// the smaller answer of the two is taken so that one cached figure serves either.
+template <typename T, int DIV, bool RS>
+inline int cluster_max_active_one(int cs) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(cs));
-  cfg.blockDim = dim3(kClThreads);
+  cfg.blockDim = dim3(RS ? kClThreadsRS : kClThreads);
   cfg.dynamicSmemBytes = kClSmemBytes;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
@@ -765,11 +828,15 @@ inline int cluster_max_active(int cs) {
   cfg.attrs = at;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, rowstats_cluster_kernel<T, DIV>, &cfg) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveClusters(&n, rowstats_cluster_kernel<T, DIV, RS>, &cfg) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   return n;
+}
+template <typename T, int DIV>
+inline int cluster_max_active(int cs) {
+  return min(cluster_max_active_one<T, DIV, false>(cs), cluster_max_active_one<T, DIV, true>(cs));
 }
 
 // Per-device cache of the function attributes and of the number of co-resident clusters the device
@@ -848,8 +915,9 @@ inline bool cluster_shape_ok(const StageParams& P, int dtype) {
   return true;
 }
 
-// Picks the cluster size (or takes `forced_cs`), and sizes the grid to the clusters that can be
-// co-resident. Returns false when the shape does not fit the kernel.
+// Picks the cluster size (or takes `forced_cs`; a forced size whose slice exceeds the ring is streamed
+// twice), and sizes the grid to the clusters that can be co-resident. Returns false when the shape does not
+// fit the kernel.
 inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, ClusterGeom* g) {
   if (!cluster_shape_ok(P, dtype)) return false;
   const int es = dtype == 0 ? 4 : 2;
@@ -860,11 +928,14 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
     static const int env_cs = [] { const char* e = std::getenv("PYRAMIDSD_CLUSTER_SIZE"); return e ? std::atoi(e) : 0; }();
     if (env_cs > 0) forced_cs = env_cs;
   }
+  // tuning aid: PYRAMIDSD_RESTREAM=1 takes the streamed-twice variant whenever a cluster size is forced
+  static const int env_rs = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM"); return e ? std::atoi(e) : 0; }();
+  bool restream = false;
   if (forced_cs > 0) {
     if (forced_cs > kClMaxRanks) return false;
     cs = forced_cs;
     cluster_slices(P.V, es, cs, &slice, &chunks);
-    if (chunks > kClSlots - 1) return false;
+    restream = chunks > kClSlots - 1 || env_rs > 0;   // a slice the ring cannot hold is streamed twice
   } else {
     // the smallest cluster whose slice leaves at least five ring slots beyond a row (measured: 4 CTAs for
     // V = 128256 bf16, 5 for V = 152064 bf16); failing that, three slots
@@ -875,13 +946,32 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
         cluster_slices(P.V, es, cs, &slice, &chunks);
         if (chunks <= wanted[pass] && cluster_max_active_any(dtype, P.div_kind, cs) > 0) { found = true; break; }
       }
-    if (!found) return false;
     // few rows: spread each row over more CTAs so that more SMs pull on HBM
     const int sms = cluster_sm_count();
-    while (cs < 8 && chunks >= 2 && rows * cs * 2 <= sms) {
+    while (found && cs < 8 && chunks >= 2 && rows * cs * 2 <= sms) {
       cs *= 2;
       cluster_slices(P.V, es, cs, &slice, &chunks);
     }
+    // Clusters of one or two CTAs are the only ones that fill every SM of the device (larger ones leave SMs
+    // of each GPC over), but for a large vocabulary their slice exceeds the ring and has to be streamed
+    // twice. Estimated time = rounds of co-resident clusters / CTAs per row, the streamed-twice variant
+    // charged for its second copy out of L2 (measured: a few percent for bf16, whose arithmetic is the
+    // limit; about a fifth for fp32, which moves twice the bytes per exponential).
+    auto rounds_per_cta = [&](int c, int n_active) {
+      return static_cast<double>((rows + n_active - 1) / n_active) / c;
+    };
+    double best = found ? rounds_per_cta(cs, cluster_max_active_any(dtype, P.div_kind, cs)) : 1e300;
+    const double second_copy = dtype == 0 ? 1.25 : 1.04;
+    for (int c2 = 2; c2 >= 1; --c2) {
+      int sl2 = 0, ch2 = 0;
+      cluster_slices(P.V, es, c2, &sl2, &ch2);
+      if (ch2 <= wanted[0]) continue;   // fits the ring: the rule above has seen it
+      const int na = cluster_max_active_any(dtype, P.div_kind, c2);
+      if (na <= 0) continue;
+      const double t = second_copy * rounds_per_cta(c2, na);
+      if (t < best) { best = t; cs = c2; slice = sl2; chunks = ch2; restream = true; found = true; }
+    }
+    if (!found) return false;
   }
   const int max_active = cluster_max_active_any(dtype, P.div_kind, cs);
   if (max_active <= 0) return false;
@@ -889,6 +979,12 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
   g->slice = slice;
   g->chunks = chunks;
   g->ring = max(chunks + 1, min(kClSlots, 3 * chunks - 1));
+  g->ra = 0;
+  if (restream) {
+    g->ring = kClSlots;
+    static const int env_ra = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_RA"); return e ? std::atoi(e) : 0; }();
+    g->ra = (env_ra >= 2 && env_ra <= kClSlots - 2) ? env_ra : 5;   // measured: 4 to 8 of the 13 slots for pass A are alike
+  }
   g->n_clusters = static_cast<int>(rows < max_active ? rows : max_active);
   return g->n_clusters > 0;
 }
@@ -897,7 +993,7 @@ template <typename T, int DIV>
 inline cudaError_t cluster_launch_typed(const StageParams& P, const ClusterGeom& g, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(g.n_clusters * g.cs));
-  cfg.blockDim = dim3(kClThreads);
+  cfg.blockDim = dim3(g.ra > 0 ? kClThreadsRS : kClThreads);
   cfg.dynamicSmemBytes = kClSmemBytes;
   cfg.stream = stream;
   cudaLaunchAttribute at[1];
@@ -907,7 +1003,8 @@ inline cudaError_t cluster_launch_typed(const StageParams& P, const ClusterGeom&
   at[0].val.clusterDim.z = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV>, P, g);
+  if (g.ra > 0) return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV, true>, P, g);
+  return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV, false>, P, g);
 }
 
 // Launches the statistics pass with the cluster kernel. Returns 0, or -2 when the launch was refused.

@@ -208,30 +208,24 @@ def test_results_are_bit_identical_run_to_run(psd, wl):
 @pytest.mark.parametrize("V", [2048, 8200, 32000, 128256])
 def test_cluster_kernel_every_cluster_size(psd, oracle, wl, dtype, cs, V):
     """The cluster kernel with the cluster size forced: slices with ragged tails, empty slices (small V
-    over many CTAs), one and several chunks per slice; shapes it cannot hold are refused, not run."""
+    over many CTAs), one and several chunks per slice; a slice of more than 12 chunks does not fit the
+    shared-memory ring and takes the streamed-twice variant (V = 128256 with one or two CTAs)."""
     B, K = 3, 5
     zs, zl, tok = wl.make_stage_inputs(B, K, V, dtype, seed=300 + V + cs, sigma=0.8)
-    dev = torch.device("cuda:0")
-    es = 4 if dtype == "f32" else 2
-    chunks = -(-(-(-V // cs)) // (8192 // es))
-    out = psd.verify_stage_ex(zs.to(dev), zl.to(dev), tok.to(dev), 0.1, kernel_variant=psd.KERNEL_CLUSTER,
-                              cluster_size=cs, raise_on_error=False)
-    if chunks > 12:
-        assert out["status"] == psd.ERR_UNSUPPORTED
-        return
-    assert out["status"] == 0
     for tau in (0.02, 0.3):
         _, _, rep = run_stage_both(psd, oracle, zs, zl, tok, tau, seed=V, offset=cs, variant=psd.KERNEL_CLUSTER,
                                    cluster_size=cs)
         assert rep["tie_div"] + rep["tie_cdf"] <= 1
 
 
-@pytest.mark.parametrize("dtype,V,B,K", [("bf16", 32768, 48, 8), ("f32", 16384, 40, 7), ("bf16", 128256, 24, 16)])
-def test_cluster_kernel_many_rows_per_cluster(psd, oracle, wl, dtype, V, B, K):
-    """More rows than resident clusters: every cluster walks several rows, so the ring, the exchange
-    buffers and the barrier phases wrap around. Also checked against the baseline kernel."""
+@pytest.mark.parametrize("dtype,V,B,K,cs", [("bf16", 32768, 48, 8, 1), ("f32", 16384, 40, 7, 0), ("bf16", 128256, 24, 16, 0),
+                                            ("bf16", 128256, 24, 16, 4), ("bf16", 128256, 40, 16, 2), ("bf16", 128256, 50, 16, 1),
+                                            ("f32", 65536, 60, 7, 1), ("f32", 152064, 24, 8, 2)])
+def test_cluster_kernel_many_rows_per_cluster(psd, oracle, wl, dtype, V, B, K, cs):
+    """More rows than resident clusters: every cluster walks several rows, so the ring(s), the exchange
+    buffers and the barrier phases wrap around -- with the slice resident in the ring and, for the large
+    vocabularies on one or two CTAs, streamed twice. Also checked against the baseline kernel."""
     zs, zl, tok = wl.make_stage_inputs(B, K, V, dtype, seed=400 + B, boost=(4.0, 12.0), sigma=0.7)
-    cs = 1 if V <= 32768 and dtype == "bf16" else 0
     nv = [(3 * b) % (K + 1) for b in range(B)]
     g1, orc, rep = run_stage_both(psd, oracle, zs, zl, tok, 0.15, mode=2, seed=4, offset=9, n_valid=nv,
                                   variant=psd.KERNEL_CLUSTER, cluster_size=cs)
@@ -267,6 +261,65 @@ def test_cluster_kernel_masked_flagged_and_identical_rows(psd, oracle, wl):
     assert gpu["row_flags"][0, 0] == 2 and gpu["next_token"][0] == -2
 
 
+def test_streamed_twice_masked_flagged_and_identical_rows(psd, oracle, wl):
+    """The same edge rows where the slice does not fit the ring (V = 128256 on one or two CTAs): the careful
+    second go of pass A then reads the row from global memory."""
+    B, K, V = 4, 3, 128256
+    zs, zl, tok = wl.make_stage_inputs(B, K, V, "bf16", seed=33, sigma=0.3)
+    zs[0, 1, 100:90000] = -float("inf")          # masked vocabulary across many chunks
+    zl[1, 0, :] = -float("inf")
+    zl[1, 0, 101234] = 2.0                       # a single live token, late in the row
+    zs[2, 1, 99999] = float("nan")
+    zl[3, 0, V - 1] = float("inf")
+    zl[3, 2] = zs[3, 2]                          # bitwise identical pair
+    zs[0, 0, :70000] = -3.0e38                   # huge negative finite logits
+    zl[0, 2, 120000] = 300.0                     # far above the row's first vectors: the optimistic sum overflows
+    for cs in (1, 2):
+        gpu, orc, _ = run_stage_both(psd, oracle, zs, zl, tok, 1.0, variant=psd.KERNEL_CLUSTER, cluster_size=cs)
+        assert gpu["next_token"][2] == -2 and gpu["accept_len"][2] == 1
+        assert gpu["next_token"][3] == -2 and gpu["accept_len"][3] == 0
+        assert gpu["next_token"][1] == 101234 or gpu["accept_len"][1] > 0
+        assert np.all(np.isfinite(gpu["div"][0])) and np.all(np.isfinite(gpu["div"][1]))
+
+
+def test_streamed_twice_equals_resident_bit_for_bit(psd, wl):
+    """PYRAMIDSD_RESTREAM=1 (read when the library first sizes a launch) makes every forced cluster size take
+    the streamed-twice variant, also where the slice would fit the ring. Its arithmetic is the resident
+    variant's, so a fresh process must return the very same bits: one chunk and several per slice, ragged
+    tails, more rows than clusters."""
+    import os, subprocess, sys, tempfile, textwrap
+    cases = [(7, 5, 2048, "f32", 1), (40, 8, 32768, "bf16", 1), (30, 8, 50000, "bf16", 2), (24, 16, 128256, "bf16", 4),
+             (33, 7, 65536, "f32", 8)]
+    code = textwrap.dedent("""
+        import sys, torch
+        sys.path.insert(0, %r)
+        from paper_2510_12966_b200 import binding as psd, workloads as wl
+        dev = torch.device("cuda:0")
+        out = {}
+        for i, (B, K, V, dt, cs) in enumerate(%r):
+            zs, zl, tok = [t.to(dev) for t in wl.make_stage_inputs(B, K, V, dt, seed=500 + i, sigma=0.7)]
+            r = psd.verify_stage_ex(zs, zl, tok, 0.2, 2, 5, 6, kernel_variant=psd.KERNEL_CLUSTER, cluster_size=cs)
+            torch.cuda.synchronize()
+            assert psd.last_status() == 0
+            out[i] = {k: v.cpu() for k, v in r.items() if torch.is_tensor(v)}
+        torch.save(out, sys.argv[1])
+        print("ok")
+    """) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), cases)
+    with tempfile.TemporaryDirectory() as tmp:
+        path = os.path.join(tmp, "streamed.pt")
+        run = subprocess.run([sys.executable, "-c", code, path], env=dict(os.environ, PYRAMIDSD_RESTREAM="1"),
+                             capture_output=True, text=True, timeout=300)
+        assert run.returncode == 0 and "ok" in run.stdout, run.stderr[-2000:]
+        streamed = torch.load(path)
+    dev = torch.device("cuda:0")
+    for i, (B, K, V, dt, cs) in enumerate(cases):
+        zs, zl, tok = [t.to(dev) for t in wl.make_stage_inputs(B, K, V, dt, seed=500 + i, sigma=0.7)]
+        r = psd.verify_stage_ex(zs, zl, tok, 0.2, 2, 5, 6, kernel_variant=psd.KERNEL_CLUSTER, cluster_size=cs)
+        torch.cuda.synchronize()
+        for k, v in streamed[i].items():
+            assert torch.equal(v.view(torch.int32), r[k].cpu().view(torch.int32)), (i, k)
+
+
 @pytest.mark.parametrize("div_kind", [1, 2])
 def test_cluster_kernel_other_divergences(psd, oracle, wl, div_kind):
     zs, zl, tok = wl.make_stage_inputs(4, 4, 20000, "f32", seed=8, sigma=0.5)
@@ -278,10 +331,14 @@ def test_cluster_kernel_other_divergences(psd, oracle, wl, div_kind):
 
 
 def test_cluster_occupancy_query(psd):
-    cs, n = psd.cluster_occupancy(64, 16, 128256, psd.BF16)
-    assert cs == 4 and n >= 16
+    cs, n = psd.cluster_occupancy(64, 16, 128256, psd.BF16)     # many rows: pairs of CTAs fill every SM
+    assert cs == 2 and n >= 64
     cs, n = psd.cluster_occupancy(256, 8, 152064, psd.BF16)
-    assert cs == 5 and n >= 16
+    assert cs == 2 and n >= 64
+    cs, n = psd.cluster_occupancy(16, 16, 128256, psd.BF16)     # fewer rows: the slice stays in shared memory
+    assert cs == 4 and n >= 16
+    cs, n = psd.cluster_occupancy(256, 8, 152064, psd.F32)      # fp32 pays more for the second copy
+    assert cs == 8 and n >= 8
     cs, n = psd.cluster_occupancy(1, 4, 32000, psd.F32)
     assert cs >= 2 and n >= 1
     assert psd.cluster_occupancy(4, 4, 1001, psd.F32) == (0, 0)
