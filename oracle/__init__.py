@@ -39,6 +39,7 @@ def lib():
         _lib = C.CDLL(build())
         _lib.psd_oracle_divergence.restype = C.c_double
         _lib.psd_oracle_residual_mass.restype = C.c_double
+        _lib.psd_oracle_bonus_uniform.restype = C.c_double
     return _lib
 
 
@@ -157,6 +158,50 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
         _ptr(out["window"]), _ptr(out["n_window"]), _ptr(out["div_q"]), _ptr(out["div_t"]), int(n_threads))
     if rc:
         raise ValueError(f"oracle verify rc={rc}")
+    return out
+
+
+def bonus_uniform(seed, offset, b):
+    """The uniform behind sequence b's bonus draw: Philox counter (b, 1, offset_lo, offset_hi), output word 1."""
+    return float(lib().psd_oracle_bonus_uniform(C.c_uint64(seed), C.c_uint64(offset), C.c_uint32(b)))
+
+
+def verify_stage_bonus(logits_small, logits_large_k1, tokens, tau, mode=FUZZY, seed=0, offset=0, n_valid=None,
+                       inv_temperature=1.0, div_kind=JS, n_threads=1, seq_ids=None):
+    """One stage whose larger model supplies K+1 rows per sequence: small [B, K, V], large [B, K+1, V]. When
+    every valid position is accepted, ``next_token`` is drawn from the large model's row after the last
+    valid position (the bonus token) instead of being -1."""
+    s, dt = _as_logits(logits_small)
+    l, dt2 = _as_logits(logits_large_k1)
+    B, K, V = s.shape
+    assert dt == dt2 and l.shape == (B, K + 1, V)
+    t = np.ascontiguousarray(tokens, dtype=np.int32).reshape(B, K)
+    nv = None if n_valid is None else np.ascontiguousarray(n_valid, dtype=np.int32)
+    ids = None if seq_ids is None else np.ascontiguousarray(seq_ids, dtype=np.int32)
+    out = {"accept_len": np.zeros(B, np.int32), "next_token": np.zeros(B, np.int32), "div": np.zeros((B, K))}
+    rc = lib().psd_oracle_verify_stage_bonus(
+        _ptr(s), _ptr(l), _ptr(t), B, K, V, dt, C.c_double(float(tau)), int(mode), C.c_uint64(seed),
+        C.c_uint64(offset), _ptr(nv), C.c_double(inv_temperature), int(div_kind), _ptr(ids),
+        _ptr(out["accept_len"]), _ptr(out["next_token"]), _ptr(out["div"]), int(n_threads))
+    if rc:
+        raise ValueError(f"oracle verify_stage_bonus rc={rc}")
+    return out
+
+
+def verify_bonus(logits_draft, logits_qual, logits_target_k1, draft_tokens, tau_q, tau_t, mode=FUZZY, seed=0,
+                 offset=0, n_threads=1, seq_ids=None):
+    """Two-stage pyramid whose target supplies K_q+1 rows per sequence: stage 1 and the window as in
+    ``verify``; stage 2 is ``verify_stage_bonus`` on the window (Philox offset + 1)."""
+    t, _ = _as_logits(logits_target_k1)
+    q, _ = _as_logits(logits_qual)
+    K_q = t.shape[1] - 1
+    base = verify(logits_draft, logits_qual, np.ascontiguousarray(t[:, :K_q]), draft_tokens, tau_q, tau_t, mode, seed,
+                  offset, n_threads=n_threads, seq_ids=seq_ids)
+    s2 = verify_stage_bonus(np.ascontiguousarray(q[:, :K_q]), t, base["window"], tau_t, mode, seed, offset + 1,
+                            n_valid=base["n_window"], n_threads=n_threads, seq_ids=seq_ids)
+    assert np.array_equal(s2["accept_len"], base["accept_len"])
+    out = dict(base)
+    out["next_token"] = s2["next_token"]
     return out
 
 

@@ -69,6 +69,17 @@ void row_uniforms(uint64_t seed, uint64_t offset, uint32_t r, double* u, double*
   *u2 = (double)(w[1] >> 8) * (1.0 / 16777216.0);
 }
 
+// The uniform that drives a sequence's bonus draw (all positions accepted, Sec. 1: the larger model's next
+// token comes for free). Counter = (b, 1, offset_lo, offset_hi): word 1 = 1 keeps it apart from every row's
+// counter (b*K + k, 0, ...). Same 24-bit mantissa rule, taken from output word 1 like the other draws.
+double bonus_uniform(uint64_t seed, uint64_t offset, uint32_t b) {
+  const uint32_t ctr[4] = {b, 1u, (uint32_t)offset, (uint32_t)(offset >> 32)};
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t w[4];
+  philox4x32_10(ctr, key, w);
+  return (double)(w[1] >> 8) * (1.0 / 16777216.0);
+}
+
 // ---- logits -> double -------------------------------------------------------------------------------
 double logit_at(const void* base, int dtype, size_t idx) {
   if (dtype == DT_F32) return (double)((const float*)base)[idx];
@@ -314,6 +325,44 @@ int psd_oracle_verify_stage(const void* logits_small, const void* logits_large, 
   return verify_stage_impl(a, out_accept_len, out_next_token, out_div, out_p_small_tok, out_p_large_tok,
                            out_resid_mass, out_row_flags, out_accept_bits, n_threads);
 }
+
+// One stage where the larger model supplies K+1 rows per sequence ([B, K+1, V]): row k < K scores the
+// token at position k, and the row after the last valid position is the distribution of the token that
+// follows a fully accepted window (Sec. 1: every accepted run ends with a token of the larger model, the
+// correction on a rejection or this bonus token otherwise). When all n_valid[b] positions are accepted,
+// next_token[b] is drawn from softmax(large[b, n_valid[b], :]) by inverse CDF with the bonus uniform; a
+// bonus row with no distribution (NaN, +inf, no finite entry) gives -2. Everything else is the plain stage.
+int psd_oracle_verify_stage_bonus(const void* logits_small, const void* logits_large_k1, const int32_t* tokens,
+                                  int B, int K, int V, int dtype, double tau, int mode, uint64_t seed,
+                                  uint64_t offset, const int32_t* n_valid, double inv_temperature, int div_kind,
+                                  const int32_t* seq_ids, int32_t* out_accept_len, int32_t* out_next_token,
+                                  double* out_div, int n_threads) {
+  const size_t es = dtype == DT_F32 ? 4 : dtype == DT_BF16 ? 2 : 8;
+  // rows 0..K-1 of every sequence, made dense, are the ordinary stage's large logits
+  std::vector<unsigned char> dense((size_t)B * K * V * es);
+  for (int b = 0; b < B; ++b)
+    std::memcpy(dense.data() + (size_t)b * K * V * es,
+                (const unsigned char*)logits_large_k1 + (size_t)b * (K + 1) * V * es, (size_t)K * V * es);
+  StageArgs a{logits_small, dense.data(), tokens, B, K, V, dtype, V, V,
+              tau, mode, seed, offset, n_valid, inv_temperature, div_kind, seq_ids};
+  const int rc = verify_stage_impl(a, out_accept_len, out_next_token, out_div, nullptr, nullptr, nullptr,
+                                   nullptr, nullptr, n_threads);
+  if (rc) return rc;
+  for (int b = 0; b < B; ++b) {
+    int nv = n_valid ? n_valid[b] : K;
+    if (nv < 0) nv = 0;
+    if (nv > K) nv = K;
+    if (out_accept_len[b] != nv) continue;   // a rejection: the correction token stands
+    std::vector<double> p;
+    const bool ok = softmax_row(logits_large_k1, dtype, ((size_t)b * (K + 1) + nv) * (size_t)V, V, inv_temperature, p);
+    if (!ok) { out_next_token[b] = -2; continue; }
+    const uint32_t b_global = (uint32_t)(seq_ids ? seq_ids[b] : b);
+    out_next_token[b] = inverse_cdf(p, bonus_uniform(seed, offset, b_global));
+  }
+  return 0;
+}
+
+double psd_oracle_bonus_uniform(uint64_t seed, uint64_t offset, uint32_t b) { return bonus_uniform(seed, offset, b); }
 
 // Two-stage pyramid (Fig. 1): stage 1 verifies the K_d draft tokens against the qualifier with tau_q;
 // the accepted prefix plus the qualifier's correction token form the window, cut to K_q; stage 2

@@ -15,10 +15,16 @@
 //
 // Roles: warps 0..7 run pass A, warps 8..15 run pass B (each warp owns 2 x 32 16-byte vectors of every
 // chunk and model; the hardware scheduler interleaves the two instruction streams on each SM
-// sub-partition), warp 16 lane 0 issues the bulk copies, warp 17 is the agent (reduces the warps'
-// partials, talks to the peers; on rank 0 it also writes the row's RowStats). Every wait is bounded: on
-// giving up a thread records PSD_ERR_TIMEOUT in the status word and stops waiting, so the kernel always
-// terminates.
+// sub-partition), warp 16 lane 0 issues the bulk copies, warps 17 and 18 are the agents (they reduce the
+// warps' partials and talk to the peers; on rank 0 the second one also writes the row's RowStats). Every
+// wait is bounded: on giving up a thread records PSD_ERR_TIMEOUT in the status word and stops waiting, so
+// the kernel always terminates.
+//
+// Streamed-twice variant (template flag RS). Clusters of one or two CTAs are the only ones that fill every
+// SM, but for a large vocabulary their slice does not fit the ring. There the slice is copied in twice:
+// part of the ring feeds pass A and is handed back by pass A, the rest feeds pass B, which runs one row
+// behind and gets its copy out of L2; a second loader thread (warp 19) serves pass B's ring. The
+// arithmetic and its order are those of the resident variant.
 #pragma once
 
 #include <cstdlib>
@@ -924,7 +930,7 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
   const long long rows = static_cast<long long>(P.B) * (P.K + P.K2);
   int cs = 0, slice = 0, chunks = 0;
   if (forced_cs <= 0) {
-    // tuning aid: PYRAMIDSD_CLUSTER_SIZE=<power of two> overrides the library's choice for every call
+    // tuning aid: PYRAMIDSD_CLUSTER_SIZE=<1..16> overrides the library's choice for every call
     static const int env_cs = [] { const char* e = std::getenv("PYRAMIDSD_CLUSTER_SIZE"); return e ? std::atoi(e) : 0; }();
     if (env_cs > 0) forced_cs = env_cs;
   }

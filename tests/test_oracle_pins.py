@@ -402,3 +402,93 @@ def test_seq_ids_select_the_philox_rows_of_the_full_batch(oracle):
     part = oracle.verify_stage(zs[pick], zl[pick], tok[pick], 0.0, mode=oracle.STRICT, seed=4, offset=2, seq_ids=pick)
     assert np.array_equal(part["accept_len"], full["accept_len"][pick])
     assert np.array_equal(part["next_token"], full["next_token"][pick])
+
+
+# ---------------------------------------------------------------- bonus token (all positions accepted)
+def test_bonus_uniform_counter_layout(oracle):
+    # counter = (b, 1, offset_lo, offset_hi): word 1 of the counter set apart from every row's (row, 0, ...)
+    seed, offset, b = 0x1122334455667788, 0x99AABBCCDDEEFF00, 5
+    w = oracle.philox4x32_10([b, 1, offset & 0xFFFFFFFF, offset >> 32], [seed & 0xFFFFFFFF, seed >> 32])
+    assert oracle.bonus_uniform(seed, offset, b) == (int(w[1]) >> 8) / 2.0**24
+    assert oracle.bonus_uniform(seed, offset, b) != oracle.row_uniforms(seed, offset, b)[1]
+
+
+def _accepting_case(rng, B, K, V):
+    """Identical small and large rows (divergence exactly 0: fuzzy tau = 0 accepts) + a free bonus row."""
+    zs = rng.normal(size=(B, K, V)).astype(np.float32)
+    zl = np.concatenate([zs, rng.normal(size=(B, 1, V)).astype(np.float32)], axis=1)
+    tok = rng.integers(0, V, size=(B, K)).astype(np.int32)
+    return zs, zl, tok
+
+
+def test_bonus_token_is_the_hot_index_of_the_row_after_the_window(oracle):
+    rng = np.random.default_rng(5)
+    B, K, V = 4, 3, 9
+    zs, zl, tok = _accepting_case(rng, B, K, V)
+    for j in range(K + 1):                       # row j of the large model: one-hot at index j + 2
+        zl[:, j, :] = -np.inf
+        zl[:, j, j + 2] = 1.5
+    zs[:] = zl[:, :K]
+    nv = np.array([0, 1, 2, 3], np.int32)        # the bonus row is the one after the last valid position
+    for offset in range(5):
+        out = oracle.verify_stage_bonus(zs, zl, tok, 0.0, oracle.FUZZY, 3, offset, n_valid=nv)
+        assert np.array_equal(out["accept_len"], nv)
+        assert np.array_equal(out["next_token"], nv + 2)
+
+
+def test_bonus_row_is_ignored_when_a_position_is_rejected(oracle):
+    rng = np.random.default_rng(6)
+    B, K, V = 6, 4, 12
+    zs = rng.normal(size=(B, K, V)).astype(np.float32)
+    zl = rng.normal(size=(B, K + 1, V)).astype(np.float32)
+    tok = rng.integers(0, V, size=(B, K)).astype(np.int32)
+    plain = oracle.verify_stage(zs, np.ascontiguousarray(zl[:, :K]), tok, 0.02, oracle.FUZZY, 1, 2)
+    bonus = oracle.verify_stage_bonus(zs, zl, tok, 0.02, oracle.FUZZY, 1, 2)
+    assert np.all(plain["accept_len"] < K)       # random rows: every sequence has a rejection
+    assert np.array_equal(plain["accept_len"], bonus["accept_len"])
+    assert np.array_equal(plain["next_token"], bonus["next_token"])
+
+
+def test_bonus_tokens_follow_the_large_models_distribution(oracle):
+    rng = np.random.default_rng(7)
+    B, K, V = 30000, 1, 16
+    row = rng.normal(size=V).astype(np.float32)
+    bon = (2.0 * rng.normal(size=V)).astype(np.float32)
+    zs = np.broadcast_to(row, (B, K, V)).copy()
+    zl = np.concatenate([zs, np.broadcast_to(bon, (B, 1, V))], axis=1).copy()
+    tok = np.zeros((B, K), np.int32)
+    out = oracle.verify_stage_bonus(zs, zl, tok, 0.0, oracle.FUZZY, 11, 4, n_threads=4)
+    assert np.all(out["accept_len"] == 1)
+    counts = np.bincount(out["next_token"], minlength=V)
+    p = sp_softmax(bon.astype(np.float64))
+    assert stats.chisquare(counts, p * B).pvalue > 1e-3
+    assert stats.chisquare(counts, sp_softmax(row.astype(np.float64)) * B).pvalue < 1e-6   # not the scoring row's law
+
+
+def test_bonus_row_without_a_distribution_gives_the_invalid_marker(oracle):
+    rng = np.random.default_rng(8)
+    zs, zl, tok = _accepting_case(rng, 3, 2, 8)
+    zl[0, 2, 3] = np.nan
+    zl[1, 2, :] = -np.inf
+    out = oracle.verify_stage_bonus(zs, zl, tok, 0.0, oracle.FUZZY, 0, 0)
+    assert np.array_equal(out["accept_len"], [2, 2, 2])
+    assert out["next_token"][0] == -2 and out["next_token"][1] == -2 and 0 <= out["next_token"][2] < 8
+
+
+def test_pyramid_bonus_composition(oracle):
+    """Two stages with a K_q+1-row target: stage 1, the window and the accept lengths are those of the plain
+    pyramid; only fully accepted windows get a token, drawn from the target's row after the window."""
+    rng = np.random.default_rng(9)
+    B, K_d, K_q, V = 8, 4, 2, 10
+    zq = rng.normal(size=(B, K_d, V)).astype(np.float32)
+    zd = zq.copy()                                   # draft == qualifier: stage 1 accepts everything
+    zt = np.concatenate([zq[:, :K_q], np.full((B, 1, V), -np.inf, np.float32)], axis=1)
+    zt[:, K_q, 7] = 0.0                              # bonus row: one-hot at 7
+    zt[B // 2:, 1] = rng.normal(size=(B - B // 2, V)) * 3   # second half: target disagrees at position 1
+    tok = rng.integers(0, V, size=(B, K_d)).astype(np.int32)
+    plain = oracle.verify(zd, zq, np.ascontiguousarray(zt[:, :K_q]), tok, 0.0, 0.0, oracle.FUZZY, 2, 6)
+    out = oracle.verify_bonus(zd, zq, zt, tok, 0.0, 0.0, oracle.FUZZY, 2, 6)
+    assert np.array_equal(out["accept_len_q"], np.full(B, K_d)) and np.array_equal(out["accept_len"], plain["accept_len"])
+    assert np.all(out["accept_len"][:B // 2] == K_q) and np.all(out["next_token"][:B // 2] == 7)
+    assert np.all(out["accept_len"][B // 2:] == 1)
+    assert np.array_equal(out["next_token"][B // 2:], plain["next_token"][B // 2:])
