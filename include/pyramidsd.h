@@ -106,6 +106,12 @@ typedef struct psd_stage_args {
   int32_t use_stream_field;      /* non-zero: take `stream` even when it is NULL (the legacy default stream) */
   int32_t kernel_variant;        /* psd_kernel_variant */
   int32_t cluster_size;          /* CTAs per cluster for the cluster kernel (1..16); 0 = chosen by the library */
+  int32_t large_has_bonus_row;   /* 1: logits_large is [B, K + 1, V] (seq_stride_large 0 then means (K + 1) * V). Row k < K scores
+                                  * position k as usual. A sequence whose valid positions were ALL accepted gets, instead of -1,
+                                  * a next token drawn from the softmax of the row after its last valid position (row
+                                  * n_valid[b], or K) -- the larger model's own next token, which ends every accepted run
+                                  * (Sec. 1) -- by inverse CDF with the uniform of Philox counter (b, 1, offset_lo, offset_hi),
+                                  * word 1; -2 if that row holds NaN, +inf or no finite logit. */
 } psd_stage_args;
 
 /* One verification stage (Sec. 3.1 for one model pair; Sec. 3.2 applies it twice). Jensen-Shannon
@@ -133,6 +139,16 @@ int pyramidsd_verify(const void* logits_draft, const void* logits_qual, const vo
                      float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
                      int32_t* out_accept_len_q, int32_t* out_next_token_q,
                      int32_t* out_accept_len, int32_t* out_next_token);
+
+/* pyramidsd_verify for a target that supplies one more row: logits_target is [B, K_q + 1, V]. Stage 1, the
+ * window and the accept lengths are those of pyramidsd_verify; a window whose tokens were all accepted by
+ * the target gets its next token from the target's row after the window (see large_has_bonus_row above)
+ * instead of -1, so the caller needs no sampler of its own (Sec. 1, Sec. 3.4). */
+int pyramidsd_verify_bonus(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                           const int32_t* draft_tokens, int B, int K_d, int K_q, int V, psd_dtype dtype,
+                           float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
+                           int32_t* out_accept_len_q, int32_t* out_next_token_q,
+                           int32_t* out_accept_len, int32_t* out_next_token);
 
 /* pyramidsd_verify with HOST pointers for every array: copies the three logits tensors and the tokens
  * to library-owned device staging buffers, runs both stages, copies the four [B] results back and

@@ -21,7 +21,7 @@ KERNEL_AUTO, KERNEL_BASELINE, KERNEL_CLUSTER = 0, 1, 2
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 
 EXPORTS = (
-    "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_host",
+    "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_bonus", "pyramidsd_verify_host",
     "pyramidsd_verify_stage_noalloc", "pyramidsd_verify_fused_lmhead",
     "pyramidsd_model_sd_throughput", "pyramidsd_model_psd_throughput", "pyramidsd_set_two_stage_policy",
     "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
@@ -46,7 +46,7 @@ class StageArgs(C.Structure):
         ("out_resid_mass", C.c_void_p), ("out_row_flags", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("stream", C.c_void_p), ("use_stream_field", C.c_int32), ("kernel_variant", C.c_int32),
-        ("cluster_size", C.c_int32),
+        ("cluster_size", C.c_int32), ("large_has_bonus_row", C.c_int32),
     ]
 
 
@@ -84,6 +84,8 @@ def load_library(path: Optional[str] = None):
     lib.pyramidsd_verify_stage_ex.restype = i32
     pyr = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, u64, u64, vp, vp, vp, vp]
     lib.pyramidsd_verify.argtypes = pyr
+    lib.pyramidsd_verify_bonus.restype = C.c_int
+    lib.pyramidsd_verify_bonus.argtypes = pyr
     lib.pyramidsd_verify.restype = i32
     lib.pyramidsd_verify_host.argtypes = pyr
     lib.pyramidsd_verify_host.restype = i32
@@ -279,10 +281,12 @@ def verify_stage_noalloc(logits_small, logits_large, draft_tokens, threshold, mo
 def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
                     B=None, K=None, V=None, n_valid=None, inv_temperature=0.0, div_kind=DIV_JS,
                     seq_stride_small=0, seq_stride_large=0, want_rows=True, workspace=None, stream=None,
-                    kernel_variant=KERNEL_AUTO, cluster_size=0, raise_on_error=True):
-    """``pyramidsd_verify_stage_ex``: every option exposed. Returns a dict of device tensors (+ "status")."""
+                    kernel_variant=KERNEL_AUTO, cluster_size=0, raise_on_error=True, large_has_bonus_row=False):
+    """``pyramidsd_verify_stage_ex``: every option exposed. Returns a dict of device tensors (+ "status").
+    With ``large_has_bonus_row`` the large logits are [B, K + 1, V]."""
     if B is None:
         B, K, V = logits_small.shape
+        assert tuple(logits_large.shape) == (B, K + (1 if large_has_bonus_row else 0), V)
     dt = dtype_code(logits_small)
     dev = logits_small.device
     out = {"accept_len": torch.empty(B, dtype=torch.int32, device=dev),
@@ -319,6 +323,7 @@ def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, p
     a.use_stream_field = 1
     a.kernel_variant = int(kernel_variant)
     a.cluster_size = int(cluster_size)
+    a.large_has_bonus_row = 1 if large_has_bonus_row else 0
     rc = load_library().pyramidsd_verify_stage_ex(C.byref(a))
     out["status"] = rc
     if raise_on_error:
@@ -344,6 +349,28 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
         out["accept_len_q"].data_ptr(), out["next_token_q"].data_ptr(),
         out["accept_len"].data_ptr(), out["next_token"].data_ptr())
     _check(rc, "pyramidsd_verify")
+    return out
+
+
+def verify_bonus(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode=FUZZY, philox_seed=0,
+                 offset=0, out=None):
+    """``pyramidsd_verify_bonus``: the two-stage pyramid with a target of K_q + 1 rows per sequence
+    (``logits_target`` [B, K_q + 1, V]); fully accepted windows get the target's bonus token."""
+    B, K_d, V = logits_draft.shape
+    K_q = logits_target.shape[1] - 1
+    dt = dtype_code(logits_draft)
+    assert logits_qual.shape == logits_draft.shape and logits_target.shape == (B, K_q + 1, V)
+    dev = logits_draft.device
+    if out is None:
+        out = {k: torch.empty(B, dtype=torch.int32, device=dev)
+               for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+    rc = load_library().pyramidsd_verify_bonus(
+        _dev_ptr(logits_draft, name="logits_draft"), _dev_ptr(logits_qual, name="logits_qual"),
+        _dev_ptr(logits_target, name="logits_target"), _dev_ptr(draft_tokens, torch.int32, "draft_tokens"),
+        B, K_d, K_q, V, dt, float(tau_q), float(tau_t), int(mode), int(philox_seed), int(offset),
+        out["accept_len_q"].data_ptr(), out["next_token_q"].data_ptr(),
+        out["accept_len"].data_ptr(), out["next_token"].data_ptr())
+    _check(rc, "pyramidsd_verify_bonus")
     return out
 
 

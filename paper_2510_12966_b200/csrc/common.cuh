@@ -61,6 +61,9 @@ struct StageParams {
   long long seq_stride_small2, seq_stride_large2;
   int K2;
   RowStats* stats2;
+  // 1: the large tensor holds K + 1 rows per sequence; a sequence whose valid positions were all accepted
+  // gets its next token from the row after the last valid one (the larger model's bonus token, Sec. 1).
+  int bonus;
 };
 
 // ---- special functions (single MUFU instruction each) -------------------------------------------------
@@ -169,6 +172,14 @@ __device__ __forceinline__ void row_uniforms(unsigned long long seed, unsigned l
                                 make_uint2(static_cast<unsigned>(seed), static_cast<unsigned>(seed >> 32)));
   *u = static_cast<float>(w.x >> 8) * (1.0f / 16777216.0f);
   *u2 = static_cast<float>(w.y >> 8) * (1.0f / 16777216.0f);
+}
+
+// The uniform behind a sequence's bonus draw: counter (b, 1, offset_lo, offset_hi), output word 1; word 1 of
+// the counter keeps it apart from every row's (r, 0, ...).
+__device__ __forceinline__ float bonus_uniform(unsigned long long seed, unsigned long long offset, unsigned b) {
+  const uint4 w = philox4x32_10(make_uint4(b, 1u, static_cast<unsigned>(offset), static_cast<unsigned>(offset >> 32)),
+                                make_uint2(static_cast<unsigned>(seed), static_cast<unsigned>(seed >> 32)));
+  return static_cast<float>(w.y >> 8) * (1.0f / 16777216.0f);
 }
 
 }  // namespace psd

@@ -165,11 +165,56 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
     if (sh_flags & (kFlagSmallNonfinite | kFlagLargeNonfinite)) next = -2;  // no distribution to draw from
     else need_draw = true;
   }
+  const bool bonus = P.bonus && L == sh_nv;   // everything accepted: the larger model's next token comes for free
+  if (bonus) {
+    // The row after the window was not part of the statistics pass: every CTA takes its normaliser here, with
+    // the same two passes and reduction trees (so all CTAs of a cluster hold the same bits).
+    const T* brow = large_seq + static_cast<long long>(L) * V;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(brow) & 15u) == 0 && (V % Elem<T>::kPerVec) == 0;
+    constexpr int E = Elem<T>::kPerVec;
+    float mx = -INFINITY;
+    if (vec_ok) {
+      for (int v = tid; v < V / E; v += kFinThreads) {
+        float x[E];
+        Elem<T>::unpack(ldg_vec(brow, v), x);
+#pragma unroll
+        for (int j = 0; j < E; ++j) mx = max_nan(mx, x[j]);
+      }
+    } else {
+      for (int i = tid; i < V; i += kFinThreads) mx = max_nan(mx, Elem<T>::load(brow, i));
+    }
+    mx = block_reduce<OpMaxNan>(mx, warp_total, -INFINITY);
+    if (!(fabsf(mx) < INFINITY)) {
+      next = -2;   // NaN, +inf or no finite logit: no distribution to draw from
+    } else {
+      const float m2 = mx * P.c;
+      float sum = 0.f;
+      if (vec_ok) {
+        for (int v = tid; v < V / E; v += kFinThreads) {
+          float x[E];
+          Elem<T>::unpack(ldg_vec(brow, v), x);
+#pragma unroll
+          for (int j = 0; j < E; ++j) sum += ex2_approx(fmaf(x[j], P.c, -m2));
+        }
+      } else {
+        for (int i = tid; i < V; i += kFinThreads) sum += ex2_approx(fmaf(Elem<T>::load(brow, i), P.c, -m2));
+      }
+      sum = block_reduce<OpSum>(sum, warp_total, 0.f);
+      if (tid == 0) {
+        sh_m2l = m2; sh_l2sl = lg2_approx(sum);
+        sh_m2s = m2; sh_l2ss = sh_l2sl;
+        sh_resid = 0.f;   // weights are p_large itself
+        sh_u2 = bonus_uniform(P.seed, P.offset, static_cast<unsigned>(b));
+      }
+      __syncthreads();
+      need_draw = true;
+    }
+  }
 
   if (need_draw) {  // uniform across the CTA
     RowView<T> row;
     row.large = large_seq + static_cast<long long>(L) * V;
-    row.small = small_seq + static_cast<long long>(L) * V;
+    row.small = bonus ? row.large : small_seq + static_cast<long long>(L) * V;   // the bonus row has no small partner
     row.V = V;
     row.vec_ok = ((reinterpret_cast<uintptr_t>(row.large) | reinterpret_cast<uintptr_t>(row.small)) & 15u) == 0 &&
                  (V % Elem<T>::kPerVec) == 0;

@@ -245,8 +245,10 @@ int validate_stage(const psd_stage_args* a) {
     if (a->K > 0 && (!a->logits_small || !a->logits_large || !a->tokens)) return PSD_ERR_INVALID_ARG;
     const long long min_stride = static_cast<long long>(a->K) * a->V;
     if (a->seq_stride_small != 0 && a->seq_stride_small < min_stride) return PSD_ERR_INVALID_ARG;
-    if (a->seq_stride_large != 0 && a->seq_stride_large < min_stride) return PSD_ERR_INVALID_ARG;
+    if (a->seq_stride_large != 0 && a->seq_stride_large < min_stride + (a->large_has_bonus_row ? a->V : 0)) return PSD_ERR_INVALID_ARG;
+    if (a->large_has_bonus_row && !a->logits_large) return PSD_ERR_INVALID_ARG;
   }
+  if (a->large_has_bonus_row != 0 && a->large_has_bonus_row != 1) return PSD_ERR_INVALID_ARG;
   if (a->workspace != nullptr) {
     if ((reinterpret_cast<uintptr_t>(a->workspace) % kAlign) != 0) return PSD_ERR_WORKSPACE;
     if (a->workspace_bytes < stage_workspace_bytes(a->B, a->K)) return PSD_ERR_WORKSPACE;
@@ -263,7 +265,8 @@ StageParams make_params(const psd_stage_args* a, void* ws, int* status) {
   P.B = a->B; P.K = a->K; P.V = a->V;
   const long long dense = static_cast<long long>(a->K) * a->V;
   P.seq_stride_small = a->seq_stride_small ? a->seq_stride_small : dense;
-  P.seq_stride_large = a->seq_stride_large ? a->seq_stride_large : dense;
+  P.seq_stride_large = a->seq_stride_large ? a->seq_stride_large : dense + (a->large_has_bonus_row ? a->V : 0);
+  P.bonus = a->large_has_bonus_row;
   const double invT = a->inv_temperature > 0.f ? static_cast<double>(a->inv_temperature) : 1.0;
   P.c = static_cast<float>(1.4426950408889634 * invT);
   P.threshold = a->threshold;
@@ -327,7 +330,7 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
                      const int32_t* draft_tokens, int B, int K_d, int K_q, int V, int dtype, float tau_q,
                      float tau_t, int mode, uint64_t seed, uint64_t offset, int32_t* out_accept_len_q,
                      int32_t* out_next_token_q, int32_t* out_accept_len, int32_t* out_next_token,
-                     cudaStream_t stream, int variant) {
+                     cudaStream_t stream, int variant, bool bonus = false) {
   if (K_q < 1 || K_d < K_q || K_d > 32 || B < 0 || V < 1) return PSD_ERR_INVALID_ARG;
   if (B == 0) return PSD_OK;
   DeviceState* ds = nullptr;
@@ -370,6 +373,7 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   s2.logits_large = logits_target;
   s2.seq_stride_small = static_cast<int64_t>(K_d) * V;  // rows 0..K_q-1 of each [K_d, V] qualifier sequence
   s2.seq_stride_large = 0;
+  s2.large_has_bonus_row = bonus ? 1 : 0;   // target [B, K_q + 1, V]: its last row per sequence is the bonus row
   s2.tokens = window;
   s2.n_valid = n_window;
   s2.K = K_q;
@@ -481,6 +485,20 @@ int pyramidsd_verify(const void* logits_draft, const void* logits_qual, const vo
   return verify_two_stage(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype, tau_q,
                           tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q, out_accept_len,
                           out_next_token, t_stream, PSD_KERNEL_AUTO);
+}
+
+int pyramidsd_verify_bonus(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                           const int32_t* draft_tokens, int B, int K_d, int K_q, int V, psd_dtype dtype,
+                           float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
+                           int32_t* out_accept_len_q, int32_t* out_next_token_q, int32_t* out_accept_len,
+                           int32_t* out_next_token) {
+  if (!valid_dtype(dtype) || !valid_mode(mode)) return PSD_ERR_INVALID_ARG;
+  if (B > 0 && (!logits_draft || !logits_qual || !logits_target || !draft_tokens || !out_accept_len_q ||
+                !out_next_token_q || !out_accept_len || !out_next_token))
+    return PSD_ERR_INVALID_ARG;
+  return verify_two_stage(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype, tau_q,
+                          tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q, out_accept_len,
+                          out_next_token, t_stream, PSD_KERNEL_AUTO, true);
 }
 
 int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, const void* logits_target,
