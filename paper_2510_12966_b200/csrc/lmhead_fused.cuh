@@ -182,7 +182,7 @@ __device__ __forceinline__ void lm_epilogue_tile(unsigned tacc, int n0, bool row
             const float E = ex2_approx(fmaxf(a, b));
             const float dd = a - b;
             const float u = ex2_approx(-fabsf(dd));
-            const float2 ps = psi_poly(make_float2(u, u));
+            const float2 ps = psi_poly<7>(make_float2(u, u));
             js = fmaf(E, fmaf(u, -fabsf(dd), ps.x), js);
             big += E;
             const float lo = E * u;                       // min(p, q)
