@@ -239,6 +239,14 @@ def run_ours(args):
                          "share_of_step": (ms_rs / ms_total) if ms_total > 0 else None},
             "gpu_launches": launches_all, "clocks": clocks,
         }
+        # The same kernel against the special-function unit, its first ceiling with bf16 logits: four ex2 per
+        # index pair (two per pass), 16 results per clock and SM, 148 SMs at the sampled SM clock.
+        n_ex2 = 4.0 * rs_bytes / (2 * es)
+        xu_peak = 16.0 * 148 * (clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0) * 1e6
+        line["roofline"]["special_function_unit"] = {
+            "achieved": n_ex2 / (ms_rs * 1e-3) if ms_rs > 0 else 0.0, "peak": xu_peak, "unit": "ex2/s",
+            "frac": (n_ex2 / (ms_rs * 1e-3) / xu_peak) if ms_rs > 0 else 0.0,
+            "peak_kind": "16 results/clk/SM (measured) x 148 SMs x sampled SM clock"}
         if e2e:
             line["e2e"] = {"value": e2e_pos_all / (e2e["ms"] * 1e-3), "unit": UNIT,
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
