@@ -97,6 +97,36 @@ def workload_from_name(name: str):
     return cfg, workloads.CONFIGS[cfg]
 
 
+def graph_replay_us_per_step(binding, step, steps_in_graph=16, replays=50):
+    """The same calls replayed from a CUDA graph: device time per step with the host's launch path taken out.
+    For the single-stream workloads, whose step is a few launches of a few microseconds each."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    try:
+        with torch.cuda.stream(side):
+            binding.set_stream()
+            step(0)
+            step(1)
+            side.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                binding.set_stream()
+                for i in range(steps_in_graph):
+                    step(i)
+    finally:
+        binding.set_stream()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (replays * steps_in_graph) * 1e3
+
+
 def positions_per_step(w, out) -> int:
     """Rows actually verified: every stage-1 row, and stage-2 rows inside each sequence's window."""
     al_q, nt_q = out["accept_len_q"], out["next_token_q"]
@@ -169,6 +199,7 @@ def run_ours(args):
     status = binding.last_status()
     if status != 0:
         raise SystemExit(f"bench.py: library status {status}")
+    graph_us = graph_replay_us_per_step(binding, step) if (world == 1 and w.B <= 4) else None
 
     # positions and algorithmic bytes of the steps that were timed
     pos_by_buf = [positions_per_step(w, o) for o in outs]
@@ -247,6 +278,8 @@ def run_ours(args):
             "achieved": n_ex2 / (ms_rs * 1e-3) if ms_rs > 0 else 0.0, "peak": xu_peak, "unit": "ex2/s",
             "frac": (n_ex2 / (ms_rs * 1e-3) / xu_peak) if ms_rs > 0 else 0.0,
             "peak_kind": "16 results/clk/SM (measured) x 148 SMs x sampled SM clock"}
+        if graph_us is not None:
+            line["config"]["us_per_step_cuda_graph_replay"] = graph_us
         if e2e:
             line["e2e"] = {"value": e2e_pos_all / (e2e["ms"] * 1e-3), "unit": UNIT,
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
@@ -301,6 +334,7 @@ def run_single_stage(args):
     ms_rs, n_rs, ms_fin, n_fin = binding.kernel_timing_end()
     launches = binding.launch_count() - launches0
     clocks = sampler.stop()
+    graph_us = graph_replay_us_per_step(binding, step, steps_in_graph=64)
     peaks, peak_kind = load_peaks()
     pos = 2 * w.B * w.K_d * args.steps
     row_bytes = 2 * w.V * 4
@@ -311,7 +345,7 @@ def run_single_stage(args):
         "data": "synthetic",
         "config": {"workload": f"{w.name}: B=1, K=4, V=32000, fp32 logits, one fuzzy (tau=0.3) and one strict call per step, 64 rounds",
                    "l2_policy": "64 rounds of 1 MB stay in L2: this is a latency figure, not a bandwidth one",
-                   "us_per_call": ms_total / args.steps / 2 * 1e3},
+                   "us_per_call": ms_total / args.steps / 2 * 1e3, "us_per_call_cuda_graph_replay": graph_us / 2},
         "roofline": {"bound": "hbm", "kernel": "rowstats (4 row pairs per launch: launch-latency-bound)", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                      "traffic": None, "launches": n_rs, "avg_launch_ms": ms_rs / max(n_rs, 1),
