@@ -22,7 +22,9 @@
  *     aligned with V * sizeof(element) a multiple of 16 take the vector path; other shapes take a
  *     scalar path — never an error. -inf logits are legal (probability 0). A row holding NaN or +inf,
  *     or no finite entry, or a token outside [0, V), is flagged and rejected; a flagged non-finite row
- *     at the first rejection emits token -2.
+ *     at the first rejection emits token -2. Finite logits are meant to be of ordinary size: beyond about
+ *     1e9 in magnitude the product with log2(e)/T is rounded by more than the exponent range of a float and
+ *     the row may be flagged as if it were not finite.
  *   - out_accept_len[b] in [0, n_valid[b]]; out_next_token[b] = resampled token at the first rejection,
  *     or -1 when every valid position was accepted.
  *   - Work is enqueued on the stream set by pyramidsd_set_stream (default: the legacy default stream)
@@ -73,7 +75,8 @@ typedef enum {
 typedef enum {
   PSD_KERNEL_AUTO = 0,
   PSD_KERNEL_BASELINE = 1, /* one CTA per row, three passes over global memory */
-  PSD_KERNEL_CLUSTER = 2   /* one thread-block cluster per row, row pair resident in shared memory */
+  PSD_KERNEL_CLUSTER = 2   /* one thread-block cluster per row pair; its slices sit in the CTAs' shared memory for both passes, or,
+                            * for clusters of 1 or 2 CTAs on a large vocabulary, are copied in once per pass (second copy from L2) */
 } psd_kernel_variant;
 
 /* Extended single-stage arguments. Zero-initialise, set struct_size = sizeof(psd_stage_args), fill what
@@ -105,7 +108,8 @@ typedef struct psd_stage_args {
   void* stream;                  /* cudaStream_t, or NULL for the stream set by pyramidsd_set_stream */
   int32_t use_stream_field;      /* non-zero: take `stream` even when it is NULL (the legacy default stream) */
   int32_t kernel_variant;        /* psd_kernel_variant */
-  int32_t cluster_size;          /* CTAs per cluster for the cluster kernel (1..16); 0 = chosen by the library */
+  int32_t cluster_size;          /* CTAs per cluster for the cluster kernel (1..16); 0 = chosen by the library. Results are
+                                  * bit-identical run to run for a given size; different sizes differ in the last bits */
   int32_t large_has_bonus_row;   /* 1: logits_large is [B, K + 1, V] (seq_stride_large 0 then means (K + 1) * V). Row k < K scores
                                   * position k as usual. A sequence whose valid positions were ALL accepted gets, instead of -1,
                                   * a next token drawn from the softmax of the row after its last valid position (row
