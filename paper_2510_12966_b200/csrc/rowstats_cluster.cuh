@@ -984,23 +984,28 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
       cs *= 2;
       cluster_slices(P.V, es, cs, &slice, &chunks);
     }
-    // Clusters of one or two CTAs are the only ones that fill every SM of the device (larger ones leave SMs
-    // of each GPC over), but for a large vocabulary their slice exceeds the ring and has to be streamed
-    // twice. Estimated time = rounds of co-resident clusters / CTAs per row, the streamed-twice variant
-    // charged for its second copy out of L2 (measured: a few percent for bf16, whose arithmetic is the
-    // limit; about a fifth for fp32, which moves twice the bytes per exponential).
+    // Small clusters fill more SMs (148 with one or two CTAs, 135 with three, 132 with four on B200; eight
+    // CTAs place only 120), but for a large vocabulary their slice exceeds the ring and has to be streamed
+    // twice. Estimated time = rounds of co-resident clusters / CTAs per row, times a measured factor:
+    //   resident: 1 + 0.01 per CTA of the cluster (the per-row exchange);
+    //   streamed twice: 1.04 for bf16 (4 % at equal SM count), 1.0 for fp32 (there the wider ring lookahead
+    //   outweighs the second copy), plus up to 0.3 once the bytes between a chunk's first and second copy --
+    //   one slice pair per CTA in flight -- outgrow what L2 keeps (48 MB and up: measured 1.04 at 55 MB,
+    //   1.25 at 90 MB).
     auto rounds_per_cta = [&](int c, int n_active) {
       return static_cast<double>((rows + n_active - 1) / n_active) / c;
     };
-    double best = found ? rounds_per_cta(cs, cluster_max_active_any(dtype, P.div_kind, cs)) : 1e300;
-    const double second_copy = dtype == 0 ? 1.25 : 1.04;
-    for (int c2 = 2; c2 >= 1; --c2) {
+    double best = found ? (1.0 + 0.01 * cs) * rounds_per_cta(cs, cluster_max_active_any(dtype, P.div_kind, cs)) : 1e300;
+    for (int c2 = 8; c2 >= 1; --c2) {
       int sl2 = 0, ch2 = 0;
       cluster_slices(P.V, es, c2, &sl2, &ch2);
-      if (ch2 <= wanted[0]) continue;   // fits the ring: the rule above has seen it
+      if (ch2 <= wanted[0]) continue;   // fits the ring with room to spare: the rule above has seen it
       const int na = cluster_max_active_any(dtype, P.div_kind, c2);
       if (na <= 0) continue;
-      const double t = second_copy * rounds_per_cta(c2, na);
+      const double in_flight_mb = 2.0 * sl2 * es * static_cast<double>(na < rows ? na : rows) * c2 / 1048576.0;
+      double factor = dtype == 0 ? 1.0 : 1.04;
+      if (in_flight_mb > 48.0) factor += 0.3 * ((in_flight_mb - 48.0) / 48.0 < 1.0 ? (in_flight_mb - 48.0) / 48.0 : 1.0);
+      const double t = factor * rounds_per_cta(c2, na);
       if (t < best) { best = t; cs = c2; slice = sl2; chunks = ch2; restream = true; found = true; }
     }
     if (!found) return false;

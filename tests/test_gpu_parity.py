@@ -337,8 +337,8 @@ def test_cluster_occupancy_query(psd):
     assert cs == 2 and n >= 64
     cs, n = psd.cluster_occupancy(16, 16, 128256, psd.BF16)     # fewer rows: the slice stays in shared memory
     assert cs == 4 and n >= 16
-    cs, n = psd.cluster_occupancy(256, 8, 152064, psd.F32)      # fp32 pays more for the second copy
-    assert cs == 8 and n >= 8
+    cs, n = psd.cluster_occupancy(256, 8, 152064, psd.F32)      # fp32: streamed twice on clusters that fill 130+ SMs
+    assert cs in (4, 5, 6) and n >= 20
     cs, n = psd.cluster_occupancy(1, 4, 32000, psd.F32)
     assert cs >= 2 and n >= 1
     assert psd.cluster_occupancy(4, 4, 1001, psd.F32) == (0, 0)
