@@ -62,7 +62,8 @@ struct ClusterGeom {
   int ring;      // ring slots in use: min(kClSlots, 3 * chunks - 1), at least chunks + 1
   int n_clusters;
   int ra;        // 0: a slice stays in the ring from pass A to pass B. > 0 (slice larger than the ring): the
-                 // slice is streamed twice, slots [0, ra) feed pass A and slots [ra, ring) feed pass B
+                 // slice is streamed twice through slots of two chunks each, slots [0, ra) feed pass A and
+                 // slots [ra, ring) feed pass B
 };
 
 // Per-row constants of pass B: -log2 of the normalisers in the scaled base-2 domain and the clamp floors.
@@ -444,6 +445,11 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
   const int C = G.chunks, R = G.ring;
   const int RA = RS ? G.ra : R;        // slots pass A cycles through
   const int RB0 = RS ? G.ra : 0;       // first slot of pass B
+  // The streamed-twice variant moves two chunks per barrier (a slot of 2 x 16 KB): its rings need no chunk
+  // granularity to hold a row, and every hand-off costs the two instruction streams issue slots.
+  constexpr int SUB = RS ? 2 : 1;
+  constexpr int kSlotStride = SUB * kClSlotBytes;
+  const int CS = (C + SUB - 1) / SUB;  // barrier steps per row slice
 
   if (tid == 0) {
     ctl->rows_closed = 0;
@@ -506,32 +512,36 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         const unsigned slot0 = slot;   // where the row starts in the ring
         float2 vs = make_float2(0.f, 0.f), vl = vs;
         int off = 0;   // chunk offset inside the slice, in logits
-        for (int cidx = 0; cidx < C; ++cidx, off += CH) {
+        for (int step = 0; step < CS; ++step) {
           if (!landed) wait_phase(&ctl->full[slot], par);
-          const unsigned char* base = my + slot * kClSlotBytes;
-          uint4 us[kClAVec], ul[kClAVec];
-#pragma unroll
-          for (int i = 0; i < kClAVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+          const unsigned char* sbase = my + slot * kSlotStride;
           const unsigned used = slot;
           if (++slot == static_cast<unsigned>(RA)) { slot = 0; par ^= 1u; }
-          landed = mbar_test(&ctl->full[slot], par);   // its latency hides behind this chunk's arithmetic
-          if (cidx == 0) {
-            // the warp's largest logit of its first vectors (the floor keeps rows that start with -inf at 0)
-            float gs = vector_max<T>(us[0], len[0] > 0), gl = vector_max<T>(ul[0], len[0] > 0);
+          landed = mbar_test(&ctl->full[slot], par);   // its latency hides behind this step's arithmetic
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              gs = fmaxf(gs, __shfl_xor_sync(0xffffffffu, gs, o));
-              gl = fmaxf(gl, __shfl_xor_sync(0xffffffffu, gl, o));
+          for (int sub = 0; sub < SUB; ++sub, off += CH) {   // a chunk beyond the slice (odd count) has no live vector
+            const unsigned char* base = sbase + sub * kClSlotBytes;
+            uint4 us[kClAVec], ul[kClAVec];
+#pragma unroll
+            for (int i = 0; i < kClAVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+            if (step == 0 && sub == 0) {
+              // the warp's largest logit of its first vectors (the floor keeps rows that start with -inf at 0)
+              float gs = vector_max<T>(us[0], len[0] > 0), gl = vector_max<T>(ul[0], len[0] > 0);
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) {
+                gs = fmaxf(gs, __shfl_xor_sync(0xffffffffu, gs, o));
+                gl = fmaxf(gl, __shfl_xor_sync(0xffffffffu, gl, o));
+              }
+              ls.ref = fmaxf(gs * c, -1e30f);
+              ll.ref = fmaxf(gl * c, -1e30f);
             }
-            ls.ref = fmaxf(gs * c, -1e30f);
-            ll.ref = fmaxf(gl * c, -1e30f);
-          }
 #pragma unroll
-          for (int i = 0; i < kClAVec; ++i) {
-            const float2 ps = lse_vector_sum2<T>(us[i], c, ls.ref), pl = lse_vector_sum2<T>(ul[i], c, ll.ref);
-            const bool live = len[i] > off;
-            vs = __fadd2_rn(vs, live ? ps : make_float2(0.f, 0.f));
-            vl = __fadd2_rn(vl, live ? pl : make_float2(0.f, 0.f));
+            for (int i = 0; i < kClAVec; ++i) {
+              const float2 ps = lse_vector_sum2<T>(us[i], c, ls.ref), pl = lse_vector_sum2<T>(ul[i], c, ll.ref);
+              const bool live = len[i] > off;
+              vs = __fadd2_rn(vs, live ? ps : make_float2(0.f, 0.f));
+              vl = __fadd2_rn(vl, live ? pl : make_float2(0.f, 0.f));
+            }
           }
           if (RS) {   // pass A is this slot's only reader: hand it back
             __syncwarp();
@@ -599,30 +609,34 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         DivAcc acc;
         acc.reset();
         int off = 0;
-        for (int cidx = 0; cidx < C; ++cidx, off += CH) {
-          if (RS && !landed) wait_phase(&ctl->full[slot], par);   // pass B's own copy of the chunk
-          const unsigned char* base = my + slot * kClSlotBytes;
-          uint4 us[kClBVec], ul[kClBVec];
-#pragma unroll
-          for (int i = 0; i < kClBVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+        for (int step = 0; step < CS; ++step) {
+          if (RS && !landed) wait_phase(&ctl->full[slot], par);   // pass B's own copy of the chunks
+          const unsigned char* sbase = my + slot * kSlotStride;
           if (RS) {
             unsigned nslot = slot + 1u, npar = par;
             if (nslot == static_cast<unsigned>(R)) { nslot = static_cast<unsigned>(RB0); npar ^= 1u; }
             landed = mbar_test(&ctl->full[nslot], npar);
           }
 #pragma unroll
-          for (int i = 0; i < kClBVec; ++i) {
-            float2 xs[N], xl[N];
-            Pairs<T>::load_clamped(us[i], rc.floor_small, rc.floor2_small, xs);
-            Pairs<T>::load_clamped(ul[i], rc.floor_large, rc.floor2_large, xl);
-            DivAcc local;
-            local.reset();
-            local.differ = (us[i].x ^ ul[i].x) | (us[i].y ^ ul[i].y) | (us[i].z ^ ul[i].z) | (us[i].w ^ ul[i].w);
-            div_accumulate<DIV, N, (sizeof(T) == 2 ? PSD_PSI_DEG_BF16 : 7)>(xl, xs, c, rc.off_large, rc.off_small, local);
-            if (len[i] > off) {   // a vector beyond the slice adds nothing
-              acc.js = __fadd2_rn(acc.js, local.js);
-              acc.big = __fadd2_rn(acc.big, local.big);
-              acc.differ |= local.differ;
+          for (int sub = 0; sub < SUB; ++sub, off += CH) {
+            const unsigned char* base = sbase + sub * kClSlotBytes;
+            uint4 us[kClBVec], ul[kClBVec];
+#pragma unroll
+            for (int i = 0; i < kClBVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+#pragma unroll
+            for (int i = 0; i < kClBVec; ++i) {
+              float2 xs[N], xl[N];
+              Pairs<T>::load_clamped(us[i], rc.floor_small, rc.floor2_small, xs);
+              Pairs<T>::load_clamped(ul[i], rc.floor_large, rc.floor2_large, xl);
+              DivAcc local;
+              local.reset();
+              local.differ = (us[i].x ^ ul[i].x) | (us[i].y ^ ul[i].y) | (us[i].z ^ ul[i].z) | (us[i].w ^ ul[i].w);
+              div_accumulate<DIV, N, (sizeof(T) == 2 ? PSD_PSI_DEG_BF16 : 7)>(xl, xs, c, rc.off_large, rc.off_small, local);
+              if (len[i] > off) {   // a vector beyond the slice adds nothing
+                acc.js = __fadd2_rn(acc.js, local.js);
+                acc.big = __fadd2_rn(acc.big, local.big);
+                acc.differ |= local.differ;
+              }
             }
           }
           __syncwarp();
@@ -657,27 +671,35 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         return (r >= rows1 ? row_ptr<T>(P.large2, P.seq_stride_large2, r - rows1, P.K2, V)
                            : row_ptr<T>(P.large, P.seq_stride_large, r, K, V)) + slice_begin;
       };
-      // chunk `cidx` of a row slice into `slot`, once the slot's readers of `fills` ring turns ago are through
-      auto fill = [&](const T* rs, const T* rl, int cidx, unsigned slot, unsigned fills) {
+      // step `step` of a row slice (SUB chunks) into `slot`, once the slot's readers of `fills` ring turns ago are through
+      auto fill = [&](const T* rs, const T* rl, int step, unsigned slot, unsigned fills) {
         if (fills > 0) wait_phase(&ctl->empty[slot], (fills - 1u) & 1u);
-        const int e0 = cidx * CH;
-        const int n = min(CH, slice_len - e0);
-        if (n > 0) {
-          const unsigned bytes = static_cast<unsigned>(n) * sizeof(T);
-          unsigned char* dst = ring + static_cast<size_t>(slot) * kClSlotBytes;
-          mbar_arrive_expect_tx(&ctl->full[slot], 2u * bytes);
-          bulk_load(dst, rs + e0, bytes, &ctl->full[slot]);
-          bulk_load(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot]);
+        unsigned total = 0;
+#pragma unroll
+        for (int sub = 0; sub < SUB; ++sub) total += static_cast<unsigned>(max(0, min(CH, slice_len - (step * SUB + sub) * CH)));
+        if (total > 0) {
+          mbar_arrive_expect_tx(&ctl->full[slot], 2u * total * static_cast<unsigned>(sizeof(T)));
+#pragma unroll
+          for (int sub = 0; sub < SUB; ++sub) {
+            const int e0 = (step * SUB + sub) * CH;
+            const int n = min(CH, slice_len - e0);
+            if (n > 0) {
+              const unsigned bytes = static_cast<unsigned>(n) * sizeof(T);
+              unsigned char* dst = ring + static_cast<size_t>(slot) * kSlotStride + sub * kClSlotBytes;
+              bulk_load(dst, rs + e0, bytes, &ctl->full[slot]);
+              bulk_load(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot]);
+            }
+          }
         } else {
-          mbar_arrive(&ctl->full[slot]);   // nothing of this chunk falls into this CTA's slice
+          mbar_arrive(&ctl->full[slot]);   // nothing of this step falls into this CTA's slice
         }
       };
       unsigned slot = lo, fills = 0;   // ring position; how often the ring has wrapped
       while (w.advance()) {
         const T* rs = row_small(w.r);
         const T* rl = row_large(w.r);
-        for (int cidx = 0; cidx < C; ++cidx) {
-          fill(rs, rl, cidx, slot, fills);
+        for (int step = 0; step < CS; ++step) {
+          fill(rs, rl, step, slot, fills);
           if (++slot == hi) { slot = lo; ++fills; }
         }
       }
@@ -1018,9 +1040,10 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
   g->ring = max(chunks + 1, min(kClSlots, 3 * chunks - 1));
   g->ra = 0;
   if (restream) {
-    g->ring = kClSlots;
+    // slots of two chunks each (32 KB): six of them, `ra` for pass A and the rest for pass B
+    g->ring = kClSlots / 2;
     static const int env_ra = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_RA"); return e ? std::atoi(e) : 0; }();
-    g->ra = (env_ra >= 2 && env_ra <= kClSlots - 2) ? env_ra : 5;   // measured: 4 to 8 of the 13 slots for pass A are alike
+    g->ra = (env_ra >= 1 && env_ra <= kClSlots / 2 - 1) ? env_ra : 3;   // measured: 3 + 3 beats 2 + 4 and 4 + 2
   }
   g->n_clusters = static_cast<int>(rows < max_active ? rows : max_active);
   return g->n_clusters > 0;
