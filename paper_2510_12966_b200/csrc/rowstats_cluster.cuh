@@ -64,6 +64,7 @@ struct ClusterGeom {
   int ra;        // 0: a slice stays in the ring from pass A to pass B. > 0 (slice larger than the ring): the
                  // slice is streamed twice through slots of two chunks each, slots [0, ra) feed pass A and
                  // slots [ra, ring) feed pass B
+  int lead;      // streamed twice: pass A hands row n to the agent once row n - lead has been released to pass B
 };
 
 // Per-row constants of pass B: -log2 of the normalisers in the scaled base-2 domain and the clamp floors.
@@ -131,6 +132,23 @@ __device__ __forceinline__ void remote_post_f4(unsigned cluster_addr, float4 v, 
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// The same copy with an L2 eviction priority: the streamed-twice variant asks L2 to keep what pass A's copy
+// brought in (pass B's copy of the same bytes follows a row slice later) and to drop pass B's copy first.
+__device__ __forceinline__ unsigned long long l2_policy_keep() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ unsigned long long l2_policy_drop() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gsrc, unsigned bytes, unsigned long long* bar,
+                                               unsigned long long policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
 }
 __device__ __forceinline__ unsigned cluster_rank() {
   unsigned r;
@@ -590,7 +608,10 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         // cannot: its slots come back from pass B). The exchange buffers are kClDepth rows deep, so row n is
         // handed over only once row n - kClDepth has been released to pass B, which is after the agent has
         // read that row's partials out of this buffer.
-        if (RS && w.n >= kClDepth) wait_phase(&ctl->b_go[d], ((w.n / kClDepth) - 1) & 1u);
+        if (RS && w.n >= G.lead) {
+          const int m = w.n - G.lead;   // 1 <= lead <= kClDepth
+          wait_phase(&ctl->b_go[m % kClDepth], (m / kClDepth) & 1u);
+        }
         if (lane == 0) {
           ctl->a_part[d][pw] = make_float4(ls.ref, ss, ll.ref, sl);
           mbar_arrive(&ctl->a_done[d]);
@@ -671,6 +692,7 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         return (r >= rows1 ? row_ptr<T>(P.large2, P.seq_stride_large2, r - rows1, P.K2, V)
                            : row_ptr<T>(P.large, P.seq_stride_large, r, K, V)) + slice_begin;
       };
+      const unsigned long long policy = RS ? (for_b ? l2_policy_drop() : l2_policy_keep()) : 0ull;
       // step `step` of a row slice (SUB chunks) into `slot`, once the slot's readers of `fills` ring turns ago are through
       auto fill = [&](const T* rs, const T* rl, int step, unsigned slot, unsigned fills) {
         if (fills > 0) wait_phase(&ctl->empty[slot], (fills - 1u) & 1u);
@@ -686,8 +708,13 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
             if (n > 0) {
               const unsigned bytes = static_cast<unsigned>(n) * sizeof(T);
               unsigned char* dst = ring + static_cast<size_t>(slot) * kSlotStride + sub * kClSlotBytes;
-              bulk_load(dst, rs + e0, bytes, &ctl->full[slot]);
-              bulk_load(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot]);
+              if (RS) {
+                bulk_load_hint(dst, rs + e0, bytes, &ctl->full[slot], policy);
+                bulk_load_hint(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot], policy);
+              } else {
+                bulk_load(dst, rs + e0, bytes, &ctl->full[slot]);
+                bulk_load(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot]);
+              }
             }
           }
         } else {
@@ -1010,8 +1037,8 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
     // CTAs place only 120), but for a large vocabulary their slice exceeds the ring and has to be streamed
     // twice. Estimated time = rounds of co-resident clusters / CTAs per row, times a measured factor:
     //   resident: 1 + 0.01 per CTA of the cluster (the per-row exchange);
-    //   streamed twice: 1.04 for bf16 (4 % at equal SM count), 1.0 for fp32 (there the wider ring lookahead
-    //   outweighs the second copy), plus up to 0.3 once the bytes between a chunk's first and second copy --
+    //   streamed twice: 1.0 (its hand-offs of two chunks at a time make up for the second copy: at equal
+    //   estimates it measures 0 to 3 % faster), plus up to 0.3 once the bytes between a chunk's first and second copy --
     //   one slice pair per CTA in flight -- outgrow what L2 keeps (48 MB and up: measured 1.04 at 55 MB,
     //   1.25 at 90 MB).
     auto rounds_per_cta = [&](int c, int n_active) {
@@ -1025,7 +1052,7 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
       const int na = cluster_max_active_any(dtype, P.div_kind, c2);
       if (na <= 0) continue;
       const double in_flight_mb = 2.0 * sl2 * es * static_cast<double>(na < rows ? na : rows) * c2 / 1048576.0;
-      double factor = dtype == 0 ? 1.0 : 1.04;
+      double factor = 1.0;
       if (in_flight_mb > 48.0) factor += 0.3 * ((in_flight_mb - 48.0) / 48.0 < 1.0 ? (in_flight_mb - 48.0) / 48.0 : 1.0);
       const double t = factor * rounds_per_cta(c2, na);
       if (t < best) { best = t; cs = c2; slice = sl2; chunks = ch2; restream = true; found = true; }
@@ -1039,11 +1066,14 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
   g->chunks = chunks;
   g->ring = max(chunks + 1, min(kClSlots, 3 * chunks - 1));
   g->ra = 0;
+  g->lead = kClDepth;
   if (restream) {
     // slots of two chunks each (32 KB): six of them, `ra` for pass A and the rest for pass B
     g->ring = kClSlots / 2;
     static const int env_ra = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_RA"); return e ? std::atoi(e) : 0; }();
     g->ra = (env_ra >= 1 && env_ra <= kClSlots / 2 - 1) ? env_ra : 3;   // measured: 3 + 3 beats 2 + 4 and 4 + 2
+    static const int env_lead = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_LEAD"); return e ? std::atoi(e) : 0; }();
+    g->lead = (env_lead >= 1 && env_lead <= kClDepth) ? env_lead : kClDepth;
   }
   g->n_clusters = static_cast<int>(rows < max_active ? rows : max_active);
   return g->n_clusters > 0;
