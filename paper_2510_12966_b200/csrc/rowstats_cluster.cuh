@@ -44,6 +44,10 @@ constexpr int kClBWarps = PSD_B_WARPS;             // warps running pass B (the 
 constexpr int kClConsumerWarps = kClAWarps + kClBWarps;
 constexpr int kClConsumers = kClConsumerWarps * 32;
 constexpr int kClThreads = kClConsumers + 96;      // + loader warp + two agent warps
+#ifndef PSD_RS_SUB
+#define PSD_RS_SUB 2
+#endif
+constexpr int kClSubRS = PSD_RS_SUB;               // chunks per slot of the streamed-twice variant
 constexpr int kClThreadsRS = kClThreads + 32;      // the streamed-twice variant has a loader warp per pass
 constexpr int kClHalfBytes = 8192;                 // one model's part of a chunk: 256 threads x 2 x 16 bytes
 constexpr int kClAVec = 16 / kClAWarps;            // 16-byte vectors per lane, chunk and model in pass A
@@ -465,7 +469,7 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
   const int RB0 = RS ? G.ra : 0;       // first slot of pass B
   // The streamed-twice variant moves two chunks per barrier (a slot of 2 x 16 KB): its rings need no chunk
   // granularity to hold a row, and every hand-off costs the two instruction streams issue slots.
-  constexpr int SUB = RS ? 2 : 1;
+  constexpr int SUB = RS ? kClSubRS : 1;
   constexpr int kSlotStride = SUB * kClSlotBytes;
   const int CS = (C + SUB - 1) / SUB;  // barrier steps per row slice
 
@@ -1069,9 +1073,9 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
   g->lead = kClDepth;
   if (restream) {
     // slots of two chunks each (32 KB): six of them, `ra` for pass A and the rest for pass B
-    g->ring = kClSlots / 2;
+    g->ring = kClSlots / kClSubRS;
     static const int env_ra = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_RA"); return e ? std::atoi(e) : 0; }();
-    g->ra = (env_ra >= 1 && env_ra <= kClSlots / 2 - 1) ? env_ra : 3;   // measured: 3 + 3 beats 2 + 4 and 4 + 2
+    g->ra = (env_ra >= 1 && env_ra <= kClSlots / kClSubRS - 1) ? env_ra : (kClSlots / kClSubRS) / 2;   // measured: 3 + 3 beats 2 + 4 and 4 + 2
     static const int env_lead = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_LEAD"); return e ? std::atoi(e) : 0; }();
     g->lead = (env_lead >= 1 && env_lead <= kClDepth) ? env_lead : kClDepth;
   }
