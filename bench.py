@@ -148,7 +148,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     binding.load_library()
     binding.set_stream()
-    binding.set_two_stage_policy(binding.TWO_STAGE_SEPARATE if args.two_stage == "separate" else binding.TWO_STAGE_FUSED)
+    binding.set_two_stage_policy({"separate": binding.TWO_STAGE_SEPARATE, "auto": binding.TWO_STAGE_AUTO}.get(args.two_stage, binding.TWO_STAGE_FUSED))
     cfg, w = workload_from_name(args.workload)
     if args.batch > 0:
         import dataclasses
@@ -212,7 +212,7 @@ def run_ours(args):
     row_bytes = 2 * w.V * es
     rs_bytes = n_pos * row_bytes   # the statistics kernel streams each verified row pair once
     timed_cap = 4096               # launches the library's event timing holds; beyond it only the first ones are timed
-    launches_per_step = 2 if args.two_stage == "fused" else 4
+    launches_per_step = {"fused": 2, "separate": 4}.get(args.two_stage) or (4 if launches >= 3 * args.steps else 2)
     if launches_per_step * args.steps > timed_cap:
         steps_timed = timed_cap // launches_per_step
         rs_bytes = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(steps_timed)) * row_bytes
@@ -554,7 +554,7 @@ def main():
     ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences per step of the CPU-oracle reference arm")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (small profiling cases)")
     ap.add_argument("--vocab", type=int, default=0, help="override the vocabulary size V of cfg5 (small profiling cases)")
-    ap.add_argument("--two-stage", choices=["fused", "separate"], default="fused",
+    ap.add_argument("--two-stage", choices=["fused", "separate", "auto"], default="fused",
                     help="schedule of the two stages (same results): one statistics launch for both, or stage by stage")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

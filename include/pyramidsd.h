@@ -240,6 +240,12 @@ size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype);
  * which wins when acceptance is low and windows are short. */
 #define PSD_TWO_STAGE_FUSED 0
 #define PSD_TWO_STAGE_SEPARATE 1
+/* PSD_TWO_STAGE_AUTO: the library chooses per call. Stage 1 also leaves each sequence's window length in a small
+ * host-mapped buffer (no copy, no synchronisation); a later call with the same B and K_q on this device reads
+ * whatever lengths are there -- those of a recent call -- and runs stage by stage when the unfilled part of
+ * the windows is more than a tenth of all rows and the batch has at least 1024 rows, else in two launches.
+ * The first call of a shape runs in two launches. */
+#define PSD_TWO_STAGE_AUTO 2
 int pyramidsd_set_two_stage_policy(int policy);
 
 /* Stream used by the entry points that carry no stream argument (a cudaStream_t; NULL = legacy default

@@ -154,7 +154,7 @@ def set_stream(stream: Optional[torch.cuda.Stream] = None) -> None:
     _check(load_library().pyramidsd_set_stream(C.c_void_p(s.cuda_stream)), "pyramidsd_set_stream")
 
 
-TWO_STAGE_FUSED, TWO_STAGE_SEPARATE = 0, 1
+TWO_STAGE_FUSED, TWO_STAGE_SEPARATE, TWO_STAGE_AUTO = 0, 1, 2
 
 
 def set_two_stage_policy(policy: int) -> None:

@@ -64,6 +64,10 @@ struct StageParams {
   // 1: the large tensor holds K + 1 rows per sequence; a sequence whose valid positions were all accepted
   // gets its next token from the row after the last valid one (the larger model's bonus token, Sec. 1).
   int bonus;
+  // Two-stage wrapper, optional: the window lengths of the first fill_cap sequences are also stored here (host
+  // memory mapped into the device), where the host reads them to choose its schedule for later calls.
+  int32_t* fill_out;
+  int fill_cap;
 };
 
 // ---- special functions (single MUFU instruction each) -------------------------------------------------

@@ -345,6 +345,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
       const int have = L + (next >= 0 ? 1 : 0);
       const int n2 = min(have, P.K_window);
       P.n_window[b] = n2;
+      if (P.fill_out != nullptr && b < P.fill_cap) P.fill_out[b] = n2;
       for (int j = 0; j < P.K_window; ++j)
         P.window[b * P.K_window + j] = (j < n2) ? ((j < L) ? P.tokens[b * K + j] : next) : 0;
     }

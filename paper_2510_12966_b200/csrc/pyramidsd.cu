@@ -52,7 +52,13 @@ struct DeviceState {
   size_t out4_elems = 0;
   void* lm_ws = nullptr;    // partial sums of the fused LM-head path
   size_t lm_ws_bytes = 0;
+  // PSD_TWO_STAGE_AUTO: window lengths of a recent call, written by the stage-1 finalisation straight into
+  // mapped host memory
+  int32_t* fill_host = nullptr;
+  int32_t* fill_dev = nullptr;
+  int fill_B = 0, fill_Kq = 0;   // the shape those lengths belong to
 };
+constexpr int kFillCap = 4096;
 DeviceState g_dev[kMaxDevices];
 
 int current_device_state(DeviceState** out) {
@@ -296,7 +302,8 @@ cudaStream_t pick_stream(const psd_stage_args* a) {
 
 // Runs one stage; `window_out`/`n_window_out`/`K_window` non-null make the finalisation also build the
 // stage-2 window of the wrapper.
-int run_stage(const psd_stage_args* a, int32_t* window_out, int32_t* n_window_out, int K_window) {
+int run_stage(const psd_stage_args* a, int32_t* window_out, int32_t* n_window_out, int K_window,
+              int32_t* fill_out = nullptr) {
   int rc = validate_stage(a);
   if (rc != PSD_OK) return rc;
   if (a->B == 0) return PSD_OK;
@@ -318,6 +325,8 @@ int run_stage(const psd_stage_args* a, int32_t* window_out, int32_t* n_window_ou
   P.window = window_out;
   P.n_window = n_window_out;
   P.K_window = K_window;
+  P.fill_out = fill_out;
+  P.fill_cap = kFillCap;
   const cudaStream_t stream = pick_stream(a);
   if (a->K > 0) {
     rc = launch_rowstats(P, a->dtype, a->kernel_variant, a->cluster_size, stream);
@@ -386,7 +395,40 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   rc = validate_stage(&s1);
   if (rc == PSD_OK) rc = validate_stage(&s2);
   if (rc != PSD_OK) return rc;
-  if (t_two_stage_policy == PSD_TWO_STAGE_SEPARATE) {
+  bool separate = t_two_stage_policy == PSD_TWO_STAGE_SEPARATE;
+  int32_t* fill_out = nullptr;
+  if (t_two_stage_policy == PSD_TWO_STAGE_AUTO) {
+    std::lock_guard<std::mutex> lock(ds->mu);
+    if (ds->fill_host == nullptr) {
+      void* h = nullptr;
+      void* d = nullptr;
+      if (cudaHostAlloc(&h, kFillCap * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess &&
+          cudaHostGetDevicePointer(&d, h, 0) == cudaSuccess) {
+        ds->fill_host = static_cast<int32_t*>(h);
+        ds->fill_dev = static_cast<int32_t*>(d);
+      } else {
+        cudaGetLastError();   // no mapped memory: stay with two launches
+      }
+    }
+    if (ds->fill_host != nullptr) {
+      const int n = B < kFillCap ? B : kFillCap;
+      const long long rows = static_cast<long long>(B) * (K_d + K_q);
+      if (ds->fill_B == B && ds->fill_Kq == K_q && rows >= 1024) {
+        long long filled = 0;
+        const volatile int32_t* f = ds->fill_host;
+        for (int i = 0; i < n; ++i) { const int v = f[i]; filled += v < 0 ? 0 : (v > K_q ? K_q : v); }
+        // rows the stage-by-stage schedule would skip, as a share of all rows
+        const double skipped = (1.0 - static_cast<double>(filled) / (static_cast<double>(n) * K_q)) * K_q / (K_d + K_q);
+        separate = skipped > 0.10;
+      } else {
+        for (int i = 0; i < n; ++i) ds->fill_host[i] = K_q;   // unknown: assume full windows until stage 1 says otherwise
+        ds->fill_B = B;
+        ds->fill_Kq = K_q;
+      }
+      fill_out = ds->fill_dev;
+    }
+  }
+  if (separate) {
     // stage by stage: stage 2's statistics run after stage 1 has fixed the windows and skip the rows beyond them.
     // Both launches take the cluster size the single-launch schedule would pick, so a row's vocabulary is
     // cut into the same slices and its statistics come out bit-identical under either policy.
@@ -399,7 +441,7 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
       psd::ClusterGeom g{};
       if (variant != PSD_KERNEL_BASELINE && psd::cluster_geometry(PS, dtype, 0, &g)) s1.cluster_size = s2.cluster_size = g.cs;
     }
-    rc = run_stage(&s1, window, n_window, K_q);
+    rc = run_stage(&s1, window, n_window, K_q, fill_out);
     if (rc != PSD_OK) return rc;
     return run_stage(&s2, nullptr, nullptr, 0);
   }
@@ -416,6 +458,8 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   P1.window = window;
   P1.n_window = n_window;
   P1.K_window = K_q;
+  P1.fill_out = fill_out;
+  P1.fill_cap = kFillCap;
   const StageParams P2 = make_params(&s2, s2.workspace, ds->status);
   StageParams PS = P1;
   PS.small2 = P2.small;
@@ -803,7 +847,7 @@ size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype) {
 }
 
 int pyramidsd_set_two_stage_policy(int policy) {
-  if (policy != PSD_TWO_STAGE_FUSED && policy != PSD_TWO_STAGE_SEPARATE) return PSD_ERR_INVALID_ARG;
+  if (policy != PSD_TWO_STAGE_FUSED && policy != PSD_TWO_STAGE_SEPARATE && policy != PSD_TWO_STAGE_AUTO) return PSD_ERR_INVALID_ARG;
   t_two_stage_policy = policy;
   return PSD_OK;
 }

@@ -473,6 +473,34 @@ def test_two_stage_policies_give_the_same_results(psd, wl, B, K_d, K_q, V, dtype
         assert 0 < int(a["accept_len_q"].sum()) < B * K_d
 
 
+def test_two_stage_auto_policy_follows_the_window_lengths(psd, wl):
+    """PSD_TWO_STAGE_AUTO: the first call of a shape runs in two launches; once stage 1 has reported short
+    windows the next call runs stage by stage (four launches), and goes back when the windows are full again.
+    The results are those of the fixed schedules, bit for bit."""
+    dev = torch.device("cuda:0")
+    B, K_d, K_q, V = 48, 16, 8, 8192            # 1152 rows
+    zd, zq, zt, tok = [t.to(dev) for t in wl.make_pyramid_inputs(B, K_d, K_q, V, "bf16", seed=41, sigma_q=0.6, sigma_d=2.5)]
+    psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+    ref_low = psd.verify(zd, zq, zt, tok, 0.02, 0.02, 0, 5, 6)      # tight threshold: short windows
+    ref_full = psd.verify(zd, zq, zt, tok, 1.0, 1.0, 0, 5, 8)       # tau > ln 2: every window full
+    torch.cuda.synchronize()
+    assert float(ref_low["accept_len_q"].float().mean()) < 3 and int(ref_full["accept_len"].min()) == K_q
+    try:
+        psd.set_two_stage_policy(psd.TWO_STAGE_AUTO)
+        launches = []
+        for tau, offset, ref in ((0.02, 6, ref_low), (0.02, 6, ref_low), (1.0, 8, ref_full), (1.0, 8, ref_full)):
+            n0 = psd.launch_count()
+            out = psd.verify(zd, zq, zt, tok, tau, tau, 0, 5, offset)
+            torch.cuda.synchronize()
+            launches.append(psd.launch_count() - n0)
+            for k in ref:
+                assert torch.equal(ref[k], out[k]), k
+        assert launches == [2, 4, 4, 2], launches
+    finally:
+        psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+    assert psd.last_status() == 0
+
+
 def test_host_entry_point_equals_device_entry_point(psd, wl):
     dev = torch.device("cuda:0")
     zd, zq, zt, tok = wl.make_pyramid_inputs(5, 8, 4, 9000, "bf16", seed=22)
