@@ -134,8 +134,10 @@ def verify_stage(logits_small, logits_large, tokens, tau, mode=FUZZY, seed=0, of
 
 
 def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode=FUZZY, seed=0, offset=0,
-           inv_temperature=1.0, div_kind=JS, n_threads=1, seq_ids=None):
-    """Two-stage pyramid on host arrays: draft/qual [B, K_d, V], target [B, K_q, V]."""
+           inv_temperature=1.0, div_kind=JS, n_threads=1, seq_ids=None, mode_t=None):
+    """Two-stage pyramid on host arrays: draft/qual [B, K_d, V], target [B, K_q, V]. ``mode`` is the
+    qualifier stage's acceptance mode and ``mode_t`` the target stage's (default: the same); the assisted
+    variant of Sec. 3.4 is ``mode=ASSISTED, mode_t=FUZZY``."""
     d, dt = _as_logits(logits_draft)
     q, dtq = _as_logits(logits_qual)
     t, dtt = _as_logits(logits_target)
@@ -152,7 +154,8 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
     }
     rc = lib().psd_oracle_verify(
         _ptr(d), _ptr(q), _ptr(t), _ptr(tok), B, K_d, K_q, V, dt,
-        C.c_double(float(tau_q)), C.c_double(float(tau_t)), int(mode), C.c_uint64(seed), C.c_uint64(offset),
+        C.c_double(float(tau_q)), C.c_double(float(tau_t)), int(mode), int(mode if mode_t is None else mode_t),
+        C.c_uint64(seed), C.c_uint64(offset),
         C.c_double(inv_temperature), int(div_kind), _ptr(ids),
         _ptr(out["accept_len_q"]), _ptr(out["next_token_q"]), _ptr(out["accept_len"]), _ptr(out["next_token"]),
         _ptr(out["window"]), _ptr(out["n_window"]), _ptr(out["div_q"]), _ptr(out["div_t"]), int(n_threads))
@@ -189,15 +192,16 @@ def verify_stage_bonus(logits_small, logits_large_k1, tokens, tau, mode=FUZZY, s
 
 
 def verify_bonus(logits_draft, logits_qual, logits_target_k1, draft_tokens, tau_q, tau_t, mode=FUZZY, seed=0,
-                 offset=0, n_threads=1, seq_ids=None):
+                 offset=0, n_threads=1, seq_ids=None, mode_t=None):
     """Two-stage pyramid whose target supplies K_q+1 rows per sequence: stage 1 and the window as in
     ``verify``; stage 2 is ``verify_stage_bonus`` on the window (Philox offset + 1)."""
     t, _ = _as_logits(logits_target_k1)
     q, _ = _as_logits(logits_qual)
     K_q = t.shape[1] - 1
     base = verify(logits_draft, logits_qual, np.ascontiguousarray(t[:, :K_q]), draft_tokens, tau_q, tau_t, mode, seed,
-                  offset, n_threads=n_threads, seq_ids=seq_ids)
-    s2 = verify_stage_bonus(np.ascontiguousarray(q[:, :K_q]), t, base["window"], tau_t, mode, seed, offset + 1,
+                  offset, n_threads=n_threads, seq_ids=seq_ids, mode_t=mode_t)
+    s2 = verify_stage_bonus(np.ascontiguousarray(q[:, :K_q]), t, base["window"], tau_t, mode if mode_t is None else mode_t,
+                            seed, offset + 1,
                             n_valid=base["n_window"], n_threads=n_threads, seq_ids=seq_ids)
     assert np.array_equal(s2["accept_len"], base["accept_len"])
     out = dict(base)

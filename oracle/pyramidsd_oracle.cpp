@@ -367,10 +367,13 @@ double psd_oracle_bonus_uniform(uint64_t seed, uint64_t offset, uint32_t b) { re
 // Two-stage pyramid (Fig. 1): stage 1 verifies the K_d draft tokens against the qualifier with tau_q;
 // the accepted prefix plus the qualifier's correction token form the window, cut to K_q; stage 2
 // verifies the window against the target with tau_t, the qualifier's distribution standing in for the
-// draft's. Stage 1 draws with `offset`, stage 2 with `offset + 1`.
+// draft's. Stage 1 draws with `offset`, stage 2 with `offset + 1`. Each stage has its own acceptance mode:
+// the assisted variant of Sec. 3.4 (PSD_A) replaces only the qualifier stage by assisted decoding -- strict
+// acceptance, and on rejection a draw from the qualifier's own distribution -- while the target stage keeps
+// its threshold tau_t; the fuzzy variant (PSD_F) uses the threshold rule in both.
 int psd_oracle_verify(const void* logits_draft, const void* logits_qual, const void* logits_target,
                       const int32_t* draft_tokens, int B, int K_d, int K_q, int V, int dtype,
-                      double tau_q, double tau_t, int mode, uint64_t seed, uint64_t offset,
+                      double tau_q, double tau_t, int mode_q, int mode_t, uint64_t seed, uint64_t offset,
                       double inv_temperature, int div_kind, const int32_t* seq_ids,
                       int32_t* out_accept_len_q, int32_t* out_next_token_q,
                       int32_t* out_accept_len, int32_t* out_next_token,
@@ -379,7 +382,7 @@ int psd_oracle_verify(const void* logits_draft, const void* logits_qual, const v
                       int n_threads) {
   if (K_q > K_d || K_q < 0) return -1;
   StageArgs s1{logits_draft, logits_qual, draft_tokens, B, K_d, V, dtype, V, V,
-               tau_q, mode, seed, offset, nullptr, inv_temperature, div_kind, seq_ids};
+               tau_q, mode_q, seed, offset, nullptr, inv_temperature, div_kind, seq_ids};
   int rc = verify_stage_impl(s1, out_accept_len_q, out_next_token_q, out_div_q, nullptr, nullptr, nullptr,
                              nullptr, nullptr, n_threads);
   if (rc) return rc;
@@ -401,7 +404,7 @@ int psd_oracle_verify(const void* logits_draft, const void* logits_qual, const v
     std::memcpy(qual_view.data() + (size_t)b * K_q * V * es,
                 (const unsigned char*)logits_qual + (size_t)b * K_d * V * es, (size_t)K_q * V * es);
   StageArgs s2{qual_view.data(), logits_target, window.data(), B, K_q, V, dtype, V, V,
-               tau_t, mode, seed, offset + 1, n2.data(), inv_temperature, div_kind, seq_ids};
+               tau_t, mode_t, seed, offset + 1, n2.data(), inv_temperature, div_kind, seq_ids};
   rc = verify_stage_impl(s2, out_accept_len, out_next_token, out_div_t, nullptr, nullptr, nullptr,
                          nullptr, nullptr, n_threads);
   if (out_window) std::memcpy(out_window, window.data(), window.size() * sizeof(int32_t));

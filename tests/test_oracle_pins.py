@@ -368,6 +368,50 @@ def test_pyramid_all_accepted_first_stage(oracle):
 
 
 # ---------------------------------------------------------------- fused LM-head logits
+def test_pyramid_assisted_qualifier_stage_keeps_the_fuzzy_target_stage(oracle):
+    # Sec. 3.4 (PSD_A): assisted decoding takes the place of tau_Q only; the target stage keeps tau_T.
+    # (a) composition on random inputs: stage 1 is the assisted stage, stage 2 the fuzzy stage on the window.
+    rng = np.random.default_rng(19)
+    B, K_d, K_q, V = 12, 5, 3, 30
+    zt_full = rng.normal(0, 3, (B, K_d, V)).astype(np.float32)
+    zq = (zt_full + rng.normal(0, 0.7, (B, K_d, V))).astype(np.float32)
+    zd = (zt_full + rng.normal(0, 1.0, (B, K_d, V))).astype(np.float32)
+    zt = np.ascontiguousarray(zt_full[:, :K_q])
+    tok = np.stack([[rng.choice(V, p=sp_softmax(zd[b, k])) for k in range(K_d)] for b in range(B)]).astype(np.int32)
+    out = oracle.verify(zd, zq, zt, tok, 0.9, 0.15, mode=oracle.ASSISTED, mode_t=oracle.FUZZY, seed=3, offset=20)
+    s1 = oracle.verify_stage(zd, zq, tok, 0.9, mode=oracle.ASSISTED, seed=3, offset=20)
+    assert np.array_equal(out["accept_len_q"], s1["accept_len"]) and np.array_equal(out["next_token_q"], s1["next_token"])
+    assert 0 < s1["accept_len"].sum() < B * K_d            # tau_q = 0.9 > ln 2 would accept everything if it were used
+    s2 = oracle.verify_stage(np.ascontiguousarray(zq[:, :K_q]), zt, out["window"], 0.15, mode=oracle.FUZZY, seed=3,
+                             offset=21, n_valid=out["n_window"])
+    assert np.array_equal(out["accept_len"], s2["accept_len"]) and np.array_equal(out["next_token"], s2["next_token"])
+    same = oracle.verify(zd, zq, zt, tok, 0.9, 0.15, mode=oracle.ASSISTED, seed=3, offset=20)   # mode_t defaults to mode
+    s2a = oracle.verify_stage(np.ascontiguousarray(zq[:, :K_q]), zt, out["window"], 0.15, mode=oracle.ASSISTED, seed=3,
+                              offset=21, n_valid=out["n_window"])
+    assert np.array_equal(same["accept_len"], s2a["accept_len"]) and not np.array_equal(same["accept_len"], out["accept_len"])
+    # (b) the laws, K_d = K_q = 1, V = 16: the window token (draft token if accepted, else a draw from the
+    # qualifier) follows min(p_q, p_d) + (1 - sum min) * p_q; a target stage with tau_T above ln 2 accepts it
+    # whatever it is (threshold rule: the token plays no part), and with tau_T < 0 rejects it and draws from
+    # the residual max(0, p_t - p_q), again whatever the window token was.
+    V, n = 16, 300_000
+    p_d, p_q, p_t = (sp_softmax(rng.normal(0, 1.5, V)) for _ in range(3))
+    x = rng.choice(V, size=n, p=p_d).astype(np.int32).reshape(n, 1)
+    zd1, zq1, zt1 = (np.broadcast_to(_logits_from_probs(p), (n, 1, V)).copy() for p in (p_d, p_q, p_t))
+    acc_all = oracle.verify(zd1, zq1, zt1, x, 0.0, 1.0, mode=oracle.ASSISTED, mode_t=oracle.FUZZY, seed=4, offset=6, n_threads=8)
+    assert np.all(acc_all["n_window"] == 1) and np.all(acc_all["accept_len"] == 1) and np.all(acc_all["next_token"] == -1)
+    law = np.minimum(p_q, p_d) + (1 - np.minimum(p_q, p_d).sum()) * p_q
+    counts = np.bincount(acc_all["window"][:, 0], minlength=V)
+    assert stats.chisquare(counts, law * n).pvalue > 1e-3
+    assert stats.chisquare(counts, p_q * n).pvalue < 1e-6 and stats.chisquare(counts, p_d * n).pvalue < 1e-6
+    rej_all = oracle.verify(zd1, zq1, zt1, x, 0.0, -1.0, mode=oracle.ASSISTED, mode_t=oracle.FUZZY, seed=4, offset=6, n_threads=8)
+    assert np.all(rej_all["accept_len"] == 0) and np.array_equal(rej_all["window"], acc_all["window"])
+    resid = np.maximum(p_t - p_q, 0.0)
+    live = resid > 0
+    counts = np.bincount(rej_all["next_token"], minlength=V)
+    assert np.all(counts[~live] == 0)
+    assert stats.chisquare(counts[live], resid[live] / resid.sum() * n).pvalue > 1e-3
+
+
 def test_lmhead_logits_match_library_matmul(oracle):
     import torch
     g = torch.Generator().manual_seed(0)
