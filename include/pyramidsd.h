@@ -15,6 +15,8 @@
  * Random numbers: one Philox4x32-10 block per row, counter (r, 0, offset_lo, offset_hi), key
  * (seed_lo, seed_hi); u = (word0 >> 8) * 2^-24 decides the strict coin flip, u' = (word1 >> 8) * 2^-24
  * drives the inverse CDF. The two-stage wrapper uses `offset` for stage 1 and `offset + 1` for stage 2.
+ * r is the row's index in the WHOLE batch: r = (seq_index_base + b) * K + k (low 32 bits), so that a call on a
+ * slice of a batch -- a shard on another GPU, a micro-batch -- draws what the call on the whole batch draws.
  *
  * Conventions shared by every entry point unless stated otherwise:
  *   - All data pointers are DEVICE pointers owned by the caller; the library never frees or keeps them.
@@ -29,13 +31,19 @@
  *     or -1 when every valid position was accepted.
  *   - Work is enqueued on the stream set by pyramidsd_set_stream (default: the legacy default stream)
  *     or given in the argument struct; calls return without synchronising. Scratch memory comes from
- *     the caller's workspace when one is supplied (pyramidsd_workspace_bytes), otherwise from a
- *     library-owned per-device buffer that is grown with cudaMalloc on first use (that growth
- *     synchronises the device once).
+ *     the caller's workspace when one is supplied (pyramidsd_workspace_bytes /
+ *     pyramidsd_pyramid_workspace_bytes), otherwise from library-owned buffers kept per (device, stream):
+ *     a call only ever touches the buffers of the stream it runs on, so calls on different streams, from
+ *     one host thread or several, do not share scratch. Such a buffer is created with cudaMalloc the
+ *     first time a stream is used and grown when a larger call arrives (growing waits for that stream's
+ *     earlier work, frees, allocates). At most PSD_MAX_STREAMS streams per device get buffers; a call on
+ *     yet another stream without a workspace returns PSD_ERR_WORKSPACE. Two host threads that share one
+ *     stream are serialised for the duration of the enqueue.
  *   - Return value: PSD_OK or a negative psd_status. Arguments are validated on the host before any
  *     launch; nothing is launched on error. Device-side bounded waits that give up report
  *     PSD_ERR_TIMEOUT through pyramidsd_last_status().
  */
+#define PSD_MAX_STREAMS 16
 #ifndef PYRAMIDSD_H_
 #define PYRAMIDSD_H_
 
@@ -75,8 +83,10 @@ typedef enum {
 typedef enum {
   PSD_KERNEL_AUTO = 0,
   PSD_KERNEL_BASELINE = 1, /* one CTA per row, three passes over global memory */
-  PSD_KERNEL_CLUSTER = 2   /* one thread-block cluster per row pair; its slices sit in the CTAs' shared memory for both passes, or,
+  PSD_KERNEL_CLUSTER = 2,  /* one thread-block cluster per row pair; its slices sit in the CTAs' shared memory for both passes, or,
                             * for clusters of 1 or 2 CTAs on a large vocabulary, are copied in once per pass (second copy from L2) */
+  PSD_KERNEL_CLUSTER_STREAMED = 3 /* the cluster kernel in its copied-in-once-per-pass form whatever the slice size (needs cluster_size);
+                                   * same arithmetic, same bits as PSD_KERNEL_CLUSTER with that cluster size */
 } psd_kernel_variant;
 
 /* Extended single-stage arguments. Zero-initialise, set struct_size = sizeof(psd_stage_args), fill what
@@ -116,6 +126,9 @@ typedef struct psd_stage_args {
                                   * n_valid[b], or K) -- the larger model's own next token, which ends every accepted run
                                   * (Sec. 1) -- by inverse CDF with the uniform of Philox counter (b, 1, offset_lo, offset_hi),
                                   * word 1; -2 if that row holds NaN, +inf or no finite logit. */
+  int32_t reserved0;
+  int64_t seq_index_base;        /* index of this call's sequence 0 in the whole batch (see the Philox counter above and the
+                                  * bonus counter): 0 for an unsharded call; >= 0 */
 } psd_stage_args;
 
 /* One verification stage (Sec. 3.1 for one model pair; Sec. 3.2 applies it twice). Jensen-Shannon
@@ -143,6 +156,55 @@ int pyramidsd_verify(const void* logits_draft, const void* logits_qual, const vo
                      float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
                      int32_t* out_accept_len_q, int32_t* out_next_token_q,
                      int32_t* out_accept_len, int32_t* out_next_token);
+
+/* The two-stage pyramid with every option exposed. Zero-initialise, set struct_size, fill what you need.
+ *   mode_q / mode_t   acceptance mode of the qualifier stage and of the target stage. PSD_F of the paper is
+ *                     (PSD_FUZZY, PSD_FUZZY); PSD_A (Sec. 3.4: assisted decoding in place of tau_Q, on rejection
+ *                     a draw from the qualifier's own distribution, the target stage unchanged) is
+ *                     (PSD_ASSISTED, PSD_FUZZY), and tau_q is then unused.
+ *   seq_index_base    as in psd_stage_args: a call on sequences [base, base + B) of a batch returns, bit for
+ *                     bit, what the call on the whole batch returns for them.
+ *   target_has_bonus_row  logits_target is [B, K_q + 1, V] (see pyramidsd_verify_bonus).
+ *   out_div_q [B, K_d], out_resid_q [B, K_d], out_div_t [B, K_q], out_resid_t [B, K_q]: per-row divergence and
+ *                     residual mass of the two stages, or NULL. Stage-2 rows at or beyond the window hold 0.
+ *   out_window [B, K_q], out_n_window [B]: the stage-2 window and its length, or NULL.
+ *   schedule          PSD_TWO_STAGE_DEFAULT (the thread's policy) or one of the schedules below.
+ *   workspace         >= pyramidsd_pyramid_workspace_bytes(B, K_d, K_q, V, dtype) bytes, 256-byte aligned; NULL =
+ *                     library-owned. */
+typedef struct psd_pyramid_args {
+  uint32_t struct_size;
+  int32_t dtype;                 /* psd_dtype */
+  const void* logits_draft;      /* [B, K_d, V] device */
+  const void* logits_qual;       /* [B, K_d, V] device */
+  const void* logits_target;     /* [B, K_q (+ 1), V] device */
+  const int32_t* draft_tokens;   /* [B, K_d] device */
+  int32_t B, K_d, K_q, V;
+  int32_t mode_q, mode_t;        /* psd_mode */
+  float tau_q, tau_t;
+  float inv_temperature;         /* 0 means 1 */
+  int32_t div_kind;              /* psd_div_kind */
+  uint64_t philox_seed, philox_offset;
+  int64_t seq_index_base;
+  int32_t target_has_bonus_row;
+  int32_t schedule;
+  int32_t* out_accept_len_q;     /* [B] device, required */
+  int32_t* out_next_token_q;     /* [B] device, required */
+  int32_t* out_accept_len;       /* [B] device, required */
+  int32_t* out_next_token;       /* [B] device, required */
+  float* out_div_q;
+  float* out_resid_q;
+  float* out_div_t;
+  float* out_resid_t;
+  int32_t* out_window;
+  int32_t* out_n_window;
+  void* workspace;
+  size_t workspace_bytes;
+  void* stream;                  /* cudaStream_t, or NULL for the stream set by pyramidsd_set_stream */
+  int32_t use_stream_field;      /* non-zero: take `stream` even when it is NULL */
+  int32_t kernel_variant;        /* PSD_KERNEL_AUTO or PSD_KERNEL_BASELINE */
+} psd_pyramid_args;
+int pyramidsd_verify_ex(const psd_pyramid_args* args);
+size_t pyramidsd_pyramid_workspace_bytes(int B, int K_d, int K_q, int V, psd_dtype dtype);
 
 /* pyramidsd_verify for a target that supplies one more row: logits_target is [B, K_q + 1, V]. Stage 1, the
  * window and the accept lengths are those of pyramidsd_verify; a window whose tokens were all accepted by
@@ -211,6 +273,32 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
                                   int32_t* out_accept_len, int32_t* out_next_token,
                                   float* out_div, float* out_resid_mass, void* cuda_stream);
 
+/* The same call with every option exposed. Zero-initialise, set struct_size, fill what you need.
+ *   seq_index_base  as in psd_stage_args.
+ *   tile_variant    PSD_LMHEAD_TILES_AUTO (pairs of CTAs on 256 x 256 tiles, tcgen05 cta_group::2) or
+ *                   PSD_LMHEAD_TILES_ONE_SM (one CTA per 256 x 128 tile); same results within rounding. */
+#define PSD_LMHEAD_TILES_AUTO 0
+#define PSD_LMHEAD_TILES_ONE_SM 1
+typedef struct psd_lmhead_args {
+  uint32_t struct_size;
+  int32_t mode;                  /* psd_mode */
+  const void* hidden;            /* [B*K, d_model] bf16 device */
+  const void* w_t;               /* [V, d_model] bf16 device */
+  const void* logits_small;      /* [B, K, V] bf16 device */
+  const int32_t* tokens;         /* [B, K] device */
+  int32_t B, K, d_model, V;
+  float threshold;
+  int32_t tile_variant;
+  uint64_t philox_seed, philox_offset;
+  int64_t seq_index_base;
+  int32_t* out_accept_len;       /* [B] device, required */
+  int32_t* out_next_token;       /* [B] device, required */
+  float* out_div;                /* [B, K] or NULL */
+  float* out_resid_mass;         /* [B, K] or NULL */
+  void* stream;                  /* cudaStream_t; NULL = the legacy default stream */
+} psd_lmhead_args;
+int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args);
+
 /* Analytic throughput model of Sec. 3.3 (host arithmetic, no GPU): tokens per second of standard or
  * fuzzy speculative decoding with speculative length ell and acceptance rate beta between a small model
  * of speed v_small and a large one of speed v_large (tokens/s each),
@@ -232,44 +320,41 @@ int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, fl
  * wrapper). Pure host arithmetic; 0 on invalid arguments. */
 size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype);
 
-/* How pyramidsd_verify / pyramidsd_verify_host schedule the two stages (per host thread; results are
- * bit-identical either way: both use the same split of a row over CTAs). PSD_TWO_STAGE_FUSED (default): two launches -- one statistics launch over the stage-1 rows
- * and all B*K_q stage-2 rows, one finalisation launch for both stages; best when windows are (nearly) full,
- * as in the paper's pipeline, which keeps drafting until the window holds K_q tokens (Fig. 1).
- * PSD_TWO_STAGE_SEPARATE: four launches, stage by stage; stage 2 then skips the rows beyond each window,
- * which wins when acceptance is low and windows are short. */
-#define PSD_TWO_STAGE_FUSED 0
-#define PSD_TWO_STAGE_SEPARATE 1
-/* PSD_TWO_STAGE_AUTO: the library chooses per call. Stage 1 also leaves each sequence's window length in a small
- * host-mapped buffer (no copy, no synchronisation); a later call with the same B and K_q on this device reads
- * whatever lengths are there -- those of a recent call -- and runs stage by stage when the unfilled part of
- * the windows is more than a tenth of all rows and the batch has at least 1024 rows, else in two launches.
- * The first call of a shape runs in two launches. */
-#define PSD_TWO_STAGE_AUTO 2
+/* How the two-stage calls schedule their launches (per host thread; every schedule returns the same results, bit
+ * for bit: all of them cut a row over the CTAs of a cluster the same way).
+ *   PSD_TWO_STAGE_FUSED     two launches: one statistics launch over the B*K_d stage-1 row pairs and all B*K_q
+ *                           stage-2 row pairs, one finalisation launch for both stages. Best when windows are
+ *                           (nearly) full, as in the paper's pipeline, which keeps drafting until the window holds
+ *                           K_q tokens (Fig. 1).
+ *   PSD_TWO_STAGE_SEPARATE  four launches, stage by stage; stage 2 then skips the rows beyond each window, which
+ *                           wins when acceptance is low and windows are short.
+ *   PSD_TWO_STAGE_AUTO      (the default) the library chooses between the two per call. Stage 1 also leaves each
+ *                           sequence's window length in a small host-mapped buffer (no copy, no synchronisation);
+ *                           a later call with the same B and K_q on this device reads whatever lengths are there
+ *                           -- those of a recent call -- and runs stage by stage when the unfilled part of the
+ *                           windows is more than a tenth of all rows and the batch has at least 1024 rows, else
+ *                           in two launches. The first call of a shape runs in two launches.
+ *   PSD_TWO_STAGE_FUSED_ROWS two launches like FUSED, but positions k < K_q are walked as row triples (draft,
+ *                           qualifier, target): the qualifier row, which stage 1 uses as its large model and
+ *                           stage 2 as its small one (Fig. 1), is read, widened and normalised once --
+ *                           (2 K_d + K_q) V s bytes instead of 2 (K_d + K_q) V s. Applies where the statistics
+ *                           kernel streams its rows twice (large batches); elsewhere it is FUSED. */
+#define PSD_TWO_STAGE_DEFAULT 0
+#define PSD_TWO_STAGE_FUSED 1
+#define PSD_TWO_STAGE_SEPARATE 2
+#define PSD_TWO_STAGE_AUTO 3
+#define PSD_TWO_STAGE_FUSED_ROWS 4
+/* PSD_TWO_STAGE_DEFAULT restores the library default. */
 int pyramidsd_set_two_stage_policy(int policy);
 
 /* Stream used by the entry points that carry no stream argument (a cudaStream_t; NULL = legacy default
  * stream). Per host thread. */
 int pyramidsd_set_stream(void* cuda_stream);
 
-/* Synchronises the library stream and returns PSD_OK, PSD_ERR_TIMEOUT if a device-side bounded wait gave
- * up since the last call, or PSD_ERR_CUDA if the stream reports an error. Clears the status word. */
+/* Synchronises the stream of this host thread's most recent call (the library stream if there was none) and
+ * returns PSD_OK, PSD_ERR_TIMEOUT if a device-side bounded wait gave up on that stream since its status was last
+ * read, or PSD_ERR_CUDA if the stream reports an error. Clears that stream's status word. */
 int pyramidsd_last_status(void);
-
-/* Per-kernel device timing for benchmarks. Between _begin and _end the library brackets each of its
- * kernel launches (on the calling thread) with CUDA events on the launch stream, up to 4096 launches.
- * _end synchronises those events, switches timing off, and returns the summed milliseconds and launch
- * counts of the row-statistics kernel and of the finalisation kernel (any output may be NULL). */
-int pyramidsd_kernel_timing_begin(void);
-int pyramidsd_kernel_timing_end(double* ms_rowstats, int* n_rowstats, double* ms_finalize, int* n_finalize);
-
-/* Number of kernels the library has launched from this process since load (all entry points). */
-uint64_t pyramidsd_launch_count(void);
-
-/* The cluster size (CTAs per row pair) the library picks for a [B, K, V] stage of this dtype and the
- * number of such clusters the current device keeps resident at once; 0 and 0 when the shape takes the
- * baseline kernel. Lets a caller size batches to whole waves. Needs a CUDA device. */
-int pyramidsd_cluster_occupancy(int B, int K, int V, psd_dtype dtype, int* out_cluster_size, int* out_max_active_clusters);
 
 const char* pyramidsd_version(void);
 const char* pyramidsd_status_string(int status);

@@ -17,12 +17,14 @@ from .build import LIB_PATH
 F32, BF16 = 0, 1
 FUZZY, STRICT, FUZZY_SD_FALLBACK, ASSISTED = 0, 1, 2, 3
 DIV_JS, DIV_TV, DIV_KL = 0, 1, 2
-KERNEL_AUTO, KERNEL_BASELINE, KERNEL_CLUSTER = 0, 1, 2
+KERNEL_AUTO, KERNEL_BASELINE, KERNEL_CLUSTER, KERNEL_CLUSTER_STREAMED = 0, 1, 2, 3
+LMHEAD_TILES_AUTO, LMHEAD_TILES_ONE_SM = 0, 1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 
 EXPORTS = (
-    "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_bonus", "pyramidsd_verify_host",
-    "pyramidsd_verify_stage_noalloc", "pyramidsd_verify_fused_lmhead",
+    "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_ex", "pyramidsd_verify_bonus",
+    "pyramidsd_verify_host", "pyramidsd_pyramid_workspace_bytes", "pyramidsd_selftest_wait_timeout",
+    "pyramidsd_verify_stage_noalloc", "pyramidsd_verify_fused_lmhead", "pyramidsd_verify_fused_lmhead_ex",
     "pyramidsd_model_sd_throughput", "pyramidsd_model_psd_throughput", "pyramidsd_set_two_stage_policy",
     "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
     "pyramidsd_kernel_timing_begin", "pyramidsd_kernel_timing_end",
@@ -47,6 +49,44 @@ class StageArgs(C.Structure):
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("stream", C.c_void_p), ("use_stream_field", C.c_int32), ("kernel_variant", C.c_int32),
         ("cluster_size", C.c_int32), ("large_has_bonus_row", C.c_int32),
+        ("reserved0", C.c_int32), ("seq_index_base", C.c_int64),
+    ]
+
+
+class PyramidArgs(C.Structure):
+    """Mirror of ``psd_pyramid_args``."""
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("dtype", C.c_int32),
+        ("logits_draft", C.c_void_p), ("logits_qual", C.c_void_p), ("logits_target", C.c_void_p),
+        ("draft_tokens", C.c_void_p),
+        ("B", C.c_int32), ("K_d", C.c_int32), ("K_q", C.c_int32), ("V", C.c_int32),
+        ("mode_q", C.c_int32), ("mode_t", C.c_int32),
+        ("tau_q", C.c_float), ("tau_t", C.c_float),
+        ("inv_temperature", C.c_float), ("div_kind", C.c_int32),
+        ("philox_seed", C.c_uint64), ("philox_offset", C.c_uint64),
+        ("seq_index_base", C.c_int64),
+        ("target_has_bonus_row", C.c_int32), ("schedule", C.c_int32),
+        ("out_accept_len_q", C.c_void_p), ("out_next_token_q", C.c_void_p),
+        ("out_accept_len", C.c_void_p), ("out_next_token", C.c_void_p),
+        ("out_div_q", C.c_void_p), ("out_resid_q", C.c_void_p), ("out_div_t", C.c_void_p), ("out_resid_t", C.c_void_p),
+        ("out_window", C.c_void_p), ("out_n_window", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("stream", C.c_void_p), ("use_stream_field", C.c_int32), ("kernel_variant", C.c_int32),
+    ]
+
+
+class LmheadArgs(C.Structure):
+    """Mirror of ``psd_lmhead_args``."""
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("mode", C.c_int32),
+        ("hidden", C.c_void_p), ("w_t", C.c_void_p), ("logits_small", C.c_void_p), ("tokens", C.c_void_p),
+        ("B", C.c_int32), ("K", C.c_int32), ("d_model", C.c_int32), ("V", C.c_int32),
+        ("threshold", C.c_float), ("tile_variant", C.c_int32),
+        ("philox_seed", C.c_uint64), ("philox_offset", C.c_uint64),
+        ("seq_index_base", C.c_int64),
+        ("out_accept_len", C.c_void_p), ("out_next_token", C.c_void_p),
+        ("out_div", C.c_void_p), ("out_resid_mass", C.c_void_p),
+        ("stream", C.c_void_p),
     ]
 
 
@@ -82,6 +122,14 @@ def load_library(path: Optional[str] = None):
     lib.pyramidsd_model_psd_throughput.restype = C.c_double
     lib.pyramidsd_verify_stage_ex.argtypes = [C.POINTER(StageArgs)]
     lib.pyramidsd_verify_stage_ex.restype = i32
+    lib.pyramidsd_verify_ex.argtypes = [C.POINTER(PyramidArgs)]
+    lib.pyramidsd_verify_ex.restype = i32
+    lib.pyramidsd_verify_fused_lmhead_ex.argtypes = [C.POINTER(LmheadArgs)]
+    lib.pyramidsd_verify_fused_lmhead_ex.restype = i32
+    lib.pyramidsd_pyramid_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    lib.pyramidsd_pyramid_workspace_bytes.restype = C.c_size_t
+    lib.pyramidsd_selftest_wait_timeout.argtypes = [vp]
+    lib.pyramidsd_selftest_wait_timeout.restype = i32
     pyr = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, u64, u64, vp, vp, vp, vp]
     lib.pyramidsd_verify.argtypes = pyr
     lib.pyramidsd_verify_bonus.restype = C.c_int
@@ -154,16 +202,27 @@ def set_stream(stream: Optional[torch.cuda.Stream] = None) -> None:
     _check(load_library().pyramidsd_set_stream(C.c_void_p(s.cuda_stream)), "pyramidsd_set_stream")
 
 
-TWO_STAGE_FUSED, TWO_STAGE_SEPARATE, TWO_STAGE_AUTO = 0, 1, 2
+TWO_STAGE_DEFAULT, TWO_STAGE_FUSED, TWO_STAGE_SEPARATE, TWO_STAGE_AUTO, TWO_STAGE_FUSED_ROWS = 0, 1, 2, 3, 4
 
 
 def set_two_stage_policy(policy: int) -> None:
-    """``pyramidsd_set_two_stage_policy``: one statistics launch for both stages, or stage by stage."""
+    """``pyramidsd_set_two_stage_policy``: one statistics launch for both stages (row pairs or row triples),
+    stage by stage, or chosen per call (the default)."""
     _check(load_library().pyramidsd_set_two_stage_policy(int(policy)), "pyramidsd_set_two_stage_policy")
 
 
 def last_status() -> int:
     return load_library().pyramidsd_last_status()
+
+
+def selftest_wait_timeout(stream=None) -> int:
+    """``pyramidsd_selftest_wait_timeout``: one kernel whose bounded wait runs out on purpose."""
+    s = torch.cuda.current_stream() if stream is None else stream
+    return load_library().pyramidsd_selftest_wait_timeout(C.c_void_p(s.cuda_stream))
+
+
+def pyramid_workspace_bytes(B: int, K_d: int, K_q: int, V: int, dtype: int) -> int:
+    return int(load_library().pyramidsd_pyramid_workspace_bytes(B, K_d, K_q, V, dtype))
 
 
 def launch_count() -> int:
@@ -222,7 +281,7 @@ def verify_stage(logits_small, logits_large, draft_tokens, threshold, mode=FUZZY
 
 
 def verify_fused_lmhead(hidden, w_t, logits_small, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
-                        want_rows=True, stream=None, raise_on_error=True):
+                        want_rows=True, stream=None, raise_on_error=True, tile_variant=None, seq_index_base=0):
     """``pyramidsd_verify_fused_lmhead``: hidden [B*K, d] bf16, w_t [V, d] bf16 (LM-head weight, out x in),
     logits_small [B, K, V] bf16, tokens [B, K]. Returns a dict of device tensors (+ "status")."""
     B, K, V = logits_small.shape
@@ -235,13 +294,29 @@ def verify_fused_lmhead(hidden, w_t, logits_small, tokens, threshold, mode=FUZZY
         out["div"] = torch.empty((B, K), dtype=torch.float32, device=dev)
         out["resid_mass"] = torch.empty((B, K), dtype=torch.float32, device=dev)
     s = torch.cuda.current_stream() if stream is None else stream
-    rc = load_library().pyramidsd_verify_fused_lmhead(
-        _dev_ptr(hidden, torch.bfloat16, "hidden"), _dev_ptr(w_t, torch.bfloat16, "w_t"),
-        _dev_ptr(logits_small, torch.bfloat16, "logits_small"), _dev_ptr(tokens, torch.int32, "tokens"),
-        B, K, d, V, float(threshold), int(mode), int(philox_seed), int(offset),
-        out["accept_len"].data_ptr(), out["next_token"].data_ptr(),
-        out["div"].data_ptr() if want_rows else None, out["resid_mass"].data_ptr() if want_rows else None,
-        C.c_void_p(s.cuda_stream))
+    if tile_variant is None and seq_index_base == 0:
+        rc = load_library().pyramidsd_verify_fused_lmhead(
+            _dev_ptr(hidden, torch.bfloat16, "hidden"), _dev_ptr(w_t, torch.bfloat16, "w_t"),
+            _dev_ptr(logits_small, torch.bfloat16, "logits_small"), _dev_ptr(tokens, torch.int32, "tokens"),
+            B, K, d, V, float(threshold), int(mode), int(philox_seed), int(offset),
+            out["accept_len"].data_ptr(), out["next_token"].data_ptr(),
+            out["div"].data_ptr() if want_rows else None, out["resid_mass"].data_ptr() if want_rows else None,
+            C.c_void_p(s.cuda_stream))
+    else:
+        a = LmheadArgs()
+        a.struct_size = C.sizeof(LmheadArgs)
+        a.mode = int(mode)
+        a.hidden, a.w_t = _dev_ptr(hidden, torch.bfloat16, "hidden"), _dev_ptr(w_t, torch.bfloat16, "w_t")
+        a.logits_small = _dev_ptr(logits_small, torch.bfloat16, "logits_small")
+        a.tokens = _dev_ptr(tokens, torch.int32, "tokens")
+        a.B, a.K, a.d_model, a.V = B, K, d, V
+        a.threshold, a.tile_variant = float(threshold), int(tile_variant or 0)
+        a.philox_seed, a.philox_offset, a.seq_index_base = int(philox_seed), int(offset), int(seq_index_base)
+        a.out_accept_len, a.out_next_token = out["accept_len"].data_ptr(), out["next_token"].data_ptr()
+        if want_rows:
+            a.out_div, a.out_resid_mass = out["div"].data_ptr(), out["resid_mass"].data_ptr()
+        a.stream = s.cuda_stream
+        rc = load_library().pyramidsd_verify_fused_lmhead_ex(C.byref(a))
     out["status"] = rc
     if raise_on_error:
         _check(rc, "pyramidsd_verify_fused_lmhead")
@@ -281,7 +356,8 @@ def verify_stage_noalloc(logits_small, logits_large, draft_tokens, threshold, mo
 def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
                     B=None, K=None, V=None, n_valid=None, inv_temperature=0.0, div_kind=DIV_JS,
                     seq_stride_small=0, seq_stride_large=0, want_rows=True, workspace=None, stream=None,
-                    kernel_variant=KERNEL_AUTO, cluster_size=0, raise_on_error=True, large_has_bonus_row=False):
+                    kernel_variant=KERNEL_AUTO, cluster_size=0, raise_on_error=True, large_has_bonus_row=False,
+                    seq_index_base=0):
     """``pyramidsd_verify_stage_ex``: every option exposed. Returns a dict of device tensors (+ "status").
     With ``large_has_bonus_row`` the large logits are [B, K + 1, V]."""
     if B is None:
@@ -324,6 +400,7 @@ def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, p
     a.kernel_variant = int(kernel_variant)
     a.cluster_size = int(cluster_size)
     a.large_has_bonus_row = 1 if large_has_bonus_row else 0
+    a.seq_index_base = int(seq_index_base)
     rc = load_library().pyramidsd_verify_stage_ex(C.byref(a))
     out["status"] = rc
     if raise_on_error:
@@ -349,6 +426,54 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
         out["accept_len_q"].data_ptr(), out["next_token_q"].data_ptr(),
         out["accept_len"].data_ptr(), out["next_token"].data_ptr())
     _check(rc, "pyramidsd_verify")
+    return out
+
+
+def verify_ex(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode_q=FUZZY, mode_t=None,
+              philox_seed=0, offset=0, *, seq_index_base=0, target_has_bonus_row=False, schedule=TWO_STAGE_DEFAULT,
+              inv_temperature=0.0, div_kind=DIV_JS, want_rows=True, want_window=True, workspace=None, stream=None,
+              kernel_variant=KERNEL_AUTO, raise_on_error=True):
+    """``pyramidsd_verify_ex``: the two-stage pyramid with per-stage modes, a sequence base, per-row outputs, the
+    window, a caller workspace and an explicit schedule. Returns a dict of device tensors (+ "status")."""
+    B, K_d, V = logits_draft.shape
+    K_q = logits_target.shape[1] - (1 if target_has_bonus_row else 0)
+    assert logits_qual.shape == logits_draft.shape and logits_target.shape[0] == B and logits_target.shape[2] == V
+    dev = logits_draft.device
+    out = {k: torch.empty(B, dtype=torch.int32, device=dev)
+           for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+    a = PyramidArgs()
+    a.struct_size = C.sizeof(PyramidArgs)
+    a.dtype = dtype_code(logits_draft)
+    a.logits_draft = _dev_ptr(logits_draft, name="logits_draft")
+    a.logits_qual = _dev_ptr(logits_qual, logits_draft.dtype, "logits_qual")
+    a.logits_target = _dev_ptr(logits_target, logits_draft.dtype, "logits_target")
+    a.draft_tokens = _dev_ptr(draft_tokens, torch.int32, "draft_tokens")
+    a.B, a.K_d, a.K_q, a.V = B, K_d, K_q, V
+    a.mode_q, a.mode_t = int(mode_q), int(mode_q if mode_t is None else mode_t)
+    a.tau_q, a.tau_t = float(tau_q), float(tau_t)
+    a.inv_temperature, a.div_kind = float(inv_temperature), int(div_kind)
+    a.philox_seed, a.philox_offset, a.seq_index_base = int(philox_seed), int(offset), int(seq_index_base)
+    a.target_has_bonus_row, a.schedule = (1 if target_has_bonus_row else 0), int(schedule)
+    for k in ("accept_len_q", "next_token_q", "accept_len", "next_token"):
+        setattr(a, "out_" + k, out[k].data_ptr())
+    if want_rows:
+        for k, n in (("div_q", K_d), ("resid_q", K_d), ("div_t", K_q), ("resid_t", K_q)):
+            out[k] = torch.empty((B, n), dtype=torch.float32, device=dev)
+            setattr(a, "out_" + k, out[k].data_ptr())
+    if want_window:
+        out["window"] = torch.empty((B, K_q), dtype=torch.int32, device=dev)
+        out["n_window"] = torch.empty(B, dtype=torch.int32, device=dev)
+        a.out_window, a.out_n_window = out["window"].data_ptr(), out["n_window"].data_ptr()
+    if workspace is not None:
+        a.workspace = workspace.data_ptr()
+        a.workspace_bytes = workspace.numel() * workspace.element_size()
+    s = torch.cuda.current_stream() if stream is None else stream
+    a.stream, a.use_stream_field = s.cuda_stream, 1
+    a.kernel_variant = int(kernel_variant)
+    rc = load_library().pyramidsd_verify_ex(C.byref(a))
+    out["status"] = rc
+    if raise_on_error:
+        _check(rc, "pyramidsd_verify_ex")
     return out
 
 

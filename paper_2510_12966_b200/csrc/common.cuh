@@ -68,6 +68,10 @@ struct StageParams {
   // memory mapped into the device), where the host reads them to choose its schedule for later calls.
   int32_t* fill_out;
   int fill_cap;
+  // Index of this call's sequence 0 in the whole batch: row (b, k) draws with Philox counter word 0 =
+  // (seq_base + b) * K + k and sequence b's bonus draw with seq_base + b, so a slice of a batch draws what the
+  // whole batch draws.
+  long long seq_base;
 };
 
 // ---- special functions (single MUFU instruction each) -------------------------------------------------

@@ -112,7 +112,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
       st = P.stats[r];
       const int x = (tokens_given != nullptr) ? (lane < n_given ? tokens_given[lane] : 0) : P.tokens[r];
       flags = st.flags | ((x < 0 || x >= V) ? kFlagTokenRange : 0);
-      row_uniforms(P.seed, P.offset, static_cast<unsigned>(r), &u, &u2);
+      row_uniforms(P.seed, P.offset, static_cast<unsigned>((P.seq_base + b) * K + lane), &u, &u2);
       const float nanf_ = __int_as_float(0x7fc00000);
       float px = nanf_, qx = nanf_;
       bool coin_ok = false;
@@ -204,7 +204,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
         sh_m2l = m2; sh_l2sl = lg2_approx(sum);
         sh_m2s = m2; sh_l2ss = sh_l2sl;
         sh_resid = 0.f;   // weights are p_large itself
-        sh_u2 = bonus_uniform(P.seed, P.offset, static_cast<unsigned>(b));
+        sh_u2 = bonus_uniform(P.seed, P.offset, static_cast<unsigned>(P.seq_base + b));
       }
       __syncthreads();
       need_draw = true;
@@ -229,6 +229,11 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
     // the tiles of a batch are independent (their loads overlap); each warp leaves its sum per tile, then one
     // thread per tile adds the 32 warp sums in warp order and hands the total to every CTA of the cluster.
     const int my_tiles = (n_tiles - static_cast<int>(cl_rank) + CL - 1) / CL;
+    // A second go happens only when the residual weights, taken again here in single precision, all come out
+    // zero although the row's residual mass did not (two rows that differ only where both probabilities
+    // underflow): the draw then comes from p_large, as for a zero residual, so a rejected row with a
+    // distribution always yields a token.
+    for (int attempt = 0; attempt < 2; ++attempt) {
     for (int m0 = 0; m0 < my_tiles; m0 += kFinBatch) {
       const int nb = min(kFinBatch, my_tiles - m0);
 #pragma unroll 4
@@ -260,6 +265,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
       double total = 0.0;
       for (int j = 0; j < n_tiles; ++j) total += tile_total[j];
       const double target = static_cast<double>(sh_u2) * total;
+      const bool redo = !(total > 0.0) && !row.from_large;
       // first tile whose inclusive cumulative weight exceeds the target; else the last non-empty tile
       int pick = -1, last_pos = -1;
       double cum = 0.0, cum_before_pick = 0.0, cum_before_last = 0.0;
@@ -270,11 +276,16 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
         cum = nxt;
       }
       if (pick < 0) { pick = last_pos; cum_before_pick = cum_before_last; }
-      sh_tile = pick;
+      sh_tile = redo ? -2 : pick;
       sh_token = -1;
       sh_target = static_cast<float>(target - cum_before_pick);
     }
     __syncthreads();
+    if (sh_tile != -2) break;
+    row.from_large = true;            // every CTA of the cluster holds the same totals and takes the same turn
+    if (CL > 1) fin_cluster_sync();   // nobody posts new totals while a peer still reads the old ones
+    __syncthreads();
+    }
     const int tile = sh_tile;
     writer = (CL > 1 && tile >= 0) ? static_cast<unsigned>(tile % CL) : 0u;   // the CTA that summed the chosen tile goes on
     if (tile >= 0 && cl_rank == writer) {

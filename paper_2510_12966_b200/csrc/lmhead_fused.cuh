@@ -499,6 +499,7 @@ struct LmFinalParams {
   float threshold;
   int mode;
   unsigned long long seed, offset;
+  long long seq_base;   // index of sequence 0 in the whole batch (Philox row counter)
   int32_t* out_accept_len;
   int32_t* out_next_token;
   float* out_div;        // [B, K] or null
@@ -567,7 +568,7 @@ __global__ void __launch_bounds__(256) lmhead_final_kernel(const LmFinalParams F
     bool acc = true;
     float u = 0.f, uu2 = 0.f;
     if (lane < K) {
-      row_uniforms(F.seed, F.offset, static_cast<unsigned>(b * K + lane), &u, &uu2);
+      row_uniforms(F.seed, F.offset, static_cast<unsigned>((F.seq_base + b) * K + lane), &u, &uu2);
       const float px = sh_px[lane], qx = sh_qx[lane];
       const float rho = (qx > 0.f) ? __fdiv_rn(px, qx) : (px > 0.f ? INFINITY : 0.f);
       const bool coin_ok = u < fminf(1.f, rho);

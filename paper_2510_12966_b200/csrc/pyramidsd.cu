@@ -2,6 +2,7 @@
 // management and kernel launches. No torch types, no CPU fallback: every step of the path runs in the
 // kernels of this directory.
 #include "../../include/pyramidsd.h"
+#include "../../include/pyramidsd_diag.h"
 
 #include <atomic>
 #include <cmath>
@@ -22,7 +23,7 @@ using psd::StageParams;
 
 std::atomic<uint64_t> g_launches{0};
 thread_local cudaStream_t t_stream = nullptr;
-thread_local int t_two_stage_policy = PSD_TWO_STAGE_FUSED;
+thread_local int t_two_stage_policy = PSD_TWO_STAGE_AUTO;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
@@ -38,28 +39,40 @@ std::mutex g_noalloc_mu;
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-// Library-owned scratch of one device: workspace for calls that bring none, the status word, and the
-// staging buffers of the host-pointer entry point. Grown on demand, never shrunk, freed at process exit
-// by the driver.
-struct DeviceState {
+// Library-owned scratch. Every (device, stream) pair that has been used without a caller workspace owns its own
+// buffers: the workspace of the stage / pyramid calls, the status word of the bounded waits, the staging
+// buffers of the host-pointer entry point and the partial sums of the fused LM-head. A call touches only the
+// buffers of the stream it runs on and holds that entry's mutex while it enqueues, so two host threads on two
+// streams share nothing and two threads on one stream take turns. Buffers are grown on demand (after waiting
+// for the stream's own earlier work, which is all that can still use them), never shrunk, and freed at
+// process exit by the driver.
+struct StreamScratch {
   std::mutex mu;
+  bool used = false;
+  cudaStream_t stream = nullptr;
   void* ws = nullptr;
   size_t ws_bytes = 0;
   int* status = nullptr;
   void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
   size_t stage_bytes[4] = {0, 0, 0, 0};
-  int32_t* out4 = nullptr;  // 4 x [B] results of the host entry point
-  size_t out4_elems = 0;
+  void* out4 = nullptr;     // 4 x [B] results of the host entry point
+  size_t out4_bytes = 0;
   void* lm_ws = nullptr;    // partial sums of the fused LM-head path
   size_t lm_ws_bytes = 0;
+};
+struct DeviceState {
+  std::mutex mu;
+  StreamScratch streams[PSD_MAX_STREAMS];
   // PSD_TWO_STAGE_AUTO: window lengths of a recent call, written by the stage-1 finalisation straight into
-  // mapped host memory
+  // mapped host memory (a hint for the schedule only: racing writers cannot change any result)
   int32_t* fill_host = nullptr;
   int32_t* fill_dev = nullptr;
   int fill_B = 0, fill_Kq = 0;   // the shape those lengths belong to
 };
 constexpr int kFillCap = 4096;
 DeviceState g_dev[kMaxDevices];
+// what pyramidsd_last_status() looks at: the scratch entry of this thread's most recent call
+thread_local StreamScratch* t_last_scratch = nullptr;
 
 int current_device_state(DeviceState** out) {
   int dev = 0;
@@ -68,23 +81,47 @@ int current_device_state(DeviceState** out) {
   return PSD_OK;
 }
 
-int grow(void** ptr, size_t* have, size_t want) {
+// The scratch entry of `stream` on the current device, created on first use; its status word exists on return.
+int scratch_for(cudaStream_t stream, StreamScratch** out) {
+  DeviceState* ds = nullptr;
+  int rc = current_device_state(&ds);
+  if (rc != PSD_OK) return rc;
+  StreamScratch* ss = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(ds->mu);
+    for (auto& e : ds->streams)
+      if (e.used && e.stream == stream) { ss = &e; break; }
+    if (ss == nullptr)
+      for (auto& e : ds->streams)
+        if (!e.used) { e.used = true; e.stream = stream; ss = &e; break; }
+  }
+  if (ss == nullptr) {
+    std::fprintf(stderr, "pyramidsd: more than %d streams in use on this device; supply a workspace\n", PSD_MAX_STREAMS);
+    return PSD_ERR_WORKSPACE;
+  }
+  *out = ss;
+  return PSD_OK;
+}
+
+// with ss->mu held
+int ensure_status(StreamScratch* ss) {
+  if (ss->status) return PSD_OK;
+  if (cudaMalloc(reinterpret_cast<void**>(&ss->status), kAlign) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
+  if (cudaMemset(ss->status, 0, kAlign) != cudaSuccess) return PSD_ERR_CUDA;
+  return PSD_OK;
+}
+
+// with ss->mu held: only work already enqueued on ss->stream can still use the old buffer
+int grow(StreamScratch* ss, void** ptr, size_t* have, size_t want) {
   if (*have >= want) return PSD_OK;
   if (*ptr) {
-    if (cudaDeviceSynchronize() != cudaSuccess) return PSD_ERR_CUDA;
+    if (cudaStreamSynchronize(ss->stream) != cudaSuccess) return PSD_ERR_CUDA;
     cudaFree(*ptr);
     *ptr = nullptr;
     *have = 0;
   }
   if (cudaMalloc(ptr, want) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
   *have = want;
-  return PSD_OK;
-}
-
-int ensure_status(DeviceState* ds) {
-  if (ds->status) return PSD_OK;
-  if (cudaMalloc(reinterpret_cast<void**>(&ds->status), kAlign) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
-  if (cudaMemset(ds->status, 0, kAlign) != cudaSuccess) return PSD_ERR_CUDA;
   return PSD_OK;
 }
 
@@ -152,15 +189,17 @@ int check_launch() {
   return PSD_OK;
 }
 
-// Statistics pass for one stage: picks the kernel variant and launches it.
-int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_size, cudaStream_t stream) {
+// Statistics pass for one stage: picks the kernel variant and launches it. `allow_triples`: a wrapper launch may
+// walk its rows as (draft, qualifier, target) triples where the geometry streams them twice.
+int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_size, cudaStream_t stream,
+                    bool allow_triples = false) {
   const long long rows = static_cast<long long>(P.B) * P.K;
   if (rows == 0 && P.K2 == 0) return PSD_OK;
   bool use_cluster = false;
   psd::ClusterGeom geom{};
-  if (variant == PSD_KERNEL_CLUSTER || variant == PSD_KERNEL_AUTO) {
-    use_cluster = psd::cluster_geometry(P, dtype, cluster_size, &geom);
-    if (!use_cluster && variant == PSD_KERNEL_CLUSTER) return PSD_ERR_UNSUPPORTED;
+  if (variant != PSD_KERNEL_BASELINE) {
+    use_cluster = psd::cluster_geometry(P, dtype, cluster_size, variant == PSD_KERNEL_CLUSTER_STREAMED, allow_triples, &geom);
+    if (!use_cluster && variant != PSD_KERNEL_AUTO) return PSD_ERR_UNSUPPORTED;
   }
   TimedLaunch timed(stream, 0);
   if (use_cluster) {
@@ -240,7 +279,9 @@ int validate_stage(const psd_stage_args* a) {
   if (a == nullptr || a->struct_size != sizeof(psd_stage_args)) return PSD_ERR_INVALID_ARG;
   if (!valid_dtype(a->dtype) || !valid_mode(a->mode) || !valid_div(a->div_kind)) return PSD_ERR_INVALID_ARG;
   if (a->B < 0 || a->K < 0 || a->K > 32 || a->V < 1) return PSD_ERR_INVALID_ARG;
-  if (a->kernel_variant < PSD_KERNEL_AUTO || a->kernel_variant > PSD_KERNEL_CLUSTER || a->cluster_size < 0) return PSD_ERR_INVALID_ARG;
+  if (a->kernel_variant < PSD_KERNEL_AUTO || a->kernel_variant > PSD_KERNEL_CLUSTER_STREAMED || a->cluster_size < 0) return PSD_ERR_INVALID_ARG;
+  if (a->kernel_variant == PSD_KERNEL_CLUSTER_STREAMED && a->cluster_size == 0) return PSD_ERR_INVALID_ARG;
+  if (a->seq_index_base < 0 || a->reserved0 != 0) return PSD_ERR_INVALID_ARG;
   if (a->V > kMaxV) return PSD_ERR_UNSUPPORTED;
   if (static_cast<long long>(a->B) * a->K > (1ll << 30)) return PSD_ERR_UNSUPPORTED;
   if (a->inv_temperature < 0.f || std::isnan(a->inv_temperature) || std::isinf(a->inv_temperature)) return PSD_ERR_INVALID_ARG;
@@ -292,6 +333,7 @@ StageParams make_params(const psd_stage_args* a, void* ws, int* status) {
   P.n_window = nullptr;
   P.K_window = 0;
   P.status = status;
+  P.seq_base = a->seq_index_base;
   return P;
 }
 
@@ -300,34 +342,24 @@ cudaStream_t pick_stream(const psd_stage_args* a) {
   return t_stream;
 }
 
-// Runs one stage; `window_out`/`n_window_out`/`K_window` non-null make the finalisation also build the
-// stage-2 window of the wrapper.
-int run_stage(const psd_stage_args* a, int32_t* window_out, int32_t* n_window_out, int K_window,
-              int32_t* fill_out = nullptr) {
-  int rc = validate_stage(a);
-  if (rc != PSD_OK) return rc;
-  if (a->B == 0) return PSD_OK;
-  DeviceState* ds = nullptr;
-  rc = current_device_state(&ds);
+// Runs one stage with the scratch entry `ss` (held by the caller); `window_out`/`n_window_out`/`K_window` non-null
+// make the finalisation also build the stage-2 window of the wrapper.
+int run_stage_locked(const psd_stage_args* a, StreamScratch* ss, cudaStream_t stream, int32_t* window_out,
+                     int32_t* n_window_out, int K_window, int32_t* fill_out = nullptr) {
+  int rc = ensure_status(ss);
   if (rc != PSD_OK) return rc;
   void* ws = a->workspace;
-  {
-    std::lock_guard<std::mutex> lock(ds->mu);
-    rc = ensure_status(ds);
+  if (ws == nullptr) {
+    rc = grow(ss, &ss->ws, &ss->ws_bytes, stage_workspace_bytes(a->B, a->K));
     if (rc != PSD_OK) return rc;
-    if (ws == nullptr) {
-      rc = grow(&ds->ws, &ds->ws_bytes, stage_workspace_bytes(a->B, a->K));
-      if (rc != PSD_OK) return rc;
-      ws = ds->ws;
-    }
+    ws = ss->ws;
   }
-  StageParams P = make_params(a, ws, ds->status);
+  StageParams P = make_params(a, ws, ss->status);
   P.window = window_out;
   P.n_window = n_window_out;
   P.K_window = K_window;
   P.fill_out = fill_out;
   P.fill_cap = kFillCap;
-  const cudaStream_t stream = pick_stream(a);
   if (a->K > 0) {
     rc = launch_rowstats(P, a->dtype, a->kernel_variant, a->cluster_size, stream);
     if (rc != PSD_OK) return rc;
@@ -335,69 +367,108 @@ int run_stage(const psd_stage_args* a, int32_t* window_out, int32_t* n_window_ou
   return launch_finalize(P, a->dtype, stream);
 }
 
-int verify_two_stage(const void* logits_draft, const void* logits_qual, const void* logits_target,
-                     const int32_t* draft_tokens, int B, int K_d, int K_q, int V, int dtype, float tau_q,
-                     float tau_t, int mode, uint64_t seed, uint64_t offset, int32_t* out_accept_len_q,
-                     int32_t* out_next_token_q, int32_t* out_accept_len, int32_t* out_next_token,
-                     cudaStream_t stream, int variant, bool bonus = false) {
-  if (K_q < 1 || K_d < K_q || K_d > 32 || B < 0 || V < 1) return PSD_ERR_INVALID_ARG;
-  if (B == 0) return PSD_OK;
+int run_stage(const psd_stage_args* a) {
+  int rc = validate_stage(a);
+  if (rc != PSD_OK) return rc;
+  if (a->B == 0) return PSD_OK;
+  const cudaStream_t stream = pick_stream(a);
+  StreamScratch* ss = nullptr;
+  rc = scratch_for(stream, &ss);
+  if (rc != PSD_OK) return rc;
+  std::lock_guard<std::mutex> lock(ss->mu);
+  t_last_scratch = ss;
+  return run_stage_locked(a, ss, stream, nullptr, nullptr, 0);
+}
+
+size_t pyramid_workspace_bytes(int B, int K_d, int K_q) { return stage_workspace_bytes(B, K_d) + stage_workspace_bytes(B, K_q); }
+
+int validate_pyramid(const psd_pyramid_args* a) {
+  if (a == nullptr || a->struct_size != sizeof(psd_pyramid_args)) return PSD_ERR_INVALID_ARG;
+  if (!valid_dtype(a->dtype) || !valid_mode(a->mode_q) || !valid_mode(a->mode_t) || !valid_div(a->div_kind)) return PSD_ERR_INVALID_ARG;
+  if (a->K_q < 1 || a->K_d < a->K_q || a->K_d > 32 || a->B < 0 || a->V < 1) return PSD_ERR_INVALID_ARG;
+  if (a->schedule < PSD_TWO_STAGE_DEFAULT || a->schedule > PSD_TWO_STAGE_FUSED_ROWS) return PSD_ERR_INVALID_ARG;
+  if (a->kernel_variant != PSD_KERNEL_AUTO && a->kernel_variant != PSD_KERNEL_BASELINE) return PSD_ERR_INVALID_ARG;
+  if (a->target_has_bonus_row != 0 && a->target_has_bonus_row != 1) return PSD_ERR_INVALID_ARG;
+  if (a->seq_index_base < 0) return PSD_ERR_INVALID_ARG;
+  if (a->B > 0 && (!a->logits_draft || !a->logits_qual || !a->logits_target || !a->draft_tokens || !a->out_accept_len_q ||
+                   !a->out_next_token_q || !a->out_accept_len || !a->out_next_token))
+    return PSD_ERR_INVALID_ARG;
+  if (a->workspace != nullptr) {
+    if ((reinterpret_cast<uintptr_t>(a->workspace) % kAlign) != 0) return PSD_ERR_WORKSPACE;
+    if (a->workspace_bytes < pyramid_workspace_bytes(a->B, a->K_d, a->K_q)) return PSD_ERR_WORKSPACE;
+  }
+  return PSD_OK;
+}
+
+// Both stages of the pyramid with the scratch entry `ss` held by the caller.
+int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, cudaStream_t stream) {
+  const int B = a->B, K_d = a->K_d, K_q = a->K_q, V = a->V, dtype = a->dtype;
   DeviceState* ds = nullptr;
   int rc = current_device_state(&ds);
   if (rc != PSD_OK) return rc;
-  // scratch: [stage-1 workspace][stage-2 workspace]; the window and its length live in stage 1's tail
+  rc = ensure_status(ss);
+  if (rc != PSD_OK) return rc;
+  // scratch: [stage-1 workspace][stage-2 workspace]; the window and its length live in stage 1's tail unless the
+  // caller wants them
   const size_t ws1 = stage_workspace_bytes(B, K_d), ws2 = stage_workspace_bytes(B, K_q);
-  char* base = nullptr;
-  {
-    std::lock_guard<std::mutex> lock(ds->mu);
-    rc = grow(&ds->ws, &ds->ws_bytes, ws1 + ws2);
+  char* base = static_cast<char*>(a->workspace);
+  if (base == nullptr) {
+    rc = grow(ss, &ss->ws, &ss->ws_bytes, ws1 + ws2);
     if (rc != PSD_OK) return rc;
-    base = static_cast<char*>(ds->ws);
+    base = static_cast<char*>(ss->ws);
   }
   int32_t* window = reinterpret_cast<int32_t*>(base + stats_bytes(static_cast<long long>(B) * K_d));
   int32_t* n_window = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(window) + align_up(static_cast<size_t>(B) * K_d * 4));
+  if (a->out_window != nullptr) window = a->out_window;
+  if (a->out_n_window != nullptr) n_window = a->out_n_window;
 
   psd_stage_args s1;
   std::memset(&s1, 0, sizeof(s1));
   s1.struct_size = sizeof(s1);
   s1.dtype = dtype;
-  s1.logits_small = logits_draft;
-  s1.logits_large = logits_qual;
-  s1.tokens = draft_tokens;
+  s1.logits_small = a->logits_draft;
+  s1.logits_large = a->logits_qual;
+  s1.tokens = a->draft_tokens;
   s1.B = B; s1.K = K_d; s1.V = V;
-  s1.mode = mode;
-  s1.div_kind = PSD_DIV_JS;
-  s1.threshold = tau_q;
-  s1.philox_seed = seed;
-  s1.philox_offset = offset;
-  s1.out_accept_len = out_accept_len_q;
-  s1.out_next_token = out_next_token_q;
+  s1.mode = a->mode_q;
+  s1.div_kind = a->div_kind;
+  s1.inv_temperature = a->inv_temperature;
+  s1.threshold = a->tau_q;
+  s1.philox_seed = a->philox_seed;
+  s1.philox_offset = a->philox_offset;
+  s1.seq_index_base = a->seq_index_base;
+  s1.out_accept_len = a->out_accept_len_q;
+  s1.out_next_token = a->out_next_token_q;
+  s1.out_div = a->out_div_q;
+  s1.out_resid_mass = a->out_resid_q;
   s1.workspace = base;
   s1.workspace_bytes = ws1;
-  s1.stream = stream;
-  s1.use_stream_field = 1;
-  s1.kernel_variant = variant;
+  s1.kernel_variant = a->kernel_variant;
   psd_stage_args s2 = s1;
-  s2.logits_small = logits_qual;   // P_MQ takes the place of P_MD in the target comparison (Fig. 1)
-  s2.logits_large = logits_target;
+  s2.logits_small = a->logits_qual;   // P_MQ takes the place of P_MD in the target comparison (Fig. 1)
+  s2.logits_large = a->logits_target;
   s2.seq_stride_small = static_cast<int64_t>(K_d) * V;  // rows 0..K_q-1 of each [K_d, V] qualifier sequence
   s2.seq_stride_large = 0;
-  s2.large_has_bonus_row = bonus ? 1 : 0;   // target [B, K_q + 1, V]: its last row per sequence is the bonus row
+  s2.large_has_bonus_row = a->target_has_bonus_row;   // target [B, K_q + 1, V]: its last row per sequence is the bonus row
   s2.tokens = window;
   s2.n_valid = n_window;
   s2.K = K_q;
-  s2.threshold = tau_t;
-  s2.philox_offset = offset + 1;
-  s2.out_accept_len = out_accept_len;
-  s2.out_next_token = out_next_token;
+  s2.mode = a->mode_t;
+  s2.threshold = a->tau_t;
+  s2.philox_offset = a->philox_offset + 1;
+  s2.out_accept_len = a->out_accept_len;
+  s2.out_next_token = a->out_next_token;
+  s2.out_div = a->out_div_t;
+  s2.out_resid_mass = a->out_resid_t;
   s2.workspace = base + ws1;
   s2.workspace_bytes = ws2;
   rc = validate_stage(&s1);
   if (rc == PSD_OK) rc = validate_stage(&s2);
   if (rc != PSD_OK) return rc;
-  bool separate = t_two_stage_policy == PSD_TWO_STAGE_SEPARATE;
+  const int policy = a->schedule != PSD_TWO_STAGE_DEFAULT ? a->schedule : t_two_stage_policy;
+  bool separate = policy == PSD_TWO_STAGE_SEPARATE;
   int32_t* fill_out = nullptr;
-  if (t_two_stage_policy == PSD_TWO_STAGE_AUTO) {
+  if (policy == PSD_TWO_STAGE_AUTO) {
     std::lock_guard<std::mutex> lock(ds->mu);
     if (ds->fill_host == nullptr) {
       void* h = nullptr;
@@ -428,6 +499,7 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
       fill_out = ds->fill_dev;
     }
   }
+  const int variant = a->kernel_variant;
   if (separate) {
     // stage by stage: stage 2's statistics run after stage 1 has fixed the windows and skip the rows beyond them.
     // Both launches take the cluster size the single-launch schedule would pick, so a row's vocabulary is
@@ -439,28 +511,23 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
       PS.seq_stride_small2 = Q.seq_stride_small; PS.seq_stride_large2 = Q.seq_stride_large;
       PS.K2 = K_q;
       psd::ClusterGeom g{};
-      if (variant != PSD_KERNEL_BASELINE && psd::cluster_geometry(PS, dtype, 0, &g)) s1.cluster_size = s2.cluster_size = g.cs;
+      if (variant != PSD_KERNEL_BASELINE && psd::cluster_geometry(PS, dtype, 0, false, false, &g)) s1.cluster_size = s2.cluster_size = g.cs;
     }
-    rc = run_stage(&s1, window, n_window, K_q, fill_out);
+    rc = run_stage_locked(&s1, ss, stream, window, n_window, K_q, fill_out);
     if (rc != PSD_OK) return rc;
-    return run_stage(&s2, nullptr, nullptr, 0);
-  }
-  {
-    std::lock_guard<std::mutex> lock(ds->mu);
-    rc = ensure_status(ds);
-    if (rc != PSD_OK) return rc;
+    return run_stage_locked(&s2, ss, stream, nullptr, nullptr, 0);
   }
   // Two launches for the whole pyramid. The statistics of both stages are independent of the stage-1
   // outcome (only the token looked up in a row and the window length depend on it), so one launch of
   // the statistics kernel covers the B*K_d stage-1 rows and the B*K_q stage-2 rows; one finalisation
   // kernel then runs stage 1, builds the window, and runs stage 2 per sequence.
-  StageParams P1 = make_params(&s1, s1.workspace, ds->status);
+  StageParams P1 = make_params(&s1, s1.workspace, ss->status);
   P1.window = window;
   P1.n_window = n_window;
   P1.K_window = K_q;
   P1.fill_out = fill_out;
   P1.fill_cap = kFillCap;
-  const StageParams P2 = make_params(&s2, s2.workspace, ds->status);
+  const StageParams P2 = make_params(&s2, s2.workspace, ss->status);
   StageParams PS = P1;
   PS.small2 = P2.small;
   PS.large2 = P2.large;
@@ -468,13 +535,13 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   PS.seq_stride_large2 = P2.seq_stride_large;
   PS.K2 = K_q;
   PS.stats2 = P2.stats;
-  rc = launch_rowstats(PS, dtype, variant, 0, stream);
+  rc = launch_rowstats(PS, dtype, variant, 0, stream, policy == PSD_TWO_STAGE_FUSED_ROWS);
   if (rc != PSD_OK) return rc;
   {
     TimedLaunch timed(stream, 1);
     cudaError_t e;
-    if (mode == PSD_FUZZY) {
-      // threshold-only acceptance: stage 2 does not depend on stage 1's drawn token, the stages run side by side
+    if (a->mode_q == PSD_FUZZY && a->mode_t == PSD_FUZZY) {
+      // threshold-only acceptance in both stages: stage 2 needs nothing of stage 1's drawn token, the stages run side by side
       const int cl = fin_cluster_size(2ll * B);
       if (dtype == PSD_F32) e = PSD_FIN_DISPATCH(finalize_pyramid_split_kernel, float, cl, 2u * B, stream, P1, P2);
       else e = PSD_FIN_DISPATCH(finalize_pyramid_split_kernel, __nv_bfloat16, cl, 2u * B, stream, P1, P2);
@@ -489,11 +556,49 @@ int verify_two_stage(const void* logits_draft, const void* logits_qual, const vo
   return check_launch();
 }
 
+cudaStream_t pick_stream(const psd_pyramid_args* a) {
+  if (a->stream != nullptr || a->use_stream_field) return static_cast<cudaStream_t>(a->stream);
+  return t_stream;
+}
+
+int verify_two_stage(const psd_pyramid_args* a) {
+  int rc = validate_pyramid(a);
+  if (rc != PSD_OK) return rc;
+  if (a->B == 0) return PSD_OK;
+  const cudaStream_t stream = pick_stream(a);
+  StreamScratch* ss = nullptr;
+  rc = scratch_for(stream, &ss);
+  if (rc != PSD_OK) return rc;
+  std::lock_guard<std::mutex> lock(ss->mu);
+  t_last_scratch = ss;
+  return verify_two_stage_locked(a, ss, stream);
+}
+
+psd_pyramid_args basic_pyramid_args(const void* logits_draft, const void* logits_qual, const void* logits_target,
+                                    const int32_t* draft_tokens, int B, int K_d, int K_q, int V, int dtype, float tau_q,
+                                    float tau_t, int mode, uint64_t seed, uint64_t offset, int32_t* out_accept_len_q,
+                                    int32_t* out_next_token_q, int32_t* out_accept_len, int32_t* out_next_token) {
+  psd_pyramid_args a;
+  std::memset(&a, 0, sizeof(a));
+  a.struct_size = sizeof(a);
+  a.dtype = dtype;
+  a.logits_draft = logits_draft; a.logits_qual = logits_qual; a.logits_target = logits_target;
+  a.draft_tokens = draft_tokens;
+  a.B = B; a.K_d = K_d; a.K_q = K_q; a.V = V;
+  a.mode_q = a.mode_t = mode;
+  a.tau_q = tau_q; a.tau_t = tau_t;
+  a.div_kind = PSD_DIV_JS;
+  a.philox_seed = seed; a.philox_offset = offset;
+  a.out_accept_len_q = out_accept_len_q; a.out_next_token_q = out_next_token_q;
+  a.out_accept_len = out_accept_len; a.out_next_token = out_next_token;
+  return a;
+}
+
 }  // namespace
 
 extern "C" {
 
-int pyramidsd_verify_stage_ex(const psd_stage_args* args) { return run_stage(args, nullptr, nullptr, 0); }
+int pyramidsd_verify_stage_ex(const psd_stage_args* args) { return run_stage(args); }
 
 int pyramidsd_verify_stage(const void* logits_small, const void* logits_large, const int32_t* draft_tokens,
                            int B, int K, int V, psd_dtype dtype, float threshold, psd_mode mode,
@@ -514,21 +619,20 @@ int pyramidsd_verify_stage(const void* logits_small, const void* logits_large, c
   a.philox_offset = offset;
   a.out_accept_len = out_accept_len;
   a.out_next_token = out_next_token;
-  return run_stage(&a, nullptr, nullptr, 0);
+  return run_stage(&a);
 }
+
+int pyramidsd_verify_ex(const psd_pyramid_args* args) { return verify_two_stage(args); }
 
 int pyramidsd_verify(const void* logits_draft, const void* logits_qual, const void* logits_target,
                      const int32_t* draft_tokens, int B, int K_d, int K_q, int V, psd_dtype dtype,
                      float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
                      int32_t* out_accept_len_q, int32_t* out_next_token_q, int32_t* out_accept_len,
                      int32_t* out_next_token) {
-  if (!valid_dtype(dtype) || !valid_mode(mode)) return PSD_ERR_INVALID_ARG;
-  if (B > 0 && (!logits_draft || !logits_qual || !logits_target || !draft_tokens || !out_accept_len_q ||
-                !out_next_token_q || !out_accept_len || !out_next_token))
-    return PSD_ERR_INVALID_ARG;
-  return verify_two_stage(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype, tau_q,
-                          tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q, out_accept_len,
-                          out_next_token, t_stream, PSD_KERNEL_AUTO);
+  const psd_pyramid_args a = basic_pyramid_args(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype,
+                                                tau_q, tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q,
+                                                out_accept_len, out_next_token);
+  return verify_two_stage(&a);
 }
 
 int pyramidsd_verify_bonus(const void* logits_draft, const void* logits_qual, const void* logits_target,
@@ -536,13 +640,11 @@ int pyramidsd_verify_bonus(const void* logits_draft, const void* logits_qual, co
                            float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
                            int32_t* out_accept_len_q, int32_t* out_next_token_q, int32_t* out_accept_len,
                            int32_t* out_next_token) {
-  if (!valid_dtype(dtype) || !valid_mode(mode)) return PSD_ERR_INVALID_ARG;
-  if (B > 0 && (!logits_draft || !logits_qual || !logits_target || !draft_tokens || !out_accept_len_q ||
-                !out_next_token_q || !out_accept_len || !out_next_token))
-    return PSD_ERR_INVALID_ARG;
-  return verify_two_stage(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype, tau_q,
-                          tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q, out_accept_len,
-                          out_next_token, t_stream, PSD_KERNEL_AUTO, true);
+  psd_pyramid_args a = basic_pyramid_args(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype,
+                                          tau_q, tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q,
+                                          out_accept_len, out_next_token);
+  a.target_has_bonus_row = 1;
+  return verify_two_stage(&a);
 }
 
 int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, const void* logits_target,
@@ -550,43 +652,36 @@ int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, con
                           float tau_q, float tau_t, psd_mode mode, uint64_t philox_seed, uint64_t offset,
                           int32_t* out_accept_len_q, int32_t* out_next_token_q, int32_t* out_accept_len,
                           int32_t* out_next_token) {
-  if (!valid_dtype(dtype) || !valid_mode(mode)) return PSD_ERR_INVALID_ARG;
-  if (K_q < 1 || K_d < K_q || K_d > 32 || B < 0 || V < 1) return PSD_ERR_INVALID_ARG;
-  if (B == 0) return PSD_OK;
-  if (!logits_draft || !logits_qual || !logits_target || !draft_tokens || !out_accept_len_q ||
-      !out_next_token_q || !out_accept_len || !out_next_token)
-    return PSD_ERR_INVALID_ARG;
-  DeviceState* ds = nullptr;
-  int rc = current_device_state(&ds);
+  psd_pyramid_args a = basic_pyramid_args(logits_draft, logits_qual, logits_target, draft_tokens, B, K_d, K_q, V, dtype,
+                                          tau_q, tau_t, mode, philox_seed, offset, out_accept_len_q, out_next_token_q,
+                                          out_accept_len, out_next_token);
+  int rc = validate_pyramid(&a);
   if (rc != PSD_OK) return rc;
+  if (B == 0) return PSD_OK;
+  const cudaStream_t s = t_stream;
+  StreamScratch* ss = nullptr;
+  rc = scratch_for(s, &ss);
+  if (rc != PSD_OK) return rc;
+  std::lock_guard<std::mutex> lock(ss->mu);
+  t_last_scratch = ss;
   const size_t es = elem_size(dtype);
   const size_t n_d = static_cast<size_t>(B) * K_d * V * es, n_t = static_cast<size_t>(B) * K_q * V * es;
   const size_t n_tok = static_cast<size_t>(B) * K_d * 4;
-  {
-    std::lock_guard<std::mutex> lock(ds->mu);
-    const size_t want[4] = {n_d, n_d, n_t, n_tok};
-    for (int i = 0; i < 4; ++i) {
-      rc = grow(&ds->stage[i], &ds->stage_bytes[i], want[i]);
-      if (rc != PSD_OK) return rc;
-    }
-    if (ds->out4_elems < static_cast<size_t>(4) * B) {
-      size_t have = ds->out4_elems * 4;
-      void* p = ds->out4;
-      rc = grow(&p, &have, static_cast<size_t>(4) * B * 4);
-      if (rc != PSD_OK) return rc;
-      ds->out4 = static_cast<int32_t*>(p);
-      ds->out4_elems = static_cast<size_t>(4) * B;
-    }
+  const size_t want[4] = {n_d, n_d, n_t, n_tok};
+  for (int i = 0; i < 4; ++i) {
+    rc = grow(ss, &ss->stage[i], &ss->stage_bytes[i], want[i]);
+    if (rc != PSD_OK) return rc;
   }
-  const cudaStream_t s = t_stream;
+  rc = grow(ss, &ss->out4, &ss->out4_bytes, static_cast<size_t>(4) * B * 4);
+  if (rc != PSD_OK) return rc;
   const void* src[4] = {logits_draft, logits_qual, logits_target, draft_tokens};
-  const size_t nbytes[4] = {n_d, n_d, n_t, n_tok};
   for (int i = 0; i < 4; ++i)
-    if (cudaMemcpyAsync(ds->stage[i], src[i], nbytes[i], cudaMemcpyHostToDevice, s) != cudaSuccess) return PSD_ERR_CUDA;
-  int32_t* o = ds->out4;
-  rc = verify_two_stage(ds->stage[0], ds->stage[1], ds->stage[2], static_cast<const int32_t*>(ds->stage[3]), B, K_d,
-                        K_q, V, dtype, tau_q, tau_t, mode, philox_seed, offset, o, o + B, o + 2 * B, o + 3 * B, s,
-                        PSD_KERNEL_AUTO);
+    if (cudaMemcpyAsync(ss->stage[i], src[i], want[i], cudaMemcpyHostToDevice, s) != cudaSuccess) return PSD_ERR_CUDA;
+  int32_t* o = static_cast<int32_t*>(ss->out4);
+  a.logits_draft = ss->stage[0]; a.logits_qual = ss->stage[1]; a.logits_target = ss->stage[2];
+  a.draft_tokens = static_cast<const int32_t*>(ss->stage[3]);
+  a.out_accept_len_q = o; a.out_next_token_q = o + B; a.out_accept_len = o + 2 * B; a.out_next_token = o + 3 * B;
+  rc = verify_two_stage_locked(&a, ss, s);
   if (rc != PSD_OK) return rc;
   int32_t* dst[4] = {out_accept_len_q, out_next_token_q, out_accept_len, out_next_token};
   for (int i = 0; i < 4; ++i)
@@ -658,10 +753,21 @@ int pyramidsd_verify_stage_noalloc(const void* logits_small, const void* logits_
   return PSD_OK;
 }
 
-int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const void* logits_small,
-                                  const int32_t* tokens, int B, int K, int d_model, int V, float threshold,
-                                  psd_mode mode, uint64_t philox_seed, uint64_t offset, int32_t* out_accept_len,
-                                  int32_t* out_next_token, float* out_div, float* out_resid_mass, void* cuda_stream) {
+int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args) {
+  if (args == nullptr || args->struct_size != sizeof(psd_lmhead_args)) return PSD_ERR_INVALID_ARG;
+  if (args->tile_variant < PSD_LMHEAD_TILES_AUTO || args->tile_variant > PSD_LMHEAD_TILES_ONE_SM || args->seq_index_base < 0) return PSD_ERR_INVALID_ARG;
+  const void* hidden = args->hidden;
+  const void* w_t = args->w_t;
+  const void* logits_small = args->logits_small;
+  const int32_t* tokens = args->tokens;
+  const int B = args->B, K = args->K, d_model = args->d_model, V = args->V, mode = args->mode;
+  const float threshold = args->threshold;
+  const uint64_t philox_seed = args->philox_seed, offset = args->philox_offset;
+  int32_t* out_accept_len = args->out_accept_len;
+  int32_t* out_next_token = args->out_next_token;
+  float* out_div = args->out_div;
+  float* out_resid_mass = args->out_resid_mass;
+  void* cuda_stream = args->stream;
   if (!valid_mode(mode) || B < 0 || K < 0 || K > 32 || V < 1 || d_model < 1 || std::isnan(threshold)) return PSD_ERR_INVALID_ARG;
   const long long M = static_cast<long long>(B) * K;
   if ((d_model % psd::kLmK) != 0) return PSD_ERR_UNSUPPORTED;
@@ -676,19 +782,18 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
     if (cudaMemsetAsync(out_next_token, 0xff, static_cast<size_t>(B) * 4, stream) != cudaSuccess) return PSD_ERR_CUDA;
     return PSD_OK;
   }
-  DeviceState* ds = nullptr;
-  int rc = current_device_state(&ds);
+  StreamScratch* ss = nullptr;
+  int rc = scratch_for(stream, &ss);
   if (rc != PSD_OK) return rc;
+  std::lock_guard<std::mutex> lock(ss->mu);
+  t_last_scratch = ss;
   const int n_tiles = (V + psd::kLmN - 1) / psd::kLmN;
   const size_t per = static_cast<size_t>(M) * n_tiles;
   const size_t bytes = align_up(per * sizeof(float2)) * 2 + align_up(per * sizeof(float4)) + align_up(static_cast<size_t>(M) * sizeof(float4));
-  {
-    std::lock_guard<std::mutex> lock(ds->mu);
-    rc = ensure_status(ds);
-    if (rc != PSD_OK) return rc;
-    rc = grow(&ds->lm_ws, &ds->lm_ws_bytes, bytes);
-    if (rc != PSD_OK) return rc;
-  }
+  rc = ensure_status(ss);
+  if (rc != PSD_OK) return rc;
+  rc = grow(ss, &ss->lm_ws, &ss->lm_ws_bytes, bytes);
+  if (rc != PSD_OK) return rc;
   // tensor maps: hidden [M, d] and W^T [V, d], bf16, K innermost, boxes of 64 x 256 / 64 x 128, 128-byte swizzle
   typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -713,7 +818,7 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
   }
-  char* ws = static_cast<char*>(ds->lm_ws);
+  char* ws = static_cast<char*>(ss->lm_ws);
   psd::LmParams L{};
   L.small = static_cast<const __nv_bfloat16*>(logits_small);
   L.tokens = tokens;
@@ -723,7 +828,7 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
   L.part_small = reinterpret_cast<float2*>(ws); ws += align_up(per * sizeof(float2));
   L.part_div = reinterpret_cast<float4*>(ws); ws += align_up(per * sizeof(float4));
   L.row_lse = reinterpret_cast<float4*>(ws);
-  L.status = ds->status;
+  L.status = ss->status;
   static bool attr_set[kMaxDevices] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -737,8 +842,8 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
   }
   int sms = psd::cluster_sm_count();
   if (sms <= 0) sms = 1;
-  // the two-SM (cta_group::2) sweeps are the default; PYRAMIDSD_LMHEAD_PAIR=0 selects the one-SM variant
-  static const bool use_pair = [] { const char* e = std::getenv("PYRAMIDSD_LMHEAD_PAIR"); return !(e && std::atoi(e) == 0); }();
+  // the two-SM (cta_group::2) sweeps are the default
+  const bool use_pair = args->tile_variant != PSD_LMHEAD_TILES_ONE_SM;
   if (use_pair) {
     static bool pair_attr[kMaxDevices] = {};
     if (!pair_attr[dev]) {
@@ -809,6 +914,7 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
   F.threshold = threshold;
   F.mode = mode;
   F.seed = philox_seed; F.offset = offset;
+  F.seq_base = args->seq_index_base;
   F.out_accept_len = out_accept_len;
   F.out_next_token = out_next_token;
   F.out_div = out_div;
@@ -819,6 +925,24 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
   }
   g_launches.fetch_add(2 + 2 * static_cast<uint64_t>((M + psd::kLmM - 1) / psd::kLmM), std::memory_order_relaxed);
   return check_launch();
+}
+
+int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const void* logits_small,
+                                  const int32_t* tokens, int B, int K, int d_model, int V, float threshold,
+                                  psd_mode mode, uint64_t philox_seed, uint64_t offset, int32_t* out_accept_len,
+                                  int32_t* out_next_token, float* out_div, float* out_resid_mass, void* cuda_stream) {
+  psd_lmhead_args a;
+  std::memset(&a, 0, sizeof(a));
+  a.struct_size = sizeof(a);
+  a.hidden = hidden; a.w_t = w_t; a.logits_small = logits_small; a.tokens = tokens;
+  a.B = B; a.K = K; a.d_model = d_model; a.V = V;
+  a.threshold = threshold;
+  a.mode = mode;
+  a.philox_seed = philox_seed; a.philox_offset = offset;
+  a.out_accept_len = out_accept_len; a.out_next_token = out_next_token;
+  a.out_div = out_div; a.out_resid_mass = out_resid_mass;
+  a.stream = cuda_stream;
+  return pyramidsd_verify_fused_lmhead_ex(&a);
 }
 
 double pyramidsd_model_sd_throughput(double beta, double ell, double v_small, double v_large) {
@@ -846,9 +970,14 @@ size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype) {
   return stage_workspace_bytes(B, K);
 }
 
+size_t pyramidsd_pyramid_workspace_bytes(int B, int K_d, int K_q, int V, psd_dtype dtype) {
+  if (B < 0 || K_q < 1 || K_d < K_q || K_d > 32 || V < 1 || !valid_dtype(dtype)) return 0;
+  return pyramid_workspace_bytes(B, K_d, K_q);
+}
+
 int pyramidsd_set_two_stage_policy(int policy) {
-  if (policy != PSD_TWO_STAGE_FUSED && policy != PSD_TWO_STAGE_SEPARATE && policy != PSD_TWO_STAGE_AUTO) return PSD_ERR_INVALID_ARG;
-  t_two_stage_policy = policy;
+  if (policy < PSD_TWO_STAGE_DEFAULT || policy > PSD_TWO_STAGE_FUSED_ROWS) return PSD_ERR_INVALID_ARG;
+  t_two_stage_policy = policy == PSD_TWO_STAGE_DEFAULT ? PSD_TWO_STAGE_AUTO : policy;
   return PSD_OK;
 }
 
@@ -858,19 +987,32 @@ int pyramidsd_set_stream(void* cuda_stream) {
 }
 
 int pyramidsd_last_status(void) {
-  DeviceState* ds = nullptr;
-  int rc = current_device_state(&ds);
-  if (rc != PSD_OK) return rc;
-  if (cudaStreamSynchronize(t_stream) != cudaSuccess) return PSD_ERR_CUDA;
-  std::lock_guard<std::mutex> lock(ds->mu);
-  if (!ds->status) return PSD_OK;
+  StreamScratch* ss = t_last_scratch;
+  if (ss == nullptr) return cudaStreamSynchronize(t_stream) == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(ss->mu);
+  if (cudaStreamSynchronize(ss->stream) != cudaSuccess) return PSD_ERR_CUDA;
+  if (!ss->status) return PSD_OK;
   int host = 0;
-  if (cudaMemcpy(&host, ds->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PSD_ERR_CUDA;
+  if (cudaMemcpy(&host, ss->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PSD_ERR_CUDA;
   if (host != 0) {
-    cudaMemset(ds->status, 0, sizeof(int));
+    cudaMemset(ss->status, 0, sizeof(int));
     return PSD_ERR_TIMEOUT;
   }
   return PSD_OK;
+}
+
+int pyramidsd_selftest_wait_timeout(void* cuda_stream) {
+  const cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  StreamScratch* ss = nullptr;
+  int rc = scratch_for(stream, &ss);
+  if (rc != PSD_OK) return rc;
+  std::lock_guard<std::mutex> lock(ss->mu);
+  t_last_scratch = ss;
+  rc = ensure_status(ss);
+  if (rc != PSD_OK) return rc;
+  psd::wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(ss->status);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return check_launch();
 }
 
 int pyramidsd_kernel_timing_begin(void) {
@@ -908,7 +1050,7 @@ int pyramidsd_cluster_occupancy(int B, int K, int V, psd_dtype dtype, int* out_c
   P.seq_stride_small = P.seq_stride_large = static_cast<long long>(K) * V;
   P.div_kind = PSD_DIV_JS;
   psd::ClusterGeom g{};
-  const bool ok = B > 0 && K > 0 && psd::cluster_geometry(P, dtype, 0, &g);
+  const bool ok = B > 0 && K > 0 && psd::cluster_geometry(P, dtype, 0, false, false, &g);
   if (out_cluster_size) *out_cluster_size = ok ? g.cs : 0;
   if (out_max_active_clusters) {
     *out_max_active_clusters = ok ? psd::cluster_max_active_any(dtype, PSD_DIV_JS, g.cs) : 0;

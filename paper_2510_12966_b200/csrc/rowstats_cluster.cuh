@@ -25,29 +25,29 @@
 // part of the ring feeds pass A and is handed back by pass A, the rest feeds pass B, which runs one row
 // behind and gets its copy out of L2; a second loader thread (warp 19) serves pass B's ring. The
 // arithmetic and its order are those of the resident variant.
+//
+// Three-row form of the streamed-twice variant (template flag TRI), for the two-stage wrapper. Stage 2 of the
+// pyramid scores the window with the qualifier's distribution in the draft's place (Fig. 1), so for a position
+// k < K_q the qualifier row is the large model of the stage-1 pair and the small model of the stage-2 pair. A
+// TRI launch walks one work item per stage-1 row: positions k < K_q are row triples (draft, qualifier, target)
+// -- three log-sum-exps in pass A, the two pairs' divergence terms in pass B, the qualifier row read, widened
+// and normalised once -- and positions k >= K_q are ordinary pairs. A triple moves one chunk of three rows per
+// ring slot, a pair two chunks of two rows; each model's sums and each pair's terms are taken in the order of
+// the two-row form, so both forms return the same bits.
 #pragma once
 
-#include <cstdlib>
+#include <type_traits>
 
 #include "common.cuh"
 
 namespace psd {
 
-#ifndef PSD_A_WARPS
-#define PSD_A_WARPS 8
-#endif
-#ifndef PSD_B_WARPS
-#define PSD_B_WARPS 8
-#endif
-constexpr int kClAWarps = PSD_A_WARPS;             // warps running pass A (0 .. kClAWarps - 1)
-constexpr int kClBWarps = PSD_B_WARPS;             // warps running pass B (the next kClBWarps)
+constexpr int kClAWarps = 8;                       // warps running pass A (0 .. kClAWarps - 1)
+constexpr int kClBWarps = 8;                       // warps running pass B (the next kClBWarps)
 constexpr int kClConsumerWarps = kClAWarps + kClBWarps;
 constexpr int kClConsumers = kClConsumerWarps * 32;
 constexpr int kClThreads = kClConsumers + 96;      // + loader warp + two agent warps
-#ifndef PSD_RS_SUB
-#define PSD_RS_SUB 2
-#endif
-constexpr int kClSubRS = PSD_RS_SUB;               // chunks per slot of the streamed-twice variant
+constexpr int kClSubRS = 2;                        // chunks per slot of the streamed-twice variant (measured: 2 beats 1, 3 and 4)
 constexpr int kClThreadsRS = kClThreads + 32;      // the streamed-twice variant has a loader warp per pass
 constexpr int kClHalfBytes = 8192;                 // one model's part of a chunk: 256 threads x 2 x 16 bytes
 constexpr int kClAVec = 16 / kClAWarps;            // 16-byte vectors per lane, chunk and model in pass A
@@ -57,6 +57,13 @@ constexpr int kClSlotBytes = 2 * kClHalfBytes;
 constexpr int kClSlots = 13;                       // ring slots
 constexpr int kClDepth = 4;                        // rows of exchange buffers in flight
 constexpr int kClMaxRanks = 16;
+// Registers per thread by role in the streamed-twice variant (640 threads start with 96 each). Its five groups of
+// four warps trade registers at the role split (setmaxnreg): the pass-A warps and the loader / agent warps give
+// some up, the pass-B warps, whose inner loop holds two vectors of three models in flight, take them.
+// 8 x 32 x 80 + 8 x 32 x 128 + 4 x 32 x 56 = 60416 <= 640 x 96. Measured against 96 everywhere: config 4's
+// statistics launch 0.558 -> 0.539 ms, config 3 unchanged; 72 / 136 / 56 and 64 / 136 / 64 spill in pass A.
+constexpr int kClRegsA = 80, kClRegsB = 128, kClRegsService = 56;
+static_assert(kClThreadsRS == 640 && kClAWarps == 8 && kClBWarps == 8, "the register split above is for 8 + 8 + 4 warps");
 constexpr unsigned kClSpinLimit = 1u << 22;        // polls before a wait gives up (a fraction of a second at the least)
 
 struct ClusterGeom {
@@ -69,6 +76,7 @@ struct ClusterGeom {
                  // slice is streamed twice through slots of two chunks each, slots [0, ra) feed pass A and
                  // slots [ra, ring) feed pass B
   int lead;      // streamed twice: pass A hands row n to the agent once row n - lead has been released to pass B
+  int tri;       // 1: the launch walks the two-stage wrapper's rows as triples (k < K2) and pairs, one item per stage-1 row
 };
 
 // Per-row constants of pass B: -log2 of the normalisers in the scaled base-2 domain and the clamp floors.
@@ -76,7 +84,10 @@ struct __align__(16) RowConsts {
   float off_small, off_large;        // log2(sum_i exp(z_i / T)) of each model
   float floor_small, floor_large;    // logits below these would give log2 p < -125
   unsigned floor2_small, floor2_large;   // the same floors as packed bf16 pairs
-  unsigned pad0, pad1;
+  unsigned floor2_third;             // row triples: the third model (the target)
+  unsigned pad0;
+  float off_third, floor_third;
+  unsigned pad1, pad2;
 };
 
 // Shared-memory control block behind the ring.
@@ -90,6 +101,12 @@ struct __align__(16) ClusterCtl {
   RowConsts row_consts[kClDepth];                  // what pass B needs of the row, published by the agent
   float4 lse_in[kClDepth][kClMaxRanks];            // partials received from every rank of the cluster
   float4 fin_in[kClDepth][kClMaxRanks];            // pass-B partials received (rank 0 only)
+  // row triples: the third model's log-sum-exp partials and the second pair's pass-B partials
+  float4 a_part3[kClDepth][kClAWarps];             // (ref_third, sum_third, unused, unused)
+  float4 b_part2[kClDepth][kClBWarps];
+  float4 row_lse3[kClDepth];                       // (m2_third, l2s_third, unused, unused)
+  float4 lse_in3[kClDepth][kClMaxRanks];
+  float4 fin_in2[kClDepth][kClMaxRanks];
   int rows_closed;                                 // rows whose pass-B partials the second agent has dealt with
 };
 
@@ -171,16 +188,37 @@ __device__ __forceinline__ uint4 lds128(const void* p) {
 // ---- row walk ---------------------------------------------------------------------------------------
 // Every role of every CTA of a cluster walks the same list: rows q, q + n_clusters, ... of the [B*K]
 // grid, skipping positions at or beyond the sequence's n_valid. `n` counts the rows taken so far.
+// Three-row launches walk one item per stage-1 row instead, position-major, with the positions taken in an
+// order that alternates triples (k < K2) and pairs (k >= K2), so that whatever the number of clusters and
+// the batch size have in common every cluster gets its share of both.
 struct RowWalk {
-  int next_r, stride, rows, rows1, K, B;
+  int next_r, stride, rows, rows1, K, K2, B;
   const int32_t* n_valid;
+  bool tri_mode;
   int n;     // ordinal of the current row among the rows this cluster takes
   int r;     // current row index (valid after advance() returned true)
-  __device__ void init(const StageParams& P, int cluster_id, int n_clusters) {
-    next_r = cluster_id; stride = n_clusters; rows = P.B * (P.K + P.K2); rows1 = P.B * P.K; K = P.K; B = P.B;
-    n_valid = P.n_valid; n = -1; r = -1;
+  int r2;    // row triples: index of the stage-2 row, b * K2 + k
+  bool tri;  // the current item is a row triple
+  __device__ void init(const StageParams& P, int cluster_id, int n_clusters, bool three_row) {
+    next_r = cluster_id; stride = n_clusters; rows1 = P.B * P.K; K = P.K; K2 = P.K2; B = P.B;
+    tri_mode = three_row;
+    rows = three_row ? rows1 : P.B * (P.K + P.K2);
+    n_valid = P.n_valid; n = -1; r = -1; r2 = -1; tri = false;
   }
   __device__ bool advance() {
+    if (tri_mode) {
+      if (next_r >= rows) return false;
+      const int cand = next_r;
+      next_r += stride;
+      const int j = cand / B, b = cand - j * B;
+      // j-th position in the alternating order: 0, K2, 1, K2 + 1, ... until one kind runs out
+      const int n_pair = K - K2, both = 2 * (K2 < n_pair ? K2 : n_pair);
+      int k;
+      if (j < both) k = (j & 1) ? K2 + (j >> 1) : (j >> 1);
+      else k = (K2 > n_pair) ? (both >> 1) + (j - both) : K2 + (both >> 1) + (j - both);
+      r = b * K + k; tri = k < K2; r2 = b * K2 + k; ++n;
+      return true;
+    }
     while (next_r < rows) {
       const int cand = next_r;
       next_r += stride;
@@ -406,9 +444,7 @@ __device__ __forceinline__ float2 psi_poly(float2 u) {
 // held to 2e-3 and take degree 4, whose error adds at most 0.35 * 4e-5 * sum max(p, q) < 3e-5 to D (measured
 // against a double-precision reference on peaked, flat, near-equal and far-apart row pairs: at most 1.6e-5,
 // against 1e-6 with degree 7), for three of the polynomial's seven instructions.
-#ifndef PSD_PSI_DEG_BF16
-#define PSD_PSI_DEG_BF16 4
-#endif
+constexpr int kPsiDegBf16 = 4;
 
 struct DivAcc {
   float2 js, big;    // sum 2^M h(d); sum 2^M
@@ -450,8 +486,10 @@ __device__ __forceinline__ V warp_sum(V v) { return warp_reduce<OpSum>(v); }
 // RS = false: a CTA's slice of a row fits the ring and is copied in once. RS = true ("re-stream"): the slice is
 // larger than the ring (small clusters, which is what fills every SM of the device), so it is copied in
 // twice -- once for each pass, the second copy coming out of L2 -- through two rings of their own.
-template <typename T, int DIV, bool RS>
+// TRI (with RS only): the launch is a two-stage wrapper's, walked as row triples and pairs (see the top).
+template <typename T, int DIV, bool RS, bool TRI>
 __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cluster_kernel(const StageParams P, const ClusterGeom G) {
+  static_assert(RS || !TRI, "row triples are streamed twice");
   extern __shared__ unsigned char smem_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   ClusterCtl* ctl = reinterpret_cast<ClusterCtl*>(ring + static_cast<size_t>(kClSlots) * kClSlotBytes);
@@ -468,10 +506,13 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
   const int RA = RS ? G.ra : R;        // slots pass A cycles through
   const int RB0 = RS ? G.ra : 0;       // first slot of pass B
   // The streamed-twice variant moves two chunks per barrier (a slot of 2 x 16 KB): its rings need no chunk
-  // granularity to hold a row, and every hand-off costs the two instruction streams issue slots.
+  // granularity to hold a row, and every hand-off costs the two instruction streams issue slots. A row triple
+  // moves one chunk of its three rows (24 KB of the same slot).
   constexpr int SUB = RS ? kClSubRS : 1;
   constexpr int kSlotStride = SUB * kClSlotBytes;
-  const int CS = (C + SUB - 1) / SUB;  // barrier steps per row slice
+  static_assert(!TRI || kSlotStride >= 3 * kClHalfBytes, "a slot holds one chunk of three rows");
+  const int CS = (C + SUB - 1) / SUB;  // barrier steps per row slice of a pair
+  auto steps_of = [&](bool tri) { return tri ? C : CS; };
 
   if (tid == 0) {
     ctl->rows_closed = 0;
@@ -503,6 +544,20 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
     while (!dead && !mbar_try(bar, parity))
       if (++spins > kClSpinLimit) give_up();
   };
+  const int rows1 = P.B * K;
+  // base of this CTA's slice of model m (0 small, 1 large, 2 third) of the walk's current item
+  auto model_row = [&](const RowWalk& w, int m) -> const T* {
+    if (TRI) {
+      if (m == 0) return row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V) + slice_begin;
+      if (m == 1) return row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V) + slice_begin;
+      return row_ptr<T>(P.large2, P.seq_stride_large2, w.r2, P.K2, V) + slice_begin;
+    }
+    const bool second = w.r >= rows1;   // second row set: stage 2 of the wrapper
+    if (m == 0) return (second ? row_ptr<T>(P.small2, P.seq_stride_small2, w.r - rows1, P.K2, V)
+                               : row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V)) + slice_begin;
+    return (second ? row_ptr<T>(P.large2, P.seq_stride_large2, w.r - rows1, P.K2, V)
+                   : row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V)) + slice_begin;
+  };
 
   if (warp < kClConsumerWarps) {
     const float c = P.c;
@@ -516,10 +571,11 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
 #pragma unroll
     for (int i = 0; i < kMaxVec; ++i) len[i] = slice_len - (pw * 32 + lane + i * pass_warps * 32) * E;
     RowWalk w;
-    w.init(P, cluster_id, G.n_clusters);
+    w.init(P, cluster_id, G.n_clusters, TRI);
     unsigned slot = 0, par = 0;
 
     if (is_a) {
+      if (RS) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kClRegsA));
       constexpr int kVecStride = kClAWarps * 32 * 16;   // bytes between a lane's vectors
       // ================================ pass A ================================
       // A row is summed optimistically against one reference per model, taken from the warp's first
@@ -527,42 +583,51 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
       // freely. Only if some lane's row sum comes out non-finite (a logit more than 2^127 above that
       // reference, or NaN / +inf) is the row redone through the careful per-vector commits -- its chunks
       // are all still in the ring, because pass B cannot enter the row before pass A has left it.
-      LseState ls, ll;
       bool landed = false;   // the answer of a test of the next chunk's barrier, asked one chunk early
-      while (w.advance()) {
-        ls.reset(); ll.reset();
+      // one row of NM models, SUBN chunks per slot
+      auto row_a = [&](auto nm_c, auto sub_c) {
+        constexpr int NM = decltype(nm_c)::value, SUBN = decltype(sub_c)::value;
+        const int steps = (C + SUBN - 1) / SUBN;
+        LseState st[NM];
+        float2 v[NM];
+#pragma unroll
+        for (int m = 0; m < NM; ++m) { st[m].reset(); v[m] = make_float2(0.f, 0.f); }
         const unsigned slot0 = slot;   // where the row starts in the ring
-        float2 vs = make_float2(0.f, 0.f), vl = vs;
         int off = 0;   // chunk offset inside the slice, in logits
-        for (int step = 0; step < CS; ++step) {
+        for (int step = 0; step < steps; ++step) {
           if (!landed) wait_phase(&ctl->full[slot], par);
           const unsigned char* sbase = my + slot * kSlotStride;
           const unsigned used = slot;
           if (++slot == static_cast<unsigned>(RA)) { slot = 0; par ^= 1u; }
           landed = mbar_test(&ctl->full[slot], par);   // its latency hides behind this step's arithmetic
 #pragma unroll
-          for (int sub = 0; sub < SUB; ++sub, off += CH) {   // a chunk beyond the slice (odd count) has no live vector
+          for (int sub = 0; sub < SUBN; ++sub, off += CH) {   // a chunk beyond the slice (odd count) has no live vector
             const unsigned char* base = sbase + sub * kClSlotBytes;
-            uint4 us[kClAVec], ul[kClAVec];
+            uint4 u[NM][kClAVec];
 #pragma unroll
-            for (int i = 0; i < kClAVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+            for (int i = 0; i < kClAVec; ++i)
+#pragma unroll
+              for (int m = 0; m < NM; ++m) u[m][i] = lds128(base + m * kClHalfBytes + i * kVecStride);
             if (step == 0 && sub == 0) {
               // the warp's largest logit of its first vectors (the floor keeps rows that start with -inf at 0)
-              float gs = vector_max<T>(us[0], len[0] > 0), gl = vector_max<T>(ul[0], len[0] > 0);
+              float g[NM];
 #pragma unroll
-              for (int o = 16; o > 0; o >>= 1) {
-                gs = fmaxf(gs, __shfl_xor_sync(0xffffffffu, gs, o));
-                gl = fmaxf(gl, __shfl_xor_sync(0xffffffffu, gl, o));
-              }
-              ls.ref = fmaxf(gs * c, -1e30f);
-              ll.ref = fmaxf(gl * c, -1e30f);
+              for (int m = 0; m < NM; ++m) g[m] = vector_max<T>(u[m][0], len[0] > 0);
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                for (int m = 0; m < NM; ++m) g[m] = fmaxf(g[m], __shfl_xor_sync(0xffffffffu, g[m], o));
+#pragma unroll
+              for (int m = 0; m < NM; ++m) st[m].ref = fmaxf(g[m] * c, -1e30f);
             }
 #pragma unroll
             for (int i = 0; i < kClAVec; ++i) {
-              const float2 ps = lse_vector_sum2<T>(us[i], c, ls.ref), pl = lse_vector_sum2<T>(ul[i], c, ll.ref);
               const bool live = len[i] > off;
-              vs = __fadd2_rn(vs, live ? ps : make_float2(0.f, 0.f));
-              vl = __fadd2_rn(vl, live ? pl : make_float2(0.f, 0.f));
+#pragma unroll
+              for (int m = 0; m < NM; ++m) {
+                const float2 ps = lse_vector_sum2<T>(u[m][i], c, st[m].ref);
+                v[m] = __fadd2_rn(v[m], live ? ps : make_float2(0.f, 0.f));
+              }
             }
           }
           if (RS) {   // pass A is this slot's only reader: hand it back
@@ -570,20 +635,19 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
             if (lane == 0) mbar_arrive(&ctl->empty[used]);
           }
         }
-        ls.s = vs.x + vs.y;
-        ll.s = vl.x + vl.y;
-        if (__any_sync(0xffffffffu, !(ls.s + ll.s < INFINITY))) {
+        float tot = 0.f;
+#pragma unroll
+        for (int m = 0; m < NM; ++m) { st[m].s = v[m].x + v[m].y; tot += st[m].s; }
+        if (__any_sync(0xffffffffu, !(tot < INFINITY))) {
           // careful second go over the row's chunks, vector by vector, moving the references as needed
-          ls.s = 0.f; ll.s = 0.f;
+#pragma unroll
+          for (int m = 0; m < NM; ++m) st[m].s = 0.f;
           unsigned sl2 = slot0;
           off = 0;
           // when the slice is streamed twice its chunks have left the ring: take the vectors from global memory
-          const int rows1 = P.B * K;
-          const bool second = w.r >= rows1;
-          const T* gs = (second ? row_ptr<T>(P.small2, P.seq_stride_small2, w.r - rows1, P.K2, V)
-                                : row_ptr<T>(P.small, P.seq_stride_small, w.r, K, V)) + slice_begin;
-          const T* gl = (second ? row_ptr<T>(P.large2, P.seq_stride_large2, w.r - rows1, P.K2, V)
-                                : row_ptr<T>(P.large, P.seq_stride_large, w.r, K, V)) + slice_begin;
+          const T* g[NM];
+#pragma unroll
+          for (int m = 0; m < NM; ++m) g[m] = model_row(w, m);
 #pragma unroll 1
           for (int cidx = 0; cidx < C; ++cidx, off += CH) {
             const unsigned char* base = my + sl2 * kClSlotBytes;
@@ -591,22 +655,25 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
             for (int i = 0; i < kClAVec; ++i) {
               const int e = off + (pw * 32 + lane + i * kClAWarps * 32) * E;   // first logit of the vector, in the slice
               const bool live = e < slice_len;
-              uint4 vs4 = make_uint4(0u, 0u, 0u, 0u), vl4 = vs4;
-              if (RS) {
-                if (live) { vs4 = *reinterpret_cast<const uint4*>(gs + e); vl4 = *reinterpret_cast<const uint4*>(gl + e); }
-              } else {
-                vs4 = lds128(base + i * kVecStride);
-                vl4 = lds128(base + kClHalfBytes + i * kVecStride);
+#pragma unroll
+              for (int m = 0; m < NM; ++m) {
+                uint4 v4 = make_uint4(0u, 0u, 0u, 0u);
+                if (RS) {
+                  if (live) v4 = *reinterpret_cast<const uint4*>(g[m] + e);
+                } else {
+                  v4 = lds128(base + m * kClHalfBytes + i * kVecStride);
+                }
+                // a NaN "reference used" makes the commit take the vector sum afresh
+                lse_commit<T>(0.f, __int_as_float(0x7fc00000), v4, live, c, st[m]);
               }
-              // a NaN "reference used" makes the commit take the vector sum afresh
-              lse_commit<T>(0.f, __int_as_float(0x7fc00000), vs4, live, c, ls);
-              lse_commit<T>(0.f, __int_as_float(0x7fc00000), vl4, live, c, ll);
             }
             if (++sl2 == static_cast<unsigned>(R)) sl2 = 0;
           }
         }
         // row finished: the warp's partial (one reference, summed S) -> a_part, then tell the agent
-        const float ss = warp_reduce<OpSum>(ls.s), sl = warp_reduce<OpSum>(ll.s);
+        float sums[NM];
+#pragma unroll
+        for (int m = 0; m < NM; ++m) sums[m] = warp_reduce<OpSum>(st[m].s);
         const int d = w.n % kClDepth;
         // With a ring of its own pass A could run rows ahead of pass B and of the agents (a resident slice
         // cannot: its slots come back from pass B). The exchange buffers are kClDepth rows deep, so row n is
@@ -617,24 +684,33 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
           wait_phase(&ctl->b_go[m % kClDepth], (m / kClDepth) & 1u);
         }
         if (lane == 0) {
-          ctl->a_part[d][pw] = make_float4(ls.ref, ss, ll.ref, sl);
+          ctl->a_part[d][pw] = make_float4(st[0].ref, sums[0], st[1].ref, sums[1]);
+          if (NM == 3) ctl->a_part3[d][pw] = make_float4(st[NM - 1].ref, sums[NM - 1], 0.f, 0.f);
           mbar_arrive(&ctl->a_done[d]);
         }
+      };
+      while (w.advance()) {
+        if (TRI && w.tri) row_a(std::integral_constant<int, 3>{}, std::integral_constant<int, 1>{});
+        else row_a(std::integral_constant<int, 2>{}, std::integral_constant<int, SUB>{});
       }
     } else {
       // ================================ pass B ================================
+      if (RS) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kClRegsB));
       constexpr int N = Pairs<T>::kN;
+      constexpr int PSI = sizeof(T) == 2 ? kPsiDegBf16 : 7;
       constexpr int kVecStride = kClBWarps * 32 * 16;   // bytes between a lane's vectors
       if (RS) slot = static_cast<unsigned>(RB0);
       bool landed = false;   // as in pass A: the next chunk's barrier is tested one chunk early
-      while (w.advance()) {
+      auto row_b = [&](auto nm_c, auto sub_c) {
+        constexpr int NM = decltype(nm_c)::value, SUBN = decltype(sub_c)::value;
+        const int steps = (C + SUBN - 1) / SUBN;
         const int d = w.n % kClDepth;
         wait_phase(&ctl->b_go[d], (w.n / kClDepth) & 1u);   // the row's constants are published: pass A is through
         const RowConsts rc = ctl->row_consts[d];
-        DivAcc acc;
-        acc.reset();
+        DivAcc acc, acc2;   // the pair (small, large); for a triple also the pair (large, third)
+        acc.reset(); acc2.reset();
         int off = 0;
-        for (int step = 0; step < CS; ++step) {
+        for (int step = 0; step < steps; ++step) {
           if (RS && !landed) wait_phase(&ctl->full[slot], par);   // pass B's own copy of the chunks
           const unsigned char* sbase = my + slot * kSlotStride;
           if (RS) {
@@ -643,24 +719,41 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
             landed = mbar_test(&ctl->full[nslot], npar);
           }
 #pragma unroll
-          for (int sub = 0; sub < SUB; ++sub, off += CH) {
+          for (int sub = 0; sub < SUBN; ++sub, off += CH) {
             const unsigned char* base = sbase + sub * kClSlotBytes;
-            uint4 us[kClBVec], ul[kClBVec];
+            uint4 u[NM][kClBVec];
 #pragma unroll
-            for (int i = 0; i < kClBVec; ++i) { us[i] = lds128(base + i * kVecStride); ul[i] = lds128(base + kClHalfBytes + i * kVecStride); }
+            for (int i = 0; i < kClBVec; ++i)
+#pragma unroll
+              for (int m = 0; m < NM; ++m) u[m][i] = lds128(base + m * kClHalfBytes + i * kVecStride);
 #pragma unroll
             for (int i = 0; i < kClBVec; ++i) {
               float2 xs[N], xl[N];
-              Pairs<T>::load_clamped(us[i], rc.floor_small, rc.floor2_small, xs);
-              Pairs<T>::load_clamped(ul[i], rc.floor_large, rc.floor2_large, xl);
+              Pairs<T>::load_clamped(u[0][i], rc.floor_small, rc.floor2_small, xs);
+              Pairs<T>::load_clamped(u[1][i], rc.floor_large, rc.floor2_large, xl);
               DivAcc local;
               local.reset();
-              local.differ = (us[i].x ^ ul[i].x) | (us[i].y ^ ul[i].y) | (us[i].z ^ ul[i].z) | (us[i].w ^ ul[i].w);
-              div_accumulate<DIV, N, (sizeof(T) == 2 ? PSD_PSI_DEG_BF16 : 7)>(xl, xs, c, rc.off_large, rc.off_small, local);
-              if (len[i] > off) {   // a vector beyond the slice adds nothing
+              local.differ = (u[0][i].x ^ u[1][i].x) | (u[0][i].y ^ u[1][i].y) | (u[0][i].z ^ u[1][i].z) | (u[0][i].w ^ u[1][i].w);
+              div_accumulate<DIV, N, PSI>(xl, xs, c, rc.off_large, rc.off_small, local);
+              const bool live = len[i] > off;   // a vector beyond the slice adds nothing
+              if (live) {
                 acc.js = __fadd2_rn(acc.js, local.js);
                 acc.big = __fadd2_rn(acc.big, local.big);
                 acc.differ |= local.differ;
+              }
+              if (NM == 3) {
+                float2 xt[N];
+                Pairs<T>::load_clamped(u[NM - 1][i], rc.floor_third, rc.floor2_third, xt);
+                DivAcc local2;
+                local2.reset();
+                local2.differ = (u[1][i].x ^ u[NM - 1][i].x) | (u[1][i].y ^ u[NM - 1][i].y) | (u[1][i].z ^ u[NM - 1][i].z) |
+                                (u[1][i].w ^ u[NM - 1][i].w);
+                div_accumulate<DIV, N, PSI>(xt, xl, c, rc.off_third, rc.off_large, local2);
+                if (live) {
+                  acc2.js = __fadd2_rn(acc2.js, local2.js);
+                  acc2.big = __fadd2_rn(acc2.big, local2.big);
+                  acc2.differ |= local2.differ;
+                }
               }
             }
           }
@@ -671,13 +764,26 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         const float js = warp_reduce<OpSum>(acc.js.x + acc.js.y);
         const float big = warp_reduce<OpSum>(acc.big.x + acc.big.y);
         const unsigned differ = __reduce_or_sync(0xffffffffu, acc.differ);
+        float js2 = 0.f, big2 = 0.f;
+        unsigned differ2 = 0u;
+        if (NM == 3) {
+          js2 = warp_reduce<OpSum>(acc2.js.x + acc2.js.y);
+          big2 = warp_reduce<OpSum>(acc2.big.x + acc2.big.y);
+          differ2 = __reduce_or_sync(0xffffffffu, acc2.differ);
+        }
         if (lane == 0) {
           ctl->b_part[d][pw] = make_float4(js, big, differ ? 1.f : 0.f, 0.f);
+          if (NM == 3) ctl->b_part2[d][pw] = make_float4(js2, big2, differ2 ? 1.f : 0.f, 0.f);
           mbar_arrive(&ctl->b_done[d]);
         }
+      };
+      while (w.advance()) {
+        if (TRI && w.tri) row_b(std::integral_constant<int, 3>{}, std::integral_constant<int, 1>{});
+        else row_b(std::integral_constant<int, 2>{}, std::integral_constant<int, SUB>{});
       }
     }
   } else if (warp == kClConsumerWarps || warp == kClConsumerWarps + 3) {
+    if (RS) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kClRegsService));
     // ================================ loader ================================
     // One thread per ring: the whole ring, or (slice streamed twice) pass A's slots [0, RA) from this warp and
     // pass B's slots [RA, R) from the last warp. The two streams run freely; pass B's copy of a chunk is
@@ -686,55 +792,55 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
     const unsigned lo = for_b ? static_cast<unsigned>(RB0) : 0u, hi = static_cast<unsigned>(for_b ? R : RA);
     if (lane == 0) {
       RowWalk w;
-      w.init(P, cluster_id, G.n_clusters);
-      const int rows1 = P.B * K;
-      auto row_small = [&](int r) {
-        return (r >= rows1 ? row_ptr<T>(P.small2, P.seq_stride_small2, r - rows1, P.K2, V)   // second set: stage 2 of the wrapper
-                           : row_ptr<T>(P.small, P.seq_stride_small, r, K, V)) + slice_begin;
-      };
-      auto row_large = [&](int r) {
-        return (r >= rows1 ? row_ptr<T>(P.large2, P.seq_stride_large2, r - rows1, P.K2, V)
-                           : row_ptr<T>(P.large, P.seq_stride_large, r, K, V)) + slice_begin;
-      };
+      w.init(P, cluster_id, G.n_clusters, TRI);
       const unsigned long long policy = RS ? (for_b ? l2_policy_drop() : l2_policy_keep()) : 0ull;
-      // step `step` of a row slice (SUB chunks) into `slot`, once the slot's readers of `fills` ring turns ago are through
-      auto fill = [&](const T* rs, const T* rl, int step, unsigned slot, unsigned fills) {
+      // step `step` of a row slice (`sub_n` chunks of `nm` models) into `slot`, once the slot's readers of
+      // `fills` ring turns ago are through
+      auto fill = [&](const T* const (&src)[3], int nm, int sub_n, int step, unsigned slot, unsigned fills) {
         if (fills > 0) wait_phase(&ctl->empty[slot], (fills - 1u) & 1u);
+        if (dead) return false;   // the slot was never handed back: nothing more is copied into this ring
         unsigned total = 0;
-#pragma unroll
-        for (int sub = 0; sub < SUB; ++sub) total += static_cast<unsigned>(max(0, min(CH, slice_len - (step * SUB + sub) * CH)));
+        for (int sub = 0; sub < sub_n; ++sub) total += static_cast<unsigned>(max(0, min(CH, slice_len - (step * sub_n + sub) * CH)));
         if (total > 0) {
-          mbar_arrive_expect_tx(&ctl->full[slot], 2u * total * static_cast<unsigned>(sizeof(T)));
-#pragma unroll
-          for (int sub = 0; sub < SUB; ++sub) {
-            const int e0 = (step * SUB + sub) * CH;
+          mbar_arrive_expect_tx(&ctl->full[slot], static_cast<unsigned>(nm) * total * static_cast<unsigned>(sizeof(T)));
+          for (int sub = 0; sub < sub_n; ++sub) {
+            const int e0 = (step * sub_n + sub) * CH;
             const int n = min(CH, slice_len - e0);
             if (n > 0) {
               const unsigned bytes = static_cast<unsigned>(n) * sizeof(T);
               unsigned char* dst = ring + static_cast<size_t>(slot) * kSlotStride + sub * kClSlotBytes;
-              if (RS) {
-                bulk_load_hint(dst, rs + e0, bytes, &ctl->full[slot], policy);
-                bulk_load_hint(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot], policy);
-              } else {
-                bulk_load(dst, rs + e0, bytes, &ctl->full[slot]);
-                bulk_load(dst + kClHalfBytes, rl + e0, bytes, &ctl->full[slot]);
+              for (int m = 0; m < nm; ++m) {
+                if (RS) bulk_load_hint(dst + m * kClHalfBytes, src[m] + e0, bytes, &ctl->full[slot], policy);
+                else bulk_load(dst + m * kClHalfBytes, src[m] + e0, bytes, &ctl->full[slot]);
               }
             }
           }
         } else {
           mbar_arrive(&ctl->full[slot]);   // nothing of this step falls into this CTA's slice
         }
+        return true;
       };
       unsigned slot = lo, fills = 0;   // ring position; how often the ring has wrapped
-      while (w.advance()) {
-        const T* rs = row_small(w.r);
-        const T* rl = row_large(w.r);
-        for (int step = 0; step < CS; ++step) {
-          fill(rs, rl, step, slot, fills);
+      while (!dead && w.advance()) {
+        const bool tri = TRI && w.tri;
+        const T* const src[3] = {model_row(w, 0), model_row(w, 1), tri ? model_row(w, 2) : nullptr};
+        const int steps = steps_of(tri);
+        for (int step = 0; step < steps; ++step) {
+          if (!fill(src, tri ? 3 : 2, tri ? 1 : SUB, step, slot, fills)) break;
           if (++slot == hi) { slot = lo; ++fills; }
         }
       }
-      // every copy issued above is waited for by its consumers before they leave
+      // Every copy issued above is waited for by its consumers before they leave -- unless a wait gave up
+      // somewhere in the CTA. Then this thread has stopped issuing, and it sees every copy it did issue land
+      // before the CTA's shared memory goes away: each slot's barrier is polled (bounded) for its latest phase.
+      if (dead || *reinterpret_cast<volatile int*>(P.status) != 0) {
+        for (unsigned s = lo; s < hi; ++s) {
+          const unsigned turns = fills + (s < slot ? 1u : 0u);   // phases of this slot's barrier armed so far
+          if (turns == 0) continue;
+          unsigned spins = 0;
+          while (!mbar_try(&ctl->full[s], (turns - 1u) & 1u) && ++spins <= kClSpinLimit) {}
+        }
+      }
     }
   } else {
     // ================================ agent ================================
@@ -748,29 +854,44 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
     // share their issue ports next to nothing. The exchange buffers are kClDepth rows deep; nothing of row m
     // can be produced anywhere in the cluster before a(m) has been sent, a(m) comes after g(m-1), and the
     // first agent holds a(m) back until the second one has closed row m - kClDepth + 1.
+    // A row triple carries a second 16-byte record through every step (third model / second pair).
+    if (RS) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kClRegsService));
     const float inv_c = 1.f / P.c;
 
-    auto event_a = [&](int n) {
+    auto event_a = [&](int n, bool tri) {
       const int d = n % kClDepth;
       wait_phase(&ctl->a_done[d], (n / kClDepth) & 1u);
       // merge the warps' partials (every lane does the same arithmetic, warp order) ...
-      float ms = -1e30f, ml = -1e30f;
+      float ms = -1e30f, ml = -1e30f, mt = -1e30f;
 #pragma unroll
       for (int k = 0; k < kClAWarps; ++k) { ms = fmaxf(ms, ctl->a_part[d][k].x); ml = fmaxf(ml, ctl->a_part[d][k].z); }
-      float ss = 0.f, sl = 0.f;
+      float ss = 0.f, sl = 0.f, stt = 0.f;
 #pragma unroll
       for (int k = 0; k < kClAWarps; ++k) {
         const float4 v = ctl->a_part[d][k];
         ss = fmaf(v.y, ex2_approx(v.x - ms), ss);
         sl = fmaf(v.w, ex2_approx(v.z - ml), sl);
       }
+      if (TRI && tri) {
+#pragma unroll
+        for (int k = 0; k < kClAWarps; ++k) mt = fmaxf(mt, ctl->a_part3[d][k].x);
+#pragma unroll
+        for (int k = 0; k < kClAWarps; ++k) {
+          const float4 v = ctl->a_part3[d][k];
+          stt = fmaf(v.y, ex2_approx(v.x - mt), stt);
+        }
+      }
       // ... open this row's phase of the local barrier for one partial per rank, and post ours to every rank
-      if (lane == 0) mbar_arrive_expect_tx(&ctl->lse_ready[d], static_cast<unsigned>(G.cs) * 16u);
-      if (lane < G.cs)
+      if (lane == 0) mbar_arrive_expect_tx(&ctl->lse_ready[d], static_cast<unsigned>(G.cs) * ((TRI && tri) ? 32u : 16u));
+      if (lane < G.cs) {
         remote_post_f4(map_to_rank(&ctl->lse_in[d][rank], lane), make_float4(ms, ss, ml, sl),
                        map_to_rank(&ctl->lse_ready[d], lane));
+        if (TRI && tri)
+          remote_post_f4(map_to_rank(&ctl->lse_in3[d][rank], lane), make_float4(mt, stt, 0.f, 0.f),
+                         map_to_rank(&ctl->lse_ready[d], lane));
+      }
     };
-    auto event_g = [&](int n) {
+    auto event_g = [&](int n, bool tri) {
       const int d = n % kClDepth;
       wait_phase(&ctl->lse_ready[d], (n / kClDepth) & 1u);
       // rank order, so that every CTA of the cluster gets the same bits; four ranks at a time keeps the
@@ -792,7 +913,21 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
           sl = fmaf(v[j].w, ex2_approx(v[j].z - ml), sl);
         }
       }
-      const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl);
+      float mt = -1e30f, stt = 0.f;
+      if (TRI && tri) {   // the third model, the same way (its partials sit in the x, y fields)
+        for (int j0 = 0; j0 < G.cs; j0 += 4) {
+          float4 v[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) v[j] = (j0 + j < G.cs) ? ctl->lse_in3[d][j0 + j] : make_float4(-1e30f, 0.f, -1e30f, 0.f);
+          const float gt = fmaxf(fmaxf(v[0].x, v[1].x), fmaxf(v[2].x, v[3].x));
+          const float nt = fmaxf(mt, gt);
+          stt *= ex2_approx(mt - nt);
+          mt = nt;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) stt = fmaf(v[j].y, ex2_approx(v[j].x - mt), stt);
+        }
+      }
+      const float l2ss = lg2_approx(ss), l2sl = lg2_approx(sl), l2st = lg2_approx(stt);
       if (lane == 0) {
         RowConsts rc;
         rc.off_small = ms + l2ss;
@@ -802,28 +937,64 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         rc.floor_large = (DIV == kDivKL) ? -INFINITY : (rc.off_large - 125.f) * inv_c;
         rc.floor2_small = Pairs<T>::floor_bits(rc.floor_small);
         rc.floor2_large = Pairs<T>::floor_bits(rc.floor_large);
-        rc.pad0 = rc.pad1 = 0u;
+        rc.off_third = mt + l2st;
+        rc.floor_third = (DIV == kDivKL) ? -INFINITY : (rc.off_third - 125.f) * inv_c;
+        rc.floor2_third = Pairs<T>::floor_bits(rc.floor_third);
+        rc.pad0 = rc.pad1 = rc.pad2 = 0u;
         ctl->row_consts[d] = rc;
         ctl->row_lse[d] = make_float4(ms, l2ss, ml, l2sl);
+        if (TRI) ctl->row_lse3[d] = make_float4(mt, l2st, 0.f, 0.f);
         mbar_arrive(&ctl->b_go[d]);
       }
     };
-    auto event_b = [&](int n) {
+    auto event_b = [&](int n, bool tri) {
       const int d = n % kClDepth;
       wait_phase(&ctl->b_done[d], (n / kClDepth) & 1u);
-      float js = 0.f, big = 0.f, differ = 0.f;
+      float js = 0.f, big = 0.f, differ = 0.f, js2 = 0.f, big2 = 0.f, differ2 = 0.f;
 #pragma unroll
       for (int k = 0; k < kClBWarps; ++k) {   // warp order
         const float4 v = ctl->b_part[d][k];
         js += v.x; big += v.y; differ += v.z;
       }
+      if (TRI && tri) {
+#pragma unroll
+        for (int k = 0; k < kClBWarps; ++k) {
+          const float4 v = ctl->b_part2[d][k];
+          js2 += v.x; big2 += v.y; differ2 += v.z;
+        }
+      }
       if (lane == 0) {
-        if (rank == 0) mbar_arrive_expect_tx(&ctl->fin_ready[d], static_cast<unsigned>(G.cs) * 16u);
+        if (rank == 0) mbar_arrive_expect_tx(&ctl->fin_ready[d], static_cast<unsigned>(G.cs) * ((TRI && tri) ? 32u : 16u));
         remote_post_f4(map_to_rank(&ctl->fin_in[d][rank], 0), make_float4(js, big, differ, 0.f),
                        map_to_rank(&ctl->fin_ready[d], 0));
+        if (TRI && tri)
+          remote_post_f4(map_to_rank(&ctl->fin_in2[d][rank], 0), make_float4(js2, big2, differ2, 0.f),
+                         map_to_rank(&ctl->fin_ready[d], 0));
       }
     };
-    auto event_f = [&](int n, int r) {   // rank 0 only
+    // statistics record of one pair from its summed pass-B partials and the two models' (m2, l2s)
+    auto make_stats = [&](float js, float big, float differ, float m2s, float l2ss, float m2l, float l2sl) {
+      RowStats st{};
+      int flags = 0;
+      if (!(fabsf(m2s + l2ss) < INFINITY)) flags |= kFlagSmallNonfinite;   // NaN, +inf, or no finite logit
+      if (!(fabsf(m2l + l2sl) < INFINITY)) flags |= kFlagLargeNonfinite;
+      if (flags) {
+        st.m2_small = st.l2s_small = st.m2_large = st.l2s_large = st.div = st.resid = __int_as_float(0x7fc00000);
+      } else {
+        float D;
+        const float res = big - 1.f;   // sum max(p,q) - sum q = sum max(0, p - q)
+        if (DIV == kDivJS) D = (0.5f * kLn2) * js;   // bits -> nats, and the 1/2 of the definition
+        else if (DIV == kDivKL) D = kLn2 * js;
+        else D = res;
+        st.m2_small = m2s; st.l2s_small = l2ss; st.m2_large = m2l; st.l2s_large = l2sl;
+        st.div = fmaxf(D, 0.f);
+        st.resid = fmaxf(res, 0.f);
+        if (differ == 0.f) { st.div = 0.f; st.resid = 0.f; }   // bitwise identical rows: exactly zero
+      }
+      st.flags = flags;
+      return st;
+    };
+    auto event_f = [&](int n, const RowWalk& w) {   // rank 0 only
       const int d = n % kClDepth;
       wait_phase(&ctl->fin_ready[d], (n / kClDepth) & 1u);
       if (lane == 0) {
@@ -833,31 +1004,23 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
           js += v.x; big += v.y; differ += v.z;
         }
         const float4 lse = ctl->row_lse[d];
-        RowStats st{};
-        int flags = 0;
-        if (!(fabsf(lse.x + lse.y) < INFINITY)) flags |= kFlagSmallNonfinite;   // NaN, +inf, or no finite logit
-        if (!(fabsf(lse.z + lse.w) < INFINITY)) flags |= kFlagLargeNonfinite;
-        if (flags) {
-          st.m2_small = st.l2s_small = st.m2_large = st.l2s_large = st.div = st.resid = __int_as_float(0x7fc00000);
-        } else {
-          float D;
-          const float res = big - 1.f;   // sum max(p,q) - sum q = sum max(0, p - q)
-          if (DIV == kDivJS) D = (0.5f * kLn2) * js;   // bits -> nats, and the 1/2 of the definition
-          else if (DIV == kDivKL) D = kLn2 * js;
-          else D = res;
-          st.m2_small = lse.x; st.l2s_small = lse.y; st.m2_large = lse.z; st.l2s_large = lse.w;
-          st.div = fmaxf(D, 0.f);
-          st.resid = fmaxf(res, 0.f);
-          if (differ == 0.f) { st.div = 0.f; st.resid = 0.f; }   // bitwise identical rows: exactly zero
+        const RowStats st = make_stats(js, big, differ, lse.x, lse.y, lse.z, lse.w);
+        if (w.r < rows1) P.stats[w.r] = st;
+        else P.stats2[w.r - rows1] = st;
+        if (TRI && w.tri) {
+          float js2 = 0.f, big2 = 0.f, differ2 = 0.f;
+          for (int j = 0; j < G.cs; ++j) {
+            const float4 v = ctl->fin_in2[d][j];
+            js2 += v.x; big2 += v.y; differ2 += v.z;
+          }
+          const float4 lse3 = ctl->row_lse3[d];
+          P.stats2[w.r2] = make_stats(js2, big2, differ2, lse.z, lse.w, lse3.x, lse3.y);
         }
-        st.flags = flags;
-        if (r < P.B * P.K) P.stats[r] = st;
-        else P.stats2[r - P.B * P.K] = st;
       }
     };
 
     RowWalk w;
-    w.init(P, cluster_id, G.n_clusters);
+    w.init(P, cluster_id, G.n_clusters, TRI);
     if (warp == kClConsumerWarps + 1) {
       // first agent: a(n), g(n) -- the path that releases pass B
       while (w.advance()) {
@@ -865,14 +1028,14 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
         unsigned spins = 0;
         while (!dead && *reinterpret_cast<volatile int*>(&ctl->rows_closed) < w.n - (kClDepth - 2))
           if (++spins > kClSpinLimit) give_up();
-        event_a(w.n);
-        event_g(w.n);
+        event_a(w.n, w.tri);
+        event_g(w.n, w.tri);
       }
     } else {
       // second agent: b(n), f(n) -- off the critical path
       while (w.advance()) {
-        event_b(w.n);
-        if (rank == 0) event_f(w.n, w.r);
+        event_b(w.n, w.tri);
+        if (rank == 0) event_f(w.n, w);
         __syncwarp();
         if (lane == 0) *reinterpret_cast<volatile int*>(&ctl->rows_closed) = w.n + 1;
       }
@@ -883,23 +1046,43 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
   cluster_sync_all();
 }
 
+// ---- self-test of the give-up path --------------------------------------------------------------------
+// One warp waits on a barrier of its own that expects an arrival nobody makes. The wait is the kernels' bounded
+// wait with a limit of a few thousand polls; when it runs out the lane records the fact in the status word the
+// way give_up() does, and the kernel ends normally.
+constexpr unsigned kSelfTestPolls = 2048;
+__global__ void wait_timeout_selftest_kernel(int* status) {
+  __shared__ unsigned long long bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  unsigned spins = 0;
+  bool done = mbar_test(&bar, 0u);
+  while (!done && ++spins <= kSelfTestPolls) done = mbar_try(&bar, 0u);
+  if (!done) atomicExch(status, 1);
+}
+
 // ---- host side --------------------------------------------------------------------------------------
-template <typename T, int DIV, bool RS>
+template <typename T, int DIV, bool RS, bool TRI>
 inline cudaError_t cluster_prepare_one() {
-  cudaError_t e = cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV, RS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV, RS, TRI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kClSmemBytes));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV, RS>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  return cudaFuncSetAttribute(rowstats_cluster_kernel<T, DIV, RS, TRI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
 }
 template <typename T, int DIV>
 inline cudaError_t cluster_prepare() {
-  const cudaError_t e = cluster_prepare_one<T, DIV, false>();
-  return e != cudaSuccess ? e : cluster_prepare_one<T, DIV, true>();
+  cudaError_t e = cluster_prepare_one<T, DIV, false, false>();
+  if (e == cudaSuccess) e = cluster_prepare_one<T, DIV, true, false>();
+  if (e == cudaSuccess) e = cluster_prepare_one<T, DIV, true, true>();
+  return e;
 }
 
-// Co-resident clusters of this size. Both variants of the kernel have the same block size and shared memory;
-// the smaller answer of the two is taken so that one cached figure serves either.
-template <typename T, int DIV, bool RS>
+// Co-resident clusters of this size. The variants of the kernel have the same shared memory and nearly the
+// same block size; the smallest answer is taken so that one cached figure serves all of them.
+template <typename T, int DIV, bool RS, bool TRI>
 inline int cluster_max_active_one(int cs) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(cs));
@@ -913,7 +1096,7 @@ inline int cluster_max_active_one(int cs) {
   cfg.attrs = at;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, rowstats_cluster_kernel<T, DIV, RS>, &cfg) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveClusters(&n, rowstats_cluster_kernel<T, DIV, RS, TRI>, &cfg) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
@@ -921,7 +1104,8 @@ inline int cluster_max_active_one(int cs) {
 }
 template <typename T, int DIV>
 inline int cluster_max_active(int cs) {
-  return min(cluster_max_active_one<T, DIV, false>(cs), cluster_max_active_one<T, DIV, true>(cs));
+  return min(min(cluster_max_active_one<T, DIV, false, false>(cs), cluster_max_active_one<T, DIV, true, false>(cs)),
+             cluster_max_active_one<T, DIV, true, true>(cs));
 }
 
 // Per-device cache of the function attributes and of the number of co-resident clusters the device
@@ -1003,24 +1187,17 @@ inline bool cluster_shape_ok(const StageParams& P, int dtype) {
 // Picks the cluster size (or takes `forced_cs`; a forced size whose slice exceeds the ring is streamed
 // twice), and sizes the grid to the clusters that can be co-resident. Returns false when the shape does not
 // fit the kernel.
-inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, ClusterGeom* g) {
+inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, bool force_streamed, bool allow_triples, ClusterGeom* g) {
   if (!cluster_shape_ok(P, dtype)) return false;
   const int es = dtype == 0 ? 4 : 2;
   const long long rows = static_cast<long long>(P.B) * (P.K + P.K2);
   int cs = 0, slice = 0, chunks = 0;
-  if (forced_cs <= 0) {
-    // tuning aid: PYRAMIDSD_CLUSTER_SIZE=<1..16> overrides the library's choice for every call
-    static const int env_cs = [] { const char* e = std::getenv("PYRAMIDSD_CLUSTER_SIZE"); return e ? std::atoi(e) : 0; }();
-    if (env_cs > 0) forced_cs = env_cs;
-  }
-  // tuning aid: PYRAMIDSD_RESTREAM=1 takes the streamed-twice variant whenever a cluster size is forced
-  static const int env_rs = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM"); return e ? std::atoi(e) : 0; }();
   bool restream = false;
   if (forced_cs > 0) {
     if (forced_cs > kClMaxRanks) return false;
     cs = forced_cs;
     cluster_slices(P.V, es, cs, &slice, &chunks);
-    restream = chunks > kClSlots - 1 || env_rs > 0;   // a slice the ring cannot hold is streamed twice
+    restream = chunks > kClSlots - 1 || force_streamed;   // a slice the ring cannot hold is streamed twice
   } else {
     // the smallest cluster whose slice leaves at least five ring slots beyond a row (measured: 4 CTAs for
     // V = 128256 bf16, 5 for V = 152064 bf16); failing that, three slots
@@ -1074,12 +1251,15 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, Clu
   if (restream) {
     // slots of two chunks each (32 KB): six of them, `ra` for pass A and the rest for pass B
     g->ring = kClSlots / kClSubRS;
-    static const int env_ra = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_RA"); return e ? std::atoi(e) : 0; }();
-    g->ra = (env_ra >= 1 && env_ra <= kClSlots / kClSubRS - 1) ? env_ra : (kClSlots / kClSubRS) / 2;   // measured: 3 + 3 beats 2 + 4 and 4 + 2
-    static const int env_lead = [] { const char* e = std::getenv("PYRAMIDSD_RESTREAM_LEAD"); return e ? std::atoi(e) : 0; }();
-    g->lead = (env_lead >= 1 && env_lead <= kClDepth) ? env_lead : kClDepth;
+    g->ra = (kClSlots / kClSubRS) / 2;   // measured: 3 + 3 beats 2 + 4 and 4 + 2
+    g->lead = kClDepth;                  // measured: a shorter lead changes neither the time nor the DRAM traffic
   }
-  g->n_clusters = static_cast<int>(rows < max_active ? rows : max_active);
+  // A wrapper launch whose second row set pairs the first set's large rows (the qualifier's, in place) with a
+  // third tensor can be walked as row triples where it is streamed twice anyway.
+  g->tri = (allow_triples && restream && P.K2 > 0 && P.K2 <= P.K && P.n_valid == nullptr && P.small2 == P.large &&
+            P.seq_stride_small2 == P.seq_stride_large) ? 1 : 0;
+  const long long items = g->tri ? static_cast<long long>(P.B) * P.K : rows;
+  g->n_clusters = static_cast<int>(items < max_active ? items : max_active);
   return g->n_clusters > 0;
 }
 
@@ -1097,8 +1277,9 @@ inline cudaError_t cluster_launch_typed(const StageParams& P, const ClusterGeom&
   at[0].val.clusterDim.z = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  if (g.ra > 0) return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV, true>, P, g);
-  return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV, false>, P, g);
+  if (g.ra > 0 && g.tri) return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV, true, true>, P, g);
+  if (g.ra > 0) return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV, true, false>, P, g);
+  return cudaLaunchKernelEx(&cfg, rowstats_cluster_kernel<T, DIV, false, false>, P, g);
 }
 
 // Launches the statistics pass with the cluster kernel. Returns 0, or -2 when the launch was refused.

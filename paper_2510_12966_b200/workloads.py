@@ -148,3 +148,11 @@ def shard_batch(B: int, rank: int, world_size: int) -> Tuple[int, int]:
     base, rem = divmod(B, world_size)
     lo = rank * base + min(rank, rem)
     return lo, lo + base + (1 if rank < rem else 0)
+
+
+def shard_call(B: int, rank: int, world_size: int) -> Tuple[int, int, int]:
+    """What ``rank`` hands to a verification call on its shard of a batch of B sequences: the slice [lo, hi) of
+    every per-sequence tensor and the ``seq_index_base`` (= lo) that keeps each sequence's random draws those of
+    the unsharded call."""
+    lo, hi = shard_batch(B, rank, world_size)
+    return lo, hi, lo

@@ -6,6 +6,10 @@ oracle's own margin shows the decision was a near tie, and every such case is co
   (ii)  coin flip:      |u - min(1, p_large(x)/p_small(x))| < tol_coin (1e-5 fp32, 2e-3 bf16);
   (iii) inverse CDF:    the oracle's target u' * W lies within tol_cdf * W of the prefix-sum boundary that
                         separates the two tokens (1e-6 fp32, 1e-4 bf16).
+  (iv)  unresolved residual: the oracle's residual mass at the rejected row is below 1e-6 -- less than single
+                        precision, in which the library takes sum max(p, q) - 1, can tell from zero. The library
+                        then draws from p_large, as the rule for a zero residual says; its token must have
+                        positive p_large.
 A sequence whose accept length differs because of (i)/(ii) is not compared further.
 Floating-point outputs (divergence, residual mass, token probabilities) must agree within `tol_val`:
 1e-5 absolute with fp32 logits, 2e-3 absolute with bf16 logits.
@@ -20,6 +24,7 @@ TOL = {
     "bf16": dict(val=2e-3, coin=2e-3, cdf=1e-4),
 }
 TIE_DIV = 1e-4
+RESID_FLOOR = 1e-6
 
 
 def dtype_name(t: torch.Tensor) -> str:
@@ -39,7 +44,7 @@ def compare_stage(oracle, gpu, orc, zs_host, zl_host, *, dtype, mode, tau, seed,
     tol = TOL[dtype]
     B, K = orc["div"].shape
     nv = np.full(B, K, np.int32) if n_valid is None else np.clip(np.asarray(n_valid), 0, K)
-    rep = dict(rows=int(nv.sum()), seqs=B, tie_div=0, tie_coin=0, tie_cdf=0, max_err_div=0.0, max_err_prob=0.0,
+    rep = dict(rows=int(nv.sum()), seqs=B, tie_div=0, tie_coin=0, tie_cdf=0, tie_resid=0, max_err_div=0.0, max_err_prob=0.0,
                max_err_resid=0.0)
     valid = np.arange(K)[None, :] < nv[:, None]
     ok_rows = valid & (orc["row_flags"] == 0)
@@ -84,6 +89,10 @@ def compare_stage(oracle, gpu, orc, zs_host, zl_host, *, dtype, mode, tau, seed,
         p, _ = oracle.softmax(zl_host[b, Lo], inv_temperature)
         q, _ = oracle.softmax(zs_host[b, Lo], inv_temperature)
         w = np.maximum(p - q, 0.0)
+        if mode != 3 and 0 < orc["resid_mass"][b, Lo] < RESID_FLOOR:
+            assert p[tg] > 0, f"seq {b}: gpu token {tg} has zero probability under the large model"
+            rep["tie_resid"] += 1
+            continue
         if mode == 3 or not (orc["resid_mass"][b, Lo] > 0):
             w = p
         c = np.cumsum(w)

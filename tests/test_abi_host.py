@@ -17,7 +17,7 @@ def lib():
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "pyramidsd.h")).read()
+    text = "".join(open(os.path.join(ROOT, "include", h)).read() for h in sorted(os.listdir(os.path.join(ROOT, "include"))))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(pyramidsd_[a-z0-9_]+)\s*\(", text)))
 
@@ -32,18 +32,26 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_struct_layout_matches_header(lib, tmp_path):
-    """sizeof(psd_stage_args) as the C compiler sees it equals the ctypes mirror."""
+    """The argument structs as the C compiler sees them equal their ctypes mirrors: size and the offset of every field."""
     import subprocess
     from paper_2510_12966_b200 import binding
+    pairs = (("psd_stage_args", binding.StageArgs), ("psd_pyramid_args", binding.PyramidArgs), ("psd_lmhead_args", binding.LmheadArgs))
+    prints = []
+    for cname, mirror in pairs:
+        prints.append(f'printf("%zu", sizeof({cname}));')
+        for fname, _ in mirror._fields_:
+            prints.append(f'printf(" %zu", offsetof({cname}, {fname}));')
+        prints.append('printf("\\n");')
     src = tmp_path / "sz.c"
-    src.write_text('#include "pyramidsd.h"\n#include <stdio.h>\n#include <stddef.h>\n'
-                   'int main(void){printf("%zu %zu %zu\\n", sizeof(psd_stage_args), offsetof(psd_stage_args, workspace),'
-                   ' offsetof(psd_stage_args, kernel_variant));return 0;}\n')
+    src.write_text('#include "pyramidsd.h"\n#include "pyramidsd_diag.h"\n#include <stdio.h>\n#include <stddef.h>\n'
+                   'int main(void){' + "".join(prints) + 'return 0;}\n')
     exe = tmp_path / "sz"
-    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
-    size, off_ws, off_kv = map(int, subprocess.check_output([str(exe)]).split())
-    assert size == C.sizeof(binding.StageArgs)
-    assert off_ws == binding.StageArgs.workspace.offset and off_kv == binding.StageArgs.kernel_variant.offset
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    lines = subprocess.check_output([str(exe)]).decode().strip().splitlines()
+    for (cname, mirror), line in zip(pairs, lines):
+        nums = list(map(int, line.split()))
+        assert nums[0] == C.sizeof(mirror), cname
+        assert nums[1:] == [getattr(mirror, f).offset for f, _ in mirror._fields_], cname
 
 
 def test_version_and_status_strings(lib):
@@ -76,6 +84,21 @@ def test_invalid_arguments_are_rejected_before_any_launch(lib):
     assert lib.pyramidsd_verify_stage_ex(None) == binding.ERR_INVALID_ARG
     assert lib.pyramidsd_verify(None, None, None, None, 1, 4, 8, 100, 1, 0.1, 0.1, 0, 0, 0, None, None, None, None) \
         == binding.ERR_INVALID_ARG                                                        # K_q > K_d, NULLs
+    p = binding.PyramidArgs()
+    assert lib.pyramidsd_verify_ex(C.byref(p)) == binding.ERR_INVALID_ARG                # struct_size 0
+    p.struct_size = C.sizeof(binding.PyramidArgs)
+    p.B, p.K_d, p.K_q, p.V, p.mode_q = 0, 8, 4, 100, 7
+    assert lib.pyramidsd_verify_ex(C.byref(p)) == binding.ERR_INVALID_ARG                # unknown mode
+    p.mode_q, p.schedule = binding.ASSISTED, 9
+    assert lib.pyramidsd_verify_ex(C.byref(p)) == binding.ERR_INVALID_ARG                # unknown schedule
+    p.schedule, p.seq_index_base = binding.TWO_STAGE_FUSED_ROWS, -1
+    assert lib.pyramidsd_verify_ex(C.byref(p)) == binding.ERR_INVALID_ARG                # negative sequence base
+    p.seq_index_base = 5
+    assert lib.pyramidsd_verify_ex(C.byref(p)) == binding.OK                             # B == 0: a valid empty call
+    assert binding.pyramid_workspace_bytes(64, 16, 8, 128256, binding.BF16) == \
+        binding.workspace_bytes(64, 16, 128256, binding.BF16) + binding.workspace_bytes(64, 8, 128256, binding.BF16)
+    assert binding.pyramid_workspace_bytes(64, 4, 8, 128256, binding.BF16) == 0
+    assert lib.pyramidsd_verify_fused_lmhead_ex(None) == binding.ERR_INVALID_ARG
     assert lib.pyramidsd_verify_stage(None, None, None, 0, 4, 100, 0, 0.1, 0, 0, 0, None, None) == binding.OK  # B == 0
 
 

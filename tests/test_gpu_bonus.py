@@ -155,7 +155,7 @@ def test_pyramid_bonus_matches_oracle(psd, oracle, wl, mode, policy):
         out = psd.verify_bonus(zd.to(dev), zq.to(dev), zt.to(dev), tok.to(dev), tau_q, tau_t, mode, 7, 20)
         torch.cuda.synchronize()
     finally:
-        psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+        psd.set_two_stage_policy(psd.TWO_STAGE_DEFAULT)
     assert psd.last_status() == 0
     gpu = gpu_stage_to_numpy(out)
     zt_h = host_bits(zt)

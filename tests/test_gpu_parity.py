@@ -283,41 +283,23 @@ def test_streamed_twice_masked_flagged_and_identical_rows(psd, oracle, wl):
 
 
 def test_streamed_twice_equals_resident_bit_for_bit(psd, wl):
-    """PYRAMIDSD_RESTREAM=1 (read when the library first sizes a launch) makes every forced cluster size take
-    the streamed-twice variant, also where the slice would fit the ring. Its arithmetic is the resident
-    variant's, so a fresh process must return the very same bits: one chunk and several per slice, ragged
-    tails, more rows than clusters."""
-    import os, subprocess, sys, tempfile, textwrap
+    """PSD_KERNEL_CLUSTER_STREAMED makes a forced cluster size take the streamed-twice form also where the slice
+    would fit the ring. Its arithmetic is the resident form's, so it must return the very same bits: one chunk and
+    several per slice, ragged tails, more rows than clusters."""
     cases = [(7, 5, 2048, "f32", 1), (40, 8, 32768, "bf16", 1), (30, 8, 50000, "bf16", 2), (24, 16, 128256, "bf16", 4),
              (33, 7, 65536, "f32", 8)]
-    code = textwrap.dedent("""
-        import sys, torch
-        sys.path.insert(0, %r)
-        from paper_2510_12966_b200 import binding as psd, workloads as wl
-        dev = torch.device("cuda:0")
-        out = {}
-        for i, (B, K, V, dt, cs) in enumerate(%r):
-            zs, zl, tok = [t.to(dev) for t in wl.make_stage_inputs(B, K, V, dt, seed=500 + i, sigma=0.7)]
-            r = psd.verify_stage_ex(zs, zl, tok, 0.2, 2, 5, 6, kernel_variant=psd.KERNEL_CLUSTER, cluster_size=cs)
-            torch.cuda.synchronize()
-            assert psd.last_status() == 0
-            out[i] = {k: v.cpu() for k, v in r.items() if torch.is_tensor(v)}
-        torch.save(out, sys.argv[1])
-        print("ok")
-    """) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), cases)
-    with tempfile.TemporaryDirectory() as tmp:
-        path = os.path.join(tmp, "streamed.pt")
-        run = subprocess.run([sys.executable, "-c", code, path], env=dict(os.environ, PYRAMIDSD_RESTREAM="1"),
-                             capture_output=True, text=True, timeout=300)
-        assert run.returncode == 0 and "ok" in run.stdout, run.stderr[-2000:]
-        streamed = torch.load(path)
     dev = torch.device("cuda:0")
     for i, (B, K, V, dt, cs) in enumerate(cases):
         zs, zl, tok = [t.to(dev) for t in wl.make_stage_inputs(B, K, V, dt, seed=500 + i, sigma=0.7)]
         r = psd.verify_stage_ex(zs, zl, tok, 0.2, 2, 5, 6, kernel_variant=psd.KERNEL_CLUSTER, cluster_size=cs)
+        q = psd.verify_stage_ex(zs, zl, tok, 0.2, 2, 5, 6, kernel_variant=psd.KERNEL_CLUSTER_STREAMED, cluster_size=cs)
         torch.cuda.synchronize()
-        for k, v in streamed[i].items():
-            assert torch.equal(v.view(torch.int32), r[k].cpu().view(torch.int32)), (i, k)
+        assert psd.last_status() == 0
+        for k, v in r.items():
+            if torch.is_tensor(v):
+                assert torch.equal(v.view(torch.int32), q[k].view(torch.int32)), (i, k)
+    bad = psd.verify_stage_ex(zs, zl, tok, 0.2, kernel_variant=psd.KERNEL_CLUSTER_STREAMED, raise_on_error=False)
+    assert bad["status"] == psd.ERR_INVALID_ARG          # the streamed form wants an explicit cluster size
 
 
 @pytest.mark.parametrize("div_kind", [1, 2])
@@ -466,7 +448,7 @@ def test_two_stage_policies_give_the_same_results(psd, wl, B, K_d, K_q, V, dtype
         b = psd.verify(zd, zq, zt, tok, 0.3, 0.15, 2, 3, 4)
         torch.cuda.synchronize()
     finally:
-        psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+        psd.set_two_stage_policy(psd.TWO_STAGE_DEFAULT)
     for k in a:
         assert torch.equal(a[k], b[k]), k
     if B >= 9:
@@ -484,6 +466,7 @@ def test_two_stage_auto_policy_follows_the_window_lengths(psd, wl):
     ref_low = psd.verify(zd, zq, zt, tok, 0.02, 0.02, 0, 5, 6)      # tight threshold: short windows
     ref_full = psd.verify(zd, zq, zt, tok, 1.0, 1.0, 0, 5, 8)       # tau > ln 2: every window full
     torch.cuda.synchronize()
+    psd.set_two_stage_policy(psd.TWO_STAGE_DEFAULT)
     assert float(ref_low["accept_len_q"].float().mean()) < 3 and int(ref_full["accept_len"].min()) == K_q
     try:
         psd.set_two_stage_policy(psd.TWO_STAGE_AUTO)
@@ -497,7 +480,7 @@ def test_two_stage_auto_policy_follows_the_window_lengths(psd, wl):
                 assert torch.equal(ref[k], out[k]), k
         assert launches == [2, 4, 4, 2], launches
     finally:
-        psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+        psd.set_two_stage_policy(psd.TWO_STAGE_DEFAULT)
     assert psd.last_status() == 0
 
 

@@ -1,8 +1,11 @@
 """Multi-GPU path on CPU: the batch is sharded by sequence (sequences are independent, no collective on
 the data path), each rank verifies its own slice, and the gathered per-sequence results equal the
-unsharded run. Two `gloo` ranks; the per-rank verification is done by the CPU oracle (this is test code),
-which is enough to pin the host logic that matters here: the slice arithmetic and the fact that a
-sequence keeps its Philox row index `b*K + k` of the full batch wherever it is processed."""
+unsharded run. Two `gloo` ranks. What is under test here is the host logic of a sharded run: `shard_call`
+(the slice of every per-sequence tensor and the `seq_index_base` a rank passes with it), ragged shards, and
+the gather of the results. No GPU is present, so the verification of a slice is stood in for by the CPU
+oracle, told the same thing the library is told -- the index of the slice's first sequence; that the
+library itself returns the unsharded results for such a call is the GPU test
+`test_sequence_base_makes_shards_reproduce_the_whole_batch`, which cuts its batch with the same `shard_call`."""
 import os
 import socket
 
@@ -26,8 +29,8 @@ def _worker(rank, world, port, B, K_d, K_q, V, out_dir):
     import oracle
     from paper_2510_12966_b200 import workloads
     zd, zq, zt, tok = workloads.make_pyramid_inputs(B, K_d, K_q, V, "bf16", seed=77, sigma_q=0.5, sigma_d=0.9)
-    lo, hi = workloads.shard_batch(B, rank, world)
-    ids = np.arange(lo, hi)
+    lo, hi, seq_index_base = workloads.shard_call(B, rank, world)
+    ids = seq_index_base + np.arange(hi - lo)
     res = oracle.verify(workloads.to_host_bits(zd[lo:hi]), workloads.to_host_bits(zq[lo:hi]),
                         workloads.to_host_bits(zt[lo:hi]), tok[lo:hi].numpy(), np.float32(0.3), np.float32(0.2),
                         oracle.STRICT, 5, 8, seq_ids=ids)
