@@ -148,7 +148,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     binding.load_library()
     binding.set_stream()
-    binding.set_two_stage_policy({"separate": binding.TWO_STAGE_SEPARATE, "auto": binding.TWO_STAGE_AUTO}.get(args.two_stage, binding.TWO_STAGE_FUSED))
+    schedule = {"fused": binding.TWO_STAGE_FUSED, "separate": binding.TWO_STAGE_SEPARATE, "auto": binding.TWO_STAGE_AUTO,
+                "rows": binding.TWO_STAGE_FUSED_ROWS}[args.two_stage]
     cfg, w = workload_from_name(args.workload)
     if args.batch > 0:
         import dataclasses
@@ -168,9 +169,12 @@ def run_ours(args):
              for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")} for _ in range(n_bufs)]
     mode, seed = binding.FUZZY, 0
 
+    # every rank's B sequences are a slice of one global batch of world * B: the sequence base keeps each row's
+    # random draws those of the global batch
     def step(i):
         zd, zq, zt, tok = rounds[i % n_bufs]
-        binding.verify(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, seed, 2 * i, out=outs[i % n_bufs])
+        binding.verify_ex(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, None, seed, 2 * i, seq_index_base=rank * w.B,
+                          schedule=schedule, want_rows=False, want_window=False, out=outs[i % n_bufs])
 
     def barrier():
         if world > 1:
@@ -184,15 +188,19 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     sampler.start()
     launches0 = binding.launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev0.record()
-    for i in range(args.steps):
-        step(args.warmup + i)
-    ev1.record()
-    barrier()
-    ms_total = ev0.elapsed_time(ev1)
-    launches = binding.launch_count() - launches0
+    # The timed region is K steps between a barrier + synchronize on both sides, CUDA events around it. It is
+    # taken `regions` times back to back (K steps can be a few milliseconds) and the median region is reported.
+    region_ms = []
+    for _ in range(args.regions):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for i in range(args.steps):
+            step(args.warmup + i)
+        ev1.record()
+        barrier()
+        region_ms.append(ev0.elapsed_time(ev1))
+    launches = (binding.launch_count() - launches0) // args.regions
     clocks = sampler.stop()
     # The same K steps once more with an event pair around every launch, for the per-kernel durations of the
     # roofline. Kept out of the pass above: the event records between launches cost a few microseconds each.
@@ -212,10 +220,24 @@ def run_ours(args):
     row_bytes = 2 * w.V * es
     rs_bytes = n_pos * row_bytes   # the statistics kernel streams each verified row pair once
     timed_cap = 4096               # launches the library's event timing holds; beyond it only the first ones are timed
-    launches_per_step = {"fused": 2, "separate": 4}.get(args.two_stage) or (4 if launches >= 3 * args.steps else 2)
+    launches_per_step = {"fused": 2, "rows": 2, "separate": 4}.get(args.two_stage) or (4 if launches >= 3 * args.steps else 2)
     if launches_per_step * args.steps > timed_cap:
         steps_timed = timed_cap // launches_per_step
         rs_bytes = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(steps_timed)) * row_bytes
+
+    # ---- acceptance rates and near ties of the rounds that were timed (one more call per round, with rows) ----
+    acc = {"rows_q": 0, "acc_q": 0, "rows_t": 0, "acc_t": 0, "near_q": 0, "near_t": 0}
+    for zd, zq, zt, tok in rounds:
+        o = binding.verify_ex(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, None, seed, 0, seq_index_base=rank * w.B, schedule=schedule)
+        torch.cuda.synchronize()
+        nw = o["n_window"]
+        inside = torch.arange(w.K_q, device=dev)[None, :] < nw[:, None]
+        acc["rows_q"] += w.B * w.K_d
+        acc["acc_q"] += int((o["div_q"] <= w.tau_q).sum())
+        acc["rows_t"] += int(nw.sum())
+        acc["acc_t"] += int(((o["div_t"] <= w.tau_t) & inside).sum())
+        acc["near_q"] += int(((o["div_q"] - w.tau_q).abs() < 1e-4).sum())
+        acc["near_t"] += int((((o["div_t"] - w.tau_t).abs() < 1e-4) & inside).sum())
 
     # ---- end to end through the host-pointer entry point: H2D of the step's inputs + D2H of its results ----
     e2e = None
@@ -242,9 +264,9 @@ def run_ours(args):
     # ---- max over ranks, sum of positions ----
     if world > 1:
         import torch.distributed as dist
-        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        t = torch.tensor(region_ms + [e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e_max = t[0].item(), t[1].item()
+        region_ms, ms_e2e_max = t[:-1].tolist(), t[-1].item()
         c = torch.tensor([n_pos, e2e["pos"] if e2e else 0, launches], device=dev, dtype=torch.int64)
         dist.all_reduce(c, op=dist.ReduceOp.SUM)
         n_pos_all, e2e_pos_all, launches_all = int(c[0]), int(c[1]), int(c[2])
@@ -253,6 +275,7 @@ def run_ours(args):
     else:
         n_pos_all, e2e_pos_all, launches_all = n_pos, (e2e["pos"] if e2e else 0), launches
 
+    ms_total = statistics.median(region_ms)   # per region: the max over ranks
     if rank == 0:
         peaks, peak_kind = load_peaks()
         value = n_pos_all / (ms_total * 1e-3)
@@ -261,15 +284,24 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "timed_regions": args.regions, "ms_per_step_min_max": [min(region_ms) / args.steps, max(region_ms) / args.steps],
             "config": {"workload": f"{w.name}: B={w.B} per GPU, V={w.V}, {w.dtype} logits, K_draft={w.K_d}, "
                                    f"K_qual={w.K_q}, tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0, two-stage schedule {args.two_stage}",
-                       "logits_dtype": w.dtype, "positions_per_step": n_pos / args.steps,
+                       "logits_dtype": w.dtype, "arithmetic": "f32 (logits widened from %s)" % w.dtype,
+                       "positions_per_step": n_pos / args.steps,
+                       "acceptance": {"beta_qualifier_stage": acc["acc_q"] / max(acc["rows_q"], 1),
+                                      "beta_target_stage": acc["acc_t"] / max(acc["rows_t"], 1),
+                                      "rows_within_1e-4_of_tau": {"qualifier_stage": acc["near_q"], "target_stage": acc["near_t"]},
+                                      "rows": {"qualifier_stage": acc["rows_q"], "target_stage": acc["rows_t"]}},
                        "l2_policy": "inputs larger than L2 (one round = %.0f MB), two rounds alternate" %
                                     ((2 * w.K_d + w.K_q) * w.B * w.V * es / 1e6),
                        "gb_per_s_whole_step": n_pos_all * row_bytes / (ms_total * 1e-3) / 1e9},
             "roofline": {"bound": "hbm", "kernel": "rowstats (per-row softmax/divergence statistics)",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
+                         "bytes_counted": "2*V*s per verified row pair (the call made); the least a two-stage call can "
+                                          "read, qualifier rows once, is (2*K_d + K_q)/(2*(K_d + K_q)) of it",
+                         "frac_on_fused_minimum_bytes": achieved / peaks["hbm_gbs"] * (2 * w.K_d + w.K_q) / (2.0 * (w.K_d + w.K_q)),
                          "traffic": None, "launches": n_rs, "avg_launch_ms": ms_rs / max(n_rs, 1),
                          "finalize_ms_per_launch": ms_fin / max(n_fin, 1),
                          # statistics time per step of the event pass over the step time of the timed pass
@@ -292,10 +324,17 @@ def run_ours(args):
             line["e2e"] = {"value": e2e_pos_all / (e2e["ms"] * 1e-3), "unit": UNIT,
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": e2e["ms"] / e2e["steps"], "steps": e2e["steps"]}
+        # Sec. 3.3's throughput model fed with the acceptance rates measured above and assumed model speeds
+        b_qd, b_tq = acc["acc_q"] / max(acc["rows_q"], 1), acc["acc_t"] / max(acc["rows_t"], 1)
+        line["analytic_model"] = {
+            "beta_qd": b_qd, "beta_tq": b_tq, "ell_d": w.K_d, "ell_q": w.K_q,
+            "assumed_tokens_per_s": {"draft": args.v_draft, "qualifier": args.v_qual, "target": args.v_target},
+            "sd_tokens_per_s": binding.model_sd_throughput(b_tq, w.K_q, args.v_qual, args.v_target),
+            "psd_tokens_per_s": binding.model_psd_throughput(b_qd, w.K_d, args.v_draft, args.v_qual, b_tq, w.K_q, args.v_target)}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, rounds)
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
-        traffic = read_profile_traffic(w) if args.two_stage == "fused" else None
+        traffic = read_profile_traffic(w) if args.two_stage in ("fused", "auto") and launches_per_step == 2 else None
         if traffic is not None:
             line["roofline"]["traffic"] = traffic
         print(json.dumps(line))
@@ -449,6 +488,8 @@ def run_fused(args):
         "roofline": {"bound": "tensor", "kernel": "lmhead_sweep (two tcgen05 GEMM sweeps + row reduction)",
                      "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s", "frac": achieved / tensor_peak,
                      "frac_of_burst": achieved / peaks["bf16_tflops"],
+                     "flops_counted": "both GEMM sweeps (what the tensor pipe executes); the method needs one h x W^T",
+                     "achieved_on_one_gemm": achieved / 2, "frac_on_one_gemm": achieved / 2 / tensor_peak,
                      "peak_kind": tensor_kind, "traffic": None, "launches": n_sw,
                      "avg_launch_ms": ms_sweeps / max(n_sw, 1), "finalize_ms_per_launch": ms_fin / max(n_fin, 1),
                      "weight_gb_per_s": 2 * w.V * w.d_model * 2 * n_sw / (ms_sweeps * 1e-3) / 1e9 if ms_sweeps > 0 else 0.0},
@@ -498,9 +539,18 @@ def cpu_baseline(w, rounds):
         dt += time.perf_counter() - t0
         n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
         pos += w.B * w.K_d + int(n2.sum())
+    # the same oracle on one core, on the first sequences of the first round
+    nb = min(4, w.B)
+    zd, zq, zt, tok = [workloads.to_host_bits(t[:nb]) for t in rounds[0]]
+    t0 = time.perf_counter()
+    out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, n_threads=1)
+    dt1 = time.perf_counter() - t0
+    pos1 = nb * w.K_d + int(np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0)).sum())
     return {"value": pos / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{len(rounds)} rounds of {w.name} ({w.B} sequences each, {pos} positions, {dt:.2f} s wall, "
-                      f"about {dt * cores:.0f} core-seconds)"}
+                      f"about {dt * cores:.0f} core-seconds)",
+            "one_core": {"value": pos1 / dt1, "unit": UNIT, "cores": 1,
+                         "sample": f"first {nb} sequences of one round ({pos1} positions, {dt1:.2f} s)"}}
 
 
 def run_reference(args):
@@ -512,7 +562,7 @@ def run_reference(args):
     from paper_2510_12966_b200 import workloads
     oracle.build()
     cfg, w = workload_from_name(args.workload)
-    seqs = args.cpu_seqs
+    seqs = args.cpu_seqs if args.cpu_seqs > 0 else w.B
     cores = os.cpu_count() or 1
     rounds = [workloads.workload_inputs(cfg, i, device="cpu", B=seqs) for i in range(2)]
     hosts = [[workloads.to_host_bits(t) for t in r] for r in rounds]
@@ -546,16 +596,21 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)    # ~0.15 s of timed work: long enough for the clock sampler
+    ap.add_argument("--steps", type=int, default=200)    # x 5 regions: ~0.25 s of timed work, long enough for the clock sampler
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--logits-dtype", choices=["bf16", "f32"], default=None, help="override the workload's logits dtype (cfg4's fp32 run)")
-    ap.add_argument("--cpu-seqs", type=int, default=32, help="sequences per step of the CPU-oracle reference arm")
+    ap.add_argument("--cpu-seqs", type=int, default=0, help="sequences per step of the CPU-oracle reference arm (0: the workload's B)")
+    ap.add_argument("--regions", type=int, default=5, help="the K-step timed region is taken this many times; the median is reported")
+    ap.add_argument("--v-draft", type=float, default=900.0, help="assumed draft-model speed (tokens/s) for the analytic model line")
+    ap.add_argument("--v-qual", type=float, default=400.0, help="assumed qualifier-model speed (tokens/s)")
+    ap.add_argument("--v-target", type=float, default=150.0, help="assumed target-model speed (tokens/s)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (small profiling cases)")
     ap.add_argument("--vocab", type=int, default=0, help="override the vocabulary size V of cfg5 (small profiling cases)")
-    ap.add_argument("--two-stage", choices=["fused", "separate", "auto"], default="fused",
-                    help="schedule of the two stages (same results): one statistics launch for both, or stage by stage")
+    ap.add_argument("--two-stage", choices=["fused", "separate", "auto", "rows"], default="auto",
+                    help="schedule of the two stages (same results): one statistics launch for both (row pairs, or row "
+                         "triples with `rows`), stage by stage, or the library's per-call choice (its default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -37,8 +37,10 @@
  *     one host thread or several, do not share scratch. Such a buffer is created with cudaMalloc the
  *     first time a stream is used and grown when a larger call arrives (growing waits for that stream's
  *     earlier work, frees, allocates). At most PSD_MAX_STREAMS streams per device get buffers; a call on
- *     yet another stream without a workspace returns PSD_ERR_WORKSPACE. Two host threads that share one
- *     stream are serialised for the duration of the enqueue.
+ *     yet another stream without a workspace returns PSD_ERR_WORKSPACE (see pyramidsd_release_stream). Two host
+ *     threads that share one stream are serialised for the duration of the enqueue. A stage or pyramid call
+ *     that brings its workspace uses no library buffer at all (its status word sits in the workspace's last
+ *     256 bytes and is cleared on the stream): it allocates nothing and synchronises nothing.
  *   - Return value: PSD_OK or a negative psd_status. Arguments are validated on the host before any
  *     launch; nothing is launched on error. Device-side bounded waits that give up report
  *     PSD_ERR_TIMEOUT through pyramidsd_last_status().
@@ -350,6 +352,11 @@ int pyramidsd_set_two_stage_policy(int policy);
 /* Stream used by the entry points that carry no stream argument (a cudaStream_t; NULL = legacy default
  * stream). Per host thread. */
 int pyramidsd_set_stream(void* cuda_stream);
+
+/* Gives back the library-owned buffers of `cuda_stream` on the current device (after waiting for the stream's work)
+ * and frees its place among the PSD_MAX_STREAMS streams; call it before destroying a stream the library has been
+ * used on. PSD_OK also when the stream owns nothing. */
+int pyramidsd_release_stream(void* cuda_stream);
 
 /* Synchronises the stream of this host thread's most recent call (the library stream if there was none) and
  * returns PSD_OK, PSD_ERR_TIMEOUT if a device-side bounded wait gave up on that stream since its status was last

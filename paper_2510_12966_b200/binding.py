@@ -23,7 +23,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, 
 
 EXPORTS = (
     "pyramidsd_verify_stage", "pyramidsd_verify_stage_ex", "pyramidsd_verify", "pyramidsd_verify_ex", "pyramidsd_verify_bonus",
-    "pyramidsd_verify_host", "pyramidsd_pyramid_workspace_bytes", "pyramidsd_selftest_wait_timeout",
+    "pyramidsd_verify_host", "pyramidsd_pyramid_workspace_bytes", "pyramidsd_selftest_wait_timeout", "pyramidsd_release_stream",
     "pyramidsd_verify_stage_noalloc", "pyramidsd_verify_fused_lmhead", "pyramidsd_verify_fused_lmhead_ex",
     "pyramidsd_model_sd_throughput", "pyramidsd_model_psd_throughput", "pyramidsd_set_two_stage_policy",
     "pyramidsd_row_uniforms", "pyramidsd_workspace_bytes", "pyramidsd_set_stream", "pyramidsd_last_status", "pyramidsd_launch_count",
@@ -128,6 +128,8 @@ def load_library(path: Optional[str] = None):
     lib.pyramidsd_verify_fused_lmhead_ex.restype = i32
     lib.pyramidsd_pyramid_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     lib.pyramidsd_pyramid_workspace_bytes.restype = C.c_size_t
+    lib.pyramidsd_release_stream.argtypes = [vp]
+    lib.pyramidsd_release_stream.restype = i32
     lib.pyramidsd_selftest_wait_timeout.argtypes = [vp]
     lib.pyramidsd_selftest_wait_timeout.restype = i32
     pyr = [vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, u64, u64, vp, vp, vp, vp]
@@ -213,6 +215,11 @@ def set_two_stage_policy(policy: int) -> None:
 
 def last_status() -> int:
     return load_library().pyramidsd_last_status()
+
+
+def release_stream(stream) -> None:
+    """``pyramidsd_release_stream``: free the library-owned scratch of a stream before destroying it."""
+    _check(load_library().pyramidsd_release_stream(C.c_void_p(stream.cuda_stream)), "pyramidsd_release_stream")
 
 
 def selftest_wait_timeout(stream=None) -> int:
@@ -432,15 +439,19 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
 def verify_ex(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode_q=FUZZY, mode_t=None,
               philox_seed=0, offset=0, *, seq_index_base=0, target_has_bonus_row=False, schedule=TWO_STAGE_DEFAULT,
               inv_temperature=0.0, div_kind=DIV_JS, want_rows=True, want_window=True, workspace=None, stream=None,
-              kernel_variant=KERNEL_AUTO, raise_on_error=True):
+              kernel_variant=KERNEL_AUTO, raise_on_error=True, out=None):
     """``pyramidsd_verify_ex``: the two-stage pyramid with per-stage modes, a sequence base, per-row outputs, the
-    window, a caller workspace and an explicit schedule. Returns a dict of device tensors (+ "status")."""
+    window, a caller workspace and an explicit schedule. Returns a dict of device tensors (+ "status"). ``out`` may
+    bring the four [B] int32 result tensors (keys accept_len_q, next_token_q, accept_len, next_token)."""
     B, K_d, V = logits_draft.shape
     K_q = logits_target.shape[1] - (1 if target_has_bonus_row else 0)
     assert logits_qual.shape == logits_draft.shape and logits_target.shape[0] == B and logits_target.shape[2] == V
     dev = logits_draft.device
-    out = {k: torch.empty(B, dtype=torch.int32, device=dev)
-           for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+    if out is None:
+        out = {k: torch.empty(B, dtype=torch.int32, device=dev)
+               for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+    else:
+        out = dict(out)
     a = PyramidArgs()
     a.struct_size = C.sizeof(PyramidArgs)
     a.dtype = dtype_code(logits_draft)
@@ -455,7 +466,7 @@ def verify_ex(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau
     a.philox_seed, a.philox_offset, a.seq_index_base = int(philox_seed), int(offset), int(seq_index_base)
     a.target_has_bonus_row, a.schedule = (1 if target_has_bonus_row else 0), int(schedule)
     for k in ("accept_len_q", "next_token_q", "accept_len", "next_token"):
-        setattr(a, "out_" + k, out[k].data_ptr())
+        setattr(a, "out_" + k, _dev_ptr(out[k], torch.int32, k))
     if want_rows:
         for k, n in (("div_q", K_d), ("resid_q", K_d), ("div_t", K_q), ("resid_t", K_q)):
             out[k] = torch.empty((B, n), dtype=torch.float32, device=dev)

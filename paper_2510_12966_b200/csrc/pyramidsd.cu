@@ -71,8 +71,11 @@ struct DeviceState {
 };
 constexpr int kFillCap = 4096;
 DeviceState g_dev[kMaxDevices];
-// what pyramidsd_last_status() looks at: the scratch entry of this thread's most recent call
+// what pyramidsd_last_status() looks at: the stream and the status word of this thread's most recent call (the word
+// sits in a scratch entry, or in the tail of the caller's workspace)
 thread_local StreamScratch* t_last_scratch = nullptr;
+thread_local int* t_last_status = nullptr;
+thread_local cudaStream_t t_last_stream = nullptr;
 
 int current_device_state(DeviceState** out) {
   int dev = 0;
@@ -344,17 +347,16 @@ cudaStream_t pick_stream(const psd_stage_args* a) {
 
 // Runs one stage with the scratch entry `ss` (held by the caller); `window_out`/`n_window_out`/`K_window` non-null
 // make the finalisation also build the stage-2 window of the wrapper.
-int run_stage_locked(const psd_stage_args* a, StreamScratch* ss, cudaStream_t stream, int32_t* window_out,
+int run_stage_locked(const psd_stage_args* a, StreamScratch* ss, int* status, cudaStream_t stream, int32_t* window_out,
                      int32_t* n_window_out, int K_window, int32_t* fill_out = nullptr) {
-  int rc = ensure_status(ss);
-  if (rc != PSD_OK) return rc;
+  int rc = PSD_OK;
   void* ws = a->workspace;
   if (ws == nullptr) {
     rc = grow(ss, &ss->ws, &ss->ws_bytes, stage_workspace_bytes(a->B, a->K));
     if (rc != PSD_OK) return rc;
     ws = ss->ws;
   }
-  StageParams P = make_params(a, ws, ss->status);
+  StageParams P = make_params(a, ws, status);
   P.window = window_out;
   P.n_window = n_window_out;
   P.K_window = K_window;
@@ -372,12 +374,21 @@ int run_stage(const psd_stage_args* a) {
   if (rc != PSD_OK) return rc;
   if (a->B == 0) return PSD_OK;
   const cudaStream_t stream = pick_stream(a);
+  if (a->workspace != nullptr) {
+    // the caller's workspace holds everything, the status word in its last 256 bytes: no library buffer, no allocation
+    int* status = reinterpret_cast<int*>(static_cast<char*>(a->workspace) + stage_workspace_bytes(a->B, a->K) - kAlign);
+    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return PSD_ERR_CUDA;
+    t_last_scratch = nullptr; t_last_status = status; t_last_stream = stream;
+    return run_stage_locked(a, nullptr, status, stream, nullptr, nullptr, 0);
+  }
   StreamScratch* ss = nullptr;
   rc = scratch_for(stream, &ss);
   if (rc != PSD_OK) return rc;
   std::lock_guard<std::mutex> lock(ss->mu);
-  t_last_scratch = ss;
-  return run_stage_locked(a, ss, stream, nullptr, nullptr, 0);
+  rc = ensure_status(ss);
+  if (rc != PSD_OK) return rc;
+  t_last_scratch = ss; t_last_status = ss->status; t_last_stream = stream;
+  return run_stage_locked(a, ss, ss->status, stream, nullptr, nullptr, 0);
 }
 
 size_t pyramid_workspace_bytes(int B, int K_d, int K_q) { return stage_workspace_bytes(B, K_d) + stage_workspace_bytes(B, K_q); }
@@ -401,12 +412,10 @@ int validate_pyramid(const psd_pyramid_args* a) {
 }
 
 // Both stages of the pyramid with the scratch entry `ss` held by the caller.
-int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, cudaStream_t stream) {
+int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* status, cudaStream_t stream) {
   const int B = a->B, K_d = a->K_d, K_q = a->K_q, V = a->V, dtype = a->dtype;
   DeviceState* ds = nullptr;
   int rc = current_device_state(&ds);
-  if (rc != PSD_OK) return rc;
-  rc = ensure_status(ss);
   if (rc != PSD_OK) return rc;
   // scratch: [stage-1 workspace][stage-2 workspace]; the window and its length live in stage 1's tail unless the
   // caller wants them
@@ -513,21 +522,21 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, cudaSt
       psd::ClusterGeom g{};
       if (variant != PSD_KERNEL_BASELINE && psd::cluster_geometry(PS, dtype, 0, false, false, &g)) s1.cluster_size = s2.cluster_size = g.cs;
     }
-    rc = run_stage_locked(&s1, ss, stream, window, n_window, K_q, fill_out);
+    rc = run_stage_locked(&s1, ss, status, stream, window, n_window, K_q, fill_out);
     if (rc != PSD_OK) return rc;
-    return run_stage_locked(&s2, ss, stream, nullptr, nullptr, 0);
+    return run_stage_locked(&s2, ss, status, stream, nullptr, nullptr, 0);
   }
   // Two launches for the whole pyramid. The statistics of both stages are independent of the stage-1
   // outcome (only the token looked up in a row and the window length depend on it), so one launch of
   // the statistics kernel covers the B*K_d stage-1 rows and the B*K_q stage-2 rows; one finalisation
   // kernel then runs stage 1, builds the window, and runs stage 2 per sequence.
-  StageParams P1 = make_params(&s1, s1.workspace, ss->status);
+  StageParams P1 = make_params(&s1, s1.workspace, status);
   P1.window = window;
   P1.n_window = n_window;
   P1.K_window = K_q;
   P1.fill_out = fill_out;
   P1.fill_cap = kFillCap;
-  const StageParams P2 = make_params(&s2, s2.workspace, ss->status);
+  const StageParams P2 = make_params(&s2, s2.workspace, status);
   StageParams PS = P1;
   PS.small2 = P2.small;
   PS.large2 = P2.large;
@@ -566,12 +575,20 @@ int verify_two_stage(const psd_pyramid_args* a) {
   if (rc != PSD_OK) return rc;
   if (a->B == 0) return PSD_OK;
   const cudaStream_t stream = pick_stream(a);
+  if (a->workspace != nullptr) {
+    int* status = reinterpret_cast<int*>(static_cast<char*>(a->workspace) + pyramid_workspace_bytes(a->B, a->K_d, a->K_q) - kAlign);
+    if (cudaMemsetAsync(status, 0, sizeof(int), stream) != cudaSuccess) return PSD_ERR_CUDA;
+    t_last_scratch = nullptr; t_last_status = status; t_last_stream = stream;
+    return verify_two_stage_locked(a, nullptr, status, stream);
+  }
   StreamScratch* ss = nullptr;
   rc = scratch_for(stream, &ss);
   if (rc != PSD_OK) return rc;
   std::lock_guard<std::mutex> lock(ss->mu);
-  t_last_scratch = ss;
-  return verify_two_stage_locked(a, ss, stream);
+  rc = ensure_status(ss);
+  if (rc != PSD_OK) return rc;
+  t_last_scratch = ss; t_last_status = ss->status; t_last_stream = stream;
+  return verify_two_stage_locked(a, ss, ss->status, stream);
 }
 
 psd_pyramid_args basic_pyramid_args(const void* logits_draft, const void* logits_qual, const void* logits_target,
@@ -663,7 +680,9 @@ int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, con
   rc = scratch_for(s, &ss);
   if (rc != PSD_OK) return rc;
   std::lock_guard<std::mutex> lock(ss->mu);
-  t_last_scratch = ss;
+  rc = ensure_status(ss);
+  if (rc != PSD_OK) return rc;
+  t_last_scratch = ss; t_last_status = ss->status; t_last_stream = s;
   const size_t es = elem_size(dtype);
   const size_t n_d = static_cast<size_t>(B) * K_d * V * es, n_t = static_cast<size_t>(B) * K_q * V * es;
   const size_t n_tok = static_cast<size_t>(B) * K_d * 4;
@@ -681,7 +700,7 @@ int pyramidsd_verify_host(const void* logits_draft, const void* logits_qual, con
   a.logits_draft = ss->stage[0]; a.logits_qual = ss->stage[1]; a.logits_target = ss->stage[2];
   a.draft_tokens = static_cast<const int32_t*>(ss->stage[3]);
   a.out_accept_len_q = o; a.out_next_token_q = o + B; a.out_accept_len = o + 2 * B; a.out_next_token = o + 3 * B;
-  rc = verify_two_stage_locked(&a, ss, s);
+  rc = verify_two_stage_locked(&a, ss, ss->status, s);
   if (rc != PSD_OK) return rc;
   int32_t* dst[4] = {out_accept_len_q, out_next_token_q, out_accept_len, out_next_token};
   for (int i = 0; i < 4; ++i)
@@ -786,12 +805,12 @@ int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args) {
   int rc = scratch_for(stream, &ss);
   if (rc != PSD_OK) return rc;
   std::lock_guard<std::mutex> lock(ss->mu);
-  t_last_scratch = ss;
   const int n_tiles = (V + psd::kLmN - 1) / psd::kLmN;
   const size_t per = static_cast<size_t>(M) * n_tiles;
   const size_t bytes = align_up(per * sizeof(float2)) * 2 + align_up(per * sizeof(float4)) + align_up(static_cast<size_t>(M) * sizeof(float4));
   rc = ensure_status(ss);
   if (rc != PSD_OK) return rc;
+  t_last_scratch = ss; t_last_status = ss->status; t_last_stream = stream;
   rc = grow(ss, &ss->lm_ws, &ss->lm_ws_bytes, bytes);
   if (rc != PSD_OK) return rc;
   // tensor maps: hidden [M, d] and W^T [V, d], bf16, K innermost, boxes of 64 x 256 / 64 x 128, 128-byte swizzle
@@ -986,16 +1005,40 @@ int pyramidsd_set_stream(void* cuda_stream) {
   return PSD_OK;
 }
 
+int pyramidsd_release_stream(void* cuda_stream) {
+  const cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  DeviceState* ds = nullptr;
+  int rc = current_device_state(&ds);
+  if (rc != PSD_OK) return rc;
+  std::lock_guard<std::mutex> table(ds->mu);
+  for (auto& e : ds->streams) {
+    if (!e.used || e.stream != stream) continue;
+    std::lock_guard<std::mutex> lock(e.mu);
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return PSD_ERR_CUDA;
+    void** owned[] = {&e.ws, reinterpret_cast<void**>(&e.status), &e.stage[0], &e.stage[1], &e.stage[2], &e.stage[3], &e.out4, &e.lm_ws};
+    for (void** p : owned) {
+      if (*p) cudaFree(*p);
+      *p = nullptr;
+    }
+    e.ws_bytes = e.out4_bytes = e.lm_ws_bytes = 0;
+    for (size_t& b : e.stage_bytes) b = 0;
+    if (t_last_scratch == &e) { t_last_scratch = nullptr; t_last_status = nullptr; }
+    e.used = false;
+    e.stream = nullptr;
+  }
+  return PSD_OK;
+}
+
 int pyramidsd_last_status(void) {
+  if (t_last_status == nullptr) return cudaStreamSynchronize(t_stream) == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
   StreamScratch* ss = t_last_scratch;
-  if (ss == nullptr) return cudaStreamSynchronize(t_stream) == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
-  std::lock_guard<std::mutex> lock(ss->mu);
-  if (cudaStreamSynchronize(ss->stream) != cudaSuccess) return PSD_ERR_CUDA;
-  if (!ss->status) return PSD_OK;
+  std::unique_lock<std::mutex> lock;
+  if (ss != nullptr) lock = std::unique_lock<std::mutex>(ss->mu);
+  if (cudaStreamSynchronize(t_last_stream) != cudaSuccess) return PSD_ERR_CUDA;
   int host = 0;
-  if (cudaMemcpy(&host, ss->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PSD_ERR_CUDA;
+  if (cudaMemcpy(&host, t_last_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PSD_ERR_CUDA;
   if (host != 0) {
-    cudaMemset(ss->status, 0, sizeof(int));
+    cudaMemset(t_last_status, 0, sizeof(int));
     return PSD_ERR_TIMEOUT;
   }
   return PSD_OK;
@@ -1007,9 +1050,9 @@ int pyramidsd_selftest_wait_timeout(void* cuda_stream) {
   int rc = scratch_for(stream, &ss);
   if (rc != PSD_OK) return rc;
   std::lock_guard<std::mutex> lock(ss->mu);
-  t_last_scratch = ss;
   rc = ensure_status(ss);
   if (rc != PSD_OK) return rc;
+  t_last_scratch = ss; t_last_status = ss->status; t_last_stream = stream;
   psd::wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(ss->status);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return check_launch();

@@ -305,6 +305,22 @@ def test_streams_and_host_threads_do_not_share_scratch(psd, wl):
     for k, v in ref.items():
         if torch.is_tensor(v):
             assert torch.equal(bits(v), bits(out[k])), k
+    # more streams than the library keeps scratch for: the call says so, releasing a stream makes room again
+    streams = [torch.cuda.Stream() for _ in range(20)]
+    codes = [psd.verify_ex(*t, 0.3, 0.15, stream=st, raise_on_error=False, want_rows=False, want_window=False)["status"] for st in streams]
+    torch.cuda.synchronize()
+    assert codes[0] == psd.OK and psd.ERR_WORKSPACE in codes and set(codes) <= {psd.OK, psd.ERR_WORKSPACE}
+    refused = streams[codes.index(psd.ERR_WORKSPACE)]
+    with_ws = psd.verify_ex(*t, 0.3, 0.15, psd.FUZZY_SD_FALLBACK, None, 2, 8, stream=refused, workspace=ws)   # needs no library buffer
+    refused.synchronize()
+    assert torch.equal(with_ws["accept_len"], ref["accept_len"]) and psd.last_status() == psd.OK
+    for st, code in zip(streams, codes):
+        if code == psd.OK:
+            psd.release_stream(st)
+    out = psd.verify_ex(*t, 0.3, 0.15, psd.FUZZY_SD_FALLBACK, None, 2, 8, stream=refused)
+    refused.synchronize()
+    assert torch.equal(out["accept_len"], ref["accept_len"]) and torch.equal(out["next_token"], ref["next_token"])
+    psd.release_stream(refused)
     small = torch.empty(need - 256, dtype=torch.uint8, device=dev)
     assert psd.verify_ex(*t, 0.3, 0.15, workspace=small, raise_on_error=False)["status"] == psd.ERR_WORKSPACE
 
