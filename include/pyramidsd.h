@@ -335,7 +335,8 @@ size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype);
  *                           a later call with the same B and K_q on this device reads whatever lengths are there
  *                           -- those of a recent call -- and runs stage by stage when the unfilled part of the
  *                           windows is more than a tenth of all rows and the batch has at least 1024 rows, else
- *                           in two launches. The first call of a shape runs in two launches.
+ *                           in two launches, over row triples where they apply (FUSED_ROWS below). The first call
+ *                           of a shape runs in two launches.
  *   PSD_TWO_STAGE_FUSED_ROWS two launches like FUSED, but positions k < K_q are walked as row triples (draft,
  *                           qualifier, target): the qualifier row, which stage 1 uses as its large model and
  *                           stage 2 as its small one (Fig. 1), is read, widened and normalised once --

@@ -68,6 +68,7 @@ struct DeviceState {
   int32_t* fill_host = nullptr;
   int32_t* fill_dev = nullptr;
   int fill_B = 0, fill_Kq = 0;   // the shape those lengths belong to
+  unsigned fill_calls = 0;       // calls of that shape since the lengths were last asked for
 };
 constexpr int kFillCap = 4096;
 DeviceState g_dev[kMaxDevices];
@@ -504,8 +505,11 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
         for (int i = 0; i < n; ++i) ds->fill_host[i] = K_q;   // unknown: assume full windows until stage 1 says otherwise
         ds->fill_B = B;
         ds->fill_Kq = K_q;
+        ds->fill_calls = 0;
       }
-      fill_out = ds->fill_dev;
+      // The stores into mapped host memory cost the finalisation kernel a few microseconds: while windows are full
+      // (two launches) the lengths are asked for on every sixteenth call only, stage by stage on every call.
+      if (separate || (ds->fill_calls++ % 16u) == 0u) fill_out = ds->fill_dev;
     }
   }
   const int variant = a->kernel_variant;
@@ -544,7 +548,7 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
   PS.seq_stride_large2 = P2.seq_stride_large;
   PS.K2 = K_q;
   PS.stats2 = P2.stats;
-  rc = launch_rowstats(PS, dtype, variant, 0, stream, policy == PSD_TWO_STAGE_FUSED_ROWS);
+  rc = launch_rowstats(PS, dtype, variant, 0, stream, policy == PSD_TWO_STAGE_FUSED_ROWS || policy == PSD_TWO_STAGE_AUTO);
   if (rc != PSD_OK) return rc;
   {
     TimedLaunch timed(stream, 1);

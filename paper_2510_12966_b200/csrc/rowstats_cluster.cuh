@@ -64,6 +64,8 @@ constexpr int kClMaxRanks = 16;
 // statistics launch 0.558 -> 0.539 ms, config 3 unchanged; 72 / 136 / 56 and 64 / 136 / 64 spill in pass A.
 constexpr int kClRegsA = 80, kClRegsB = 128, kClRegsService = 56;
 static_assert(kClThreadsRS == 640 && kClAWarps == 8 && kClBWarps == 8, "the register split above is for 8 + 8 + 4 warps");
+constexpr int kClLag = 3;   // streamed twice: rows pass A's loader may be ahead of the row pass B has finished (measured: 3 costs
+                            // nothing at V = 128256 and gains 4 % at V = 152064 bf16; 2 and 1 starve pass A)
 constexpr unsigned kClSpinLimit = 1u << 22;        // polls before a wait gives up (a fraction of a second at the least)
 
 struct ClusterGeom {
@@ -823,6 +825,16 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
       unsigned slot = lo, fills = 0;   // ring position; how often the ring has wrapped
       while (!dead && w.advance()) {
         const bool tri = TRI && w.tri;
+        if (RS && !for_b) {
+          // Pass A is the lighter pass; left alone it runs rows ahead of pass B until the exchange buffers stop it,
+          // and pass B's copy of the same bytes then finds part of them gone from L2. Its loader starts row n only
+          // once pass B is through row n - kClLag.
+          unsigned spins = 0;
+          while (!dead && *reinterpret_cast<volatile int*>(&ctl->rows_closed) < w.n - kClLag + 1) {
+            __nanosleep(200);
+            if (++spins > kClSpinLimit) give_up();
+          }
+        }
         const T* const src[3] = {model_row(w, 0), model_row(w, 1), tri ? model_row(w, 2) : nullptr};
         const int steps = steps_of(tri);
         for (int step = 0; step < steps; ++step) {
