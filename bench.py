@@ -334,7 +334,7 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, rounds)
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
-        traffic = read_profile_traffic(w) if args.two_stage in ("fused", "auto") and launches_per_step == 2 else None
+        traffic = read_profile_traffic(w, "pairs" if args.two_stage == "fused" else "rows") if launches_per_step == 2 else None
         if traffic is not None:
             line["roofline"]["traffic"] = traffic
         print(json.dumps(line))
@@ -513,14 +513,14 @@ def run_fused(args):
     print(json.dumps(line))
 
 
-def read_profile_traffic(w):
-    """DRAM bytes per full-size rowstats launch from the committed ncu summary, if present."""
+def read_profile_traffic(w, form):
+    """DRAM bytes per full-size rowstats launch (row-pair or row-triple form) from the committed ncu summary, if present."""
     path = os.path.join(ROOT, "profiles", "rowstats_traffic.json")
     if not os.path.exists(path):
         return None
     with open(path) as f:
         t = json.load(f)
-    per_row = t.get("dram_bytes_per_row", {}).get(f"V{w.V}_{w.dtype}")
+    per_row = t.get("dram_bytes_per_row", {}).get(f"V{w.V}_{w.dtype}_{form}")
     return None if per_row is None else per_row * w.B * (w.K_d + w.K_q)   # rows of the fused statistics launch
 
 
