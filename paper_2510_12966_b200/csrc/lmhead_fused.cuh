@@ -240,14 +240,25 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ================================ TMA producer ================================
     if (lane == 0) {
       unsigned stage = 0, fills = 0;
-      for (int tile = blockIdx.x; tile < P.n_tiles; tile += gridDim.x) {
+      for (int tile = blockIdx.x; tile < P.n_tiles && !dead; tile += gridDim.x) {
         for (int ks = 0; ks < k_steps; ++ks) {
           if (fills > 0) wait_phase(&bars->empty[stage], (fills - 1u) & 1u);
+          if (dead) break;   // the stage never came back: nothing more is copied into this ring
           unsigned char* sa = tiles + static_cast<size_t>(stage) * kLmStageBytes;
           mbar_arrive_expect_tx(&bars->full[stage], kLmStageBytes);
           tma_load_2d(sa, &map_a, ks * kLmK, P.row0, &bars->full[stage]);                 // 256 hidden rows of the block
           tma_load_2d(sa + kLmABytes, &map_b, ks * kLmK, tile * kLmN, &bars->full[stage]);  // W^T rows tile*128..
           if (++stage == kLmStages) { stage = 0; ++fills; }
+        }
+      }
+      // When a wait gave up somewhere in the CTA the consumers no longer wait for the copies issued above: this
+      // thread sees each of them land (bounded) before the shared memory goes away.
+      if (dead || *reinterpret_cast<volatile int*>(P.status) != 0) {
+        for (unsigned s = 0; s < static_cast<unsigned>(kLmStages); ++s) {
+          const unsigned turns = fills + (s < stage ? 1u : 0u);
+          if (turns == 0) continue;
+          unsigned spins = 0;
+          while (!mbar_try(&bars->full[s], (turns - 1u) & 1u) && ++spins <= kLmSpinLimit) {}
         }
       }
     }
@@ -260,10 +271,12 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       for (int tile = blockIdx.x; tile < P.n_tiles; tile += gridDim.x, ++it) {
         const int buf = it & 1;
         if (it >= 2) wait_phase(&bars->tmem_empty[buf], ((it >> 1) - 1) & 1u);   // the epilogue has drained this buffer
+        if (dead) break;
         tc_fence_after();
         const unsigned acc0 = tmem_base + static_cast<unsigned>(buf) * 256u, acc1 = acc0 + 128u;
         for (int ks = 0; ks < k_steps; ++ks) {
           wait_phase(&bars->full[stage], par);
+          if (dead) break;   // no MMA on operands that have not arrived
           tc_fence_after();
           const unsigned sa = smem_u32(tiles + static_cast<size_t>(stage) * kLmStageBytes);
           const unsigned long long da0 = umma_desc_k128(sa), da1 = umma_desc_k128(sa + 128 * 128), db = umma_desc_k128(sa + kLmABytes);
@@ -277,6 +290,7 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           tc_commit(&bars->empty[stage]);   // arrives when the MMAs that read this stage have completed
           if (++stage == kLmStages) { stage = 0; par ^= 1u; }
         }
+        if (dead) break;
         tc_commit(&bars->tmem_full[buf]);   // the accumulators of this tile are complete
       }
     }
@@ -399,15 +413,26 @@ lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     // ================================ TMA producer (both CTAs) ================================
     if (lane == 0) {
       unsigned stage = 0, fills = 0;
-      for (int tile = pair; tile < n_tiles2; tile += n_pairs) {
+      for (int tile = pair; tile < n_tiles2 && !dead; tile += n_pairs) {
         for (int ks = 0; ks < k_steps; ++ks) {
           if (fills > 0) wait_phase(&bars->empty[stage], (fills - 1u) & 1u);
+          if (dead) break;   // the stage never came back: nothing more is copied into this ring
           unsigned char* sa = tiles + static_cast<size_t>(stage) * kLm2StageBytes;
           // the even CTA's barrier counts the bytes of both CTAs
           if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2u * kLm2StageBytes);
           tma_load_2d_pair(sa, &map_a, ks * kLmK, P.row0 + static_cast<int>(rank) * 128, &bars->full[stage]);
           tma_load_2d_pair(sa + kLm2HalfBytes, &map_b, ks * kLmK, tile * kLm2N + static_cast<int>(rank) * 128, &bars->full[stage]);
           if (++stage == kLm2Stages) { stage = 0; ++fills; }
+        }
+      }
+      // After a wait gave up, the even CTA (whose barriers count both CTAs' bytes) sees every copy issued so far
+      // land, bounded, before it enters the final cluster barrier that keeps both CTAs' shared memory alive.
+      if (rank == 0 && (dead || *reinterpret_cast<volatile int*>(P.status) != 0)) {
+        for (unsigned s = 0; s < static_cast<unsigned>(kLm2Stages); ++s) {
+          const unsigned turns = fills + (s < stage ? 1u : 0u);
+          if (turns == 0) continue;
+          unsigned spins = 0;
+          while (!mbar_try(&bars->full[s], (turns - 1u) & 1u) && ++spins <= kLmSpinLimit) {}
         }
       }
     }
@@ -420,10 +445,12 @@ lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       for (int tile = pair; tile < n_tiles2; tile += n_pairs, ++it) {
         const int buf = it & 1;
         if (it >= 2) wait_phase(&bars->tmem_empty[buf], ((it >> 1) - 1) & 1u);   // both CTAs' epilogues have drained this buffer
+        if (dead) break;
         tc_fence_after();
         const unsigned acc = tmem_base + static_cast<unsigned>(buf) * 256u;
         for (int ks = 0; ks < k_steps; ++ks) {
           wait_phase(&bars->full[stage], par);
+          if (dead) break;   // no MMA on operands that have not arrived
           tc_fence_after();
           const unsigned sa = smem_u32(tiles + static_cast<size_t>(stage) * kLm2StageBytes);
           const unsigned long long da = umma_desc_k128(sa), db = umma_desc_k128(sa + kLm2HalfBytes);
@@ -433,6 +460,7 @@ lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
           tc_commit_pair(&bars->empty[stage]);   // frees the stage in both CTAs once these MMAs have read it
           if (++stage == kLm2Stages) { stage = 0; par ^= 1u; }
         }
+        if (dead) break;
         tc_commit_pair(&bars->tmem_full[buf]);   // the accumulators of this tile are complete, in both CTAs
       }
     }
