@@ -430,8 +430,16 @@ def run_fused(args):
     hs = [h, h.clone()]          # the weight (1.05 GB) stays resident like a model's; activations alternate
     zs = [z_q, z_q.clone()]
 
+    kl = args.lmhead_div == "kl"
+    div_kind = binding.DIV_KL if kl else binding.DIV_JS
+    lm_mode = binding.ASSISTED if args.lmhead_mode == "assisted" else binding.FUZZY
+    if args.lmhead_tau is not None:
+        import dataclasses
+        w = dataclasses.replace(w, tau_t=args.lmhead_tau)
+
     def step(i):
-        return binding.verify_fused_lmhead(hs[i % 2], w_t, zs[i % 2], tok, w.tau_t, binding.FUZZY, 0, i, want_rows=False)
+        return binding.verify_fused_lmhead(hs[i % 2], w_t, zs[i % 2], tok, w.tau_t, lm_mode, 0, i, want_rows=False,
+                                           div_kind=div_kind)
 
     for i in range(args.warmup):
         step(i)
@@ -460,7 +468,11 @@ def run_fused(args):
     if binding.last_status() != 0:
         raise SystemExit("bench.py: library status != 0")
     peaks, peak_kind = load_peaks()
-    flops = 2 * 2.0 * M * w.d_model * w.V
+    # Jensen-Shannon runs the GEMM twice; KL once, plus a second sweep only when a rejected row needs residual masses:
+    # never in the assisted mode, and not in the threshold mode while every position is accepted
+    one_sweep = kl and (lm_mode == binding.ASSISTED or bool((out["accept_len"] == w.K_d).all().item()))
+    sweeps = 1 if one_sweep else 2
+    flops = sweeps * 2.0 * M * w.d_model * w.V
     achieved = flops * n_sw / (ms_sweeps * 1e-3) / 1e12 if ms_sweeps > 0 else 0.0
     # end to end: activations and qualifier logits come from pinned host memory every step, results go back
     e2e = None
@@ -474,7 +486,7 @@ def run_fused(args):
                 torch.cuda.synchronize()
                 e0.record()
             hs[0].copy_(hh, non_blocking=True); zs[0].copy_(zh, non_blocking=True); tok.copy_(th, non_blocking=True)
-            o = binding.verify_fused_lmhead(hs[0], w_t, zs[0], tok, w.tau_t, binding.FUZZY, 0, it, want_rows=False)
+            o = binding.verify_fused_lmhead(hs[0], w_t, zs[0], tok, w.tau_t, lm_mode, 0, it, want_rows=False, div_kind=div_kind)
             res[0].copy_(o["accept_len"], non_blocking=True); res[1].copy_(o["next_token"], non_blocking=True)
             torch.cuda.synchronize()
         e1.record()
@@ -493,16 +505,17 @@ def run_fused(args):
         "vs_baseline": None, "dtype": "bf16 x bf16 -> f32 (GEMM), f32 (epilogue)", "data": "synthetic",
         "timed_regions": args.regions, "ms_per_step_min_max": [min(region_ms) / args.steps, max(region_ms) / args.steps],
         "config": {"workload": f"{w.name}: B={w.B}, K={w.K_d} (M={M}), d={w.d_model}, V={w.V}, LM-head weight bf16 [V, d], "
-                               f"qualifier logits bf16, tau_t={w.tau_t}, fuzzy mode, Philox seed 0",
+                               f"qualifier logits bf16, tau_t={w.tau_t}, {args.lmhead_mode} mode, Philox seed 0, divergence {'KL(large||small)' if kl else 'Jensen-Shannon'}, {sweeps} GEMM sweep(s)",
+                   "all_positions_accepted": bool((out["accept_len"] == w.K_d).all().item()),
                    "l2_policy": "the weight (1.05 GB) is larger than L2 and is streamed twice per step"},
         "roofline": {"bound": "tensor", "kernel": "lmhead_sweep (two tcgen05 GEMM sweeps + row reduction)",
                      "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s", "frac": achieved / tensor_peak,
                      "frac_of_burst": achieved / peaks["bf16_tflops"],
-                     "flops_counted": "both GEMM sweeps (what the tensor pipe executes); the method needs one h x W^T",
-                     "achieved_on_one_gemm": achieved / 2, "frac_on_one_gemm": achieved / 2 / tensor_peak,
+                     "flops_counted": "the GEMM sweeps executed (%d); the method needs one h x W^T" % sweeps,
+                     "achieved_on_one_gemm": achieved / sweeps, "frac_on_one_gemm": achieved / sweeps / tensor_peak,
                      "peak_kind": tensor_kind, "traffic": None, "launches": n_sw,
                      "avg_launch_ms": ms_sweeps / max(n_sw, 1), "finalize_ms_per_launch": ms_fin / max(n_fin, 1),
-                     "weight_gb_per_s": 2 * w.V * w.d_model * 2 * n_sw / (ms_sweeps * 1e-3) / 1e9 if ms_sweeps > 0 else 0.0},
+                     "weight_gb_per_s": sweeps * w.V * w.d_model * 2 * n_sw / (ms_sweeps * 1e-3) / 1e9 if ms_sweeps > 0 else 0.0},
         "gpu_launches": launches, "clocks": clocks,
     }
     if e2e:
@@ -621,6 +634,9 @@ def main():
     ap.add_argument("--two-stage", choices=["fused", "separate", "auto", "rows"], default="auto",
                     help="schedule of the two stages (same results): one statistics launch for both (row pairs, or row "
                          "triples with `rows`), stage by stage, or the library's per-call choice (its default)")
+    ap.add_argument("--lmhead-div", choices=["js", "kl"], default="js", help="divergence of the fused LM-head workload (cfg5)")
+    ap.add_argument("--lmhead-mode", choices=["fuzzy", "assisted"], default="fuzzy", help="acceptance mode of cfg5")
+    ap.add_argument("--lmhead-tau", type=float, default=None, help="threshold of cfg5 (default: the workload's)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -278,7 +278,12 @@ int pyramidsd_verify_fused_lmhead(const void* hidden, const void* w_t, const voi
 /* The same call with every option exposed. Zero-initialise, set struct_size, fill what you need.
  *   seq_index_base  as in psd_stage_args.
  *   tile_variant    PSD_LMHEAD_TILES_AUTO (pairs of CTAs on 256 x 256 tiles, tcgen05 cta_group::2) or
- *                   PSD_LMHEAD_TILES_ONE_SM (one CTA per 256 x 128 tile); same results within rounding. */
+ *                   PSD_LMHEAD_TILES_ONE_SM (one CTA per 256 x 128 tile); same results within rounding.
+ *   div_kind        PSD_DIV_KL: KL(large || small), whose terms separate -- sum_i p_i (log p_i - log q_i) needs the
+ *                   normalisers only at the end -- so the divergences are known after ONE sweep of the GEMM. The second
+ *                   sweep then only serves the residual masses: it is launched, and returns at once unless some rejected
+ *                   row draws from the residual (any mode but the assisted one) or out_resid_mass is wanted. With
+ *                   PSD_ASSISTED, or when every position is accepted, the weight is streamed once per call. */
 #define PSD_LMHEAD_TILES_AUTO 0
 #define PSD_LMHEAD_TILES_ONE_SM 1
 typedef struct psd_lmhead_args {
@@ -291,6 +296,8 @@ typedef struct psd_lmhead_args {
   int32_t B, K, d_model, V;
   float threshold;
   int32_t tile_variant;
+  int32_t div_kind;              /* PSD_DIV_JS or PSD_DIV_KL (PSD_DIV_TV: PSD_ERR_UNSUPPORTED) */
+  int32_t reserved0;
   uint64_t philox_seed, philox_offset;
   int64_t seq_index_base;
   int32_t* out_accept_len;       /* [B] device, required */

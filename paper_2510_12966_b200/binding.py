@@ -82,6 +82,7 @@ class LmheadArgs(C.Structure):
         ("hidden", C.c_void_p), ("w_t", C.c_void_p), ("logits_small", C.c_void_p), ("tokens", C.c_void_p),
         ("B", C.c_int32), ("K", C.c_int32), ("d_model", C.c_int32), ("V", C.c_int32),
         ("threshold", C.c_float), ("tile_variant", C.c_int32),
+        ("div_kind", C.c_int32), ("reserved0", C.c_int32),
         ("philox_seed", C.c_uint64), ("philox_offset", C.c_uint64),
         ("seq_index_base", C.c_int64),
         ("out_accept_len", C.c_void_p), ("out_next_token", C.c_void_p),
@@ -288,7 +289,8 @@ def verify_stage(logits_small, logits_large, draft_tokens, threshold, mode=FUZZY
 
 
 def verify_fused_lmhead(hidden, w_t, logits_small, tokens, threshold, mode=FUZZY, philox_seed=0, offset=0, *,
-                        want_rows=True, stream=None, raise_on_error=True, tile_variant=None, seq_index_base=0):
+                        want_rows=True, stream=None, raise_on_error=True, tile_variant=None, seq_index_base=0,
+                        div_kind=DIV_JS, want_resid=None):
     """``pyramidsd_verify_fused_lmhead``: hidden [B*K, d] bf16, w_t [V, d] bf16 (LM-head weight, out x in),
     logits_small [B, K, V] bf16, tokens [B, K]. Returns a dict of device tensors (+ "status")."""
     B, K, V = logits_small.shape
@@ -297,17 +299,19 @@ def verify_fused_lmhead(hidden, w_t, logits_small, tokens, threshold, mode=FUZZY
     dev = hidden.device
     out = {"accept_len": torch.empty(B, dtype=torch.int32, device=dev),
            "next_token": torch.empty(B, dtype=torch.int32, device=dev)}
+    want_resid = want_rows if want_resid is None else want_resid
     if want_rows:
         out["div"] = torch.empty((B, K), dtype=torch.float32, device=dev)
+    if want_resid:
         out["resid_mass"] = torch.empty((B, K), dtype=torch.float32, device=dev)
     s = torch.cuda.current_stream() if stream is None else stream
-    if tile_variant is None and seq_index_base == 0:
+    if tile_variant is None and seq_index_base == 0 and div_kind == DIV_JS:
         rc = load_library().pyramidsd_verify_fused_lmhead(
             _dev_ptr(hidden, torch.bfloat16, "hidden"), _dev_ptr(w_t, torch.bfloat16, "w_t"),
             _dev_ptr(logits_small, torch.bfloat16, "logits_small"), _dev_ptr(tokens, torch.int32, "tokens"),
             B, K, d, V, float(threshold), int(mode), int(philox_seed), int(offset),
             out["accept_len"].data_ptr(), out["next_token"].data_ptr(),
-            out["div"].data_ptr() if want_rows else None, out["resid_mass"].data_ptr() if want_rows else None,
+            out["div"].data_ptr() if want_rows else None, out["resid_mass"].data_ptr() if want_resid else None,
             C.c_void_p(s.cuda_stream))
     else:
         a = LmheadArgs()
@@ -317,11 +321,13 @@ def verify_fused_lmhead(hidden, w_t, logits_small, tokens, threshold, mode=FUZZY
         a.logits_small = _dev_ptr(logits_small, torch.bfloat16, "logits_small")
         a.tokens = _dev_ptr(tokens, torch.int32, "tokens")
         a.B, a.K, a.d_model, a.V = B, K, d, V
-        a.threshold, a.tile_variant = float(threshold), int(tile_variant or 0)
+        a.threshold, a.tile_variant, a.div_kind = float(threshold), int(tile_variant or 0), int(div_kind)
         a.philox_seed, a.philox_offset, a.seq_index_base = int(philox_seed), int(offset), int(seq_index_base)
         a.out_accept_len, a.out_next_token = out["accept_len"].data_ptr(), out["next_token"].data_ptr()
         if want_rows:
-            a.out_div, a.out_resid_mass = out["div"].data_ptr(), out["resid_mass"].data_ptr()
+            a.out_div = out["div"].data_ptr()
+        if want_resid:
+            a.out_resid_mass = out["resid_mass"].data_ptr()
         a.stream = s.cuda_stream
         rc = load_library().pyramidsd_verify_fused_lmhead_ex(C.byref(a))
     out["status"] = rc

@@ -50,6 +50,12 @@ struct LmParams {
   float4* row_lse;                // [M] (m2_small, l2s_small, m2_large, l2s_large)
   float4* part_div;               // sweep 2: [M][n_tiles] (js bits, sum max(p,q), residual mass, mass of p)
   int* status;
+  // KL(large || small) needs no second sweep for the divergence itself: sum_i p_i (log2 p_i - log2 q_i) =
+  // (1 / S_l) sum_i P_i (z_i - x_i) c - (lse_l - lse_s) with P_i = 2^(z_i c - m), which sweep 1 accumulates per
+  // tile next to (m, S_l), rescaled online like the sum.
+  float* part_t;                  // KL, sweep 1: [M][n_tiles] sum of P_i (z_i - x_i) c against the tile's own max
+  float* row_div;                 // KL: [M] the row's divergence in nats, written by the row reduction
+  int* need_sweep2;               // KL: set by the accept scan when a residual mass is needed after all; sweep 2 leaves at once if 0
 };
 
 // ---- tcgen05 / TMA wrappers -----------------------------------------------------------------------------
@@ -150,18 +156,19 @@ __device__ __forceinline__ void load_small32(const __nv_bfloat16* p, bool aligne
 // What one thread (= one row) leaves per 128-column tile.
 struct LmTilePartial {
   float2 large, small;   // sweep 1: (max, sum) of both models
+  float kl_t;            // sweep 1, KL: sum of P_i (z_i - x_i) c against `large.x`
   float4 div;            // sweep 2: (js bits, sum max(p,q), residual mass, mass of p)
 };
 
 // The epilogue of one 128-column tile for this thread's row: reads the accumulator from tensor memory 32
 // columns at a time (all 32 lanes execute the loads, whatever row_ok says) and the small model's logits
 // from global memory.
-template <int SWEEP>
+template <int SWEEP, bool KL = false>
 __device__ __forceinline__ void lm_epilogue_tile(unsigned tacc, int n0, bool row_ok, const __nv_bfloat16* small_row, float c,
                                                  float off_l, float off_s, int V, LmTilePartial& out) {
   OnlineLse ol, os;
   ol.init(); os.init();
-  float js = 0.f, big = 0.f, resid = 0.f, pmass = 0.f;
+  float js = 0.f, big = 0.f, resid = 0.f, pmass = 0.f, kl_t = 0.f;
 #pragma unroll 1
   for (int cb = 0; cb < kLmN / 32; ++cb) {
     float z[32], x[32];
@@ -172,8 +179,21 @@ __device__ __forceinline__ void lm_epilogue_tile(unsigned tacc, int n0, bool row
       const __nv_bfloat16* sp = small_row + col0;
       load_small32(sp, (reinterpret_cast<uintptr_t>(sp) & 15u) == 0, nv, x);
       if (SWEEP == 1) {
+        const float m_before = ol.m;
         ol.add<32>(z, c, nv);
         os.add<32>(x, c, nv);
+        if (KL) {
+          kl_t *= ex2_approx(m_before - ol.m);   // the group may have raised the tile's max
+          float t = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (i < nv) {
+              const float e = ex2_approx(fmaf(z[i], c, -ol.m));
+              if (e > 0.f) t = fmaf(e, (z[i] - x[i]) * c, t);   // q_i = 0 under p_i > 0 gives +inf, as it should
+            }
+          }
+          kl_t += t;
+        }
       } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -195,23 +215,28 @@ __device__ __forceinline__ void lm_epilogue_tile(unsigned tacc, int n0, bool row
   }
   out.large = make_float2(ol.m, ol.s);
   out.small = make_float2(os.m, os.s);
+  out.kl_t = kl_t;
   out.div = make_float4(js, big, resid, pmass);
 }
 
-template <int SWEEP>
+template <int SWEEP, bool KL = false>
 __device__ __forceinline__ void lm_store_partial(const LmParams& P, size_t idx, const LmTilePartial& part) {
   if (SWEEP == 1) {
     P.part_large[idx] = part.large;
     P.part_small[idx] = part.small;
+    if (KL) P.part_t[idx] = part.kl_t;
   } else {
     P.part_div[idx] = part.div;
   }
 }
 
-template <int SWEEP>
+template <int SWEEP, bool KL = false>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const LmParams P) {
   extern __shared__ unsigned char lm_smem_raw[];
+  // KL: the second sweep only serves residual masses; when the accept scan found no use for them every CTA leaves
+  // here, before it has set up anything (the flag was written by an earlier kernel: the same answer for all)
+  if (SWEEP == 2 && P.need_sweep2 != nullptr && *reinterpret_cast<volatile const int*>(P.need_sweep2) == 0) return;
   unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(lm_smem_raw) + 1023) & ~uintptr_t(1023));
   LmBarriers* bars = reinterpret_cast<LmBarriers*>(tiles + static_cast<size_t>(kLmStages) * kLmStageBytes);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -314,11 +339,11 @@ lmhead_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                             (static_cast<unsigned>(quarter * 32) << 16);
       const int n0 = tile * kLmN;
       LmTilePartial part;
-      lm_epilogue_tile<SWEEP>(tacc, n0, row_ok, small_row, c, off_l, off_s, P.V, part);
+      lm_epilogue_tile<SWEEP, KL>(tacc, n0, row_ok, small_row, c, off_l, off_s, P.V, part);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->tmem_empty[buf]);   // this warp has read its part of the accumulator
-      if (row_ok) lm_store_partial<SWEEP>(P, static_cast<size_t>(row) * P.n_tiles + tile, part);
+      if (row_ok) lm_store_partial<SWEEP, KL>(P, static_cast<size_t>(row) * P.n_tiles + tile, part);
     }
   }
   tc_fence_before();
@@ -377,10 +402,11 @@ __device__ __forceinline__ void mbar_arrive_remote_release(unsigned cluster_addr
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
-template <int SWEEP>
+template <int SWEEP, bool KL = false>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const LmParams P) {
   extern __shared__ unsigned char lm_smem_raw[];
+  if (SWEEP == 2 && P.need_sweep2 != nullptr && *reinterpret_cast<volatile const int*>(P.need_sweep2) == 0) return;   // as in the one-SM kernel
   unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(lm_smem_raw) + 1023) & ~uintptr_t(1023));
   Lm2Barriers* bars = reinterpret_cast<Lm2Barriers*>(tiles + static_cast<size_t>(kLm2Stages) * kLm2StageBytes);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -484,11 +510,11 @@ lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                             (static_cast<unsigned>(quarter * 32) << 16);
       const int tile128 = tile * 2 + half;
       LmTilePartial part;
-      lm_epilogue_tile<SWEEP>(tacc, tile128 * kLmN, row_ok, small_row, c, off_l, off_s, P.V, part);
+      lm_epilogue_tile<SWEEP, KL>(tacc, tile128 * kLmN, row_ok, small_row, c, off_l, off_s, P.V, part);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote_release(drained + static_cast<unsigned>(buf) * 8u);
-      if (row_ok && tile128 < P.n_tiles) lm_store_partial<SWEEP>(P, static_cast<size_t>(row) * P.n_tiles + tile128, part);
+      if (row_ok && tile128 < P.n_tiles) lm_store_partial<SWEEP, KL>(P, static_cast<size_t>(row) * P.n_tiles + tile128, part);
     }
   }
   tc_fence_before();
@@ -500,10 +526,13 @@ lmhead_sweep2sm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   }
 }
 
-// Per row: combine the tiles' (max, sum) partials into the row's log-sum-exp (base 2), both models.
+// Per row: combine the tiles' (max, sum) partials into the row's log-sum-exp (base 2), both models; with the KL
+// partials also the row's divergence KL(large || small) = ln 2 * (T / S_l - (lse_l - lse_s)), T rescaled to the
+// row's max like S_l.
 __global__ void __launch_bounds__(256) lmhead_reduce_kernel(const LmParams P) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (row >= P.M) return;
+  const bool kl = P.part_t != nullptr;
   float ml = -1e30f, sl = 0.f, ms = -1e30f, ss = 0.f;
   for (int t = lane; t < P.n_tiles; t += 32) {
     const float2 a = P.part_large[static_cast<size_t>(row) * P.n_tiles + t], b = P.part_small[static_cast<size_t>(row) * P.n_tiles + t];
@@ -515,7 +544,18 @@ __global__ void __launch_bounds__(256) lmhead_reduce_kernel(const LmParams P) {
     lse_merge(ml, sl, __shfl_xor_sync(0xffffffffu, ml, o), __shfl_xor_sync(0xffffffffu, sl, o));
     lse_merge(ms, ss, __shfl_xor_sync(0xffffffffu, ms, o), __shfl_xor_sync(0xffffffffu, ss, o));
   }
-  if (lane == 0) P.row_lse[row] = make_float4(ms, lg2_approx(ss), ml, lg2_approx(sl));
+  const float l2sl = lg2_approx(sl), l2ss = lg2_approx(ss);
+  if (lane == 0) P.row_lse[row] = make_float4(ms, l2ss, ml, l2sl);
+  if (kl) {
+    float tt = 0.f;   // sum over the tiles of T_t * 2^(m_t - ml): ml is the row's max after the merge above
+    for (int t = lane; t < P.n_tiles; t += 32) {
+      const float tv = P.part_t[static_cast<size_t>(row) * P.n_tiles + t];
+      const float f = ex2_approx(P.part_large[static_cast<size_t>(row) * P.n_tiles + t].x - ml);
+      if (f > 0.f) tt = fmaf(tv, f, tt);   // a tile without mass contributes nothing (0 * inf otherwise)
+    }
+    tt = warp_reduce<OpSum>(tt);
+    if (lane == 0) P.row_div[row] = fmaxf(kLn2 * (__fdiv_rn(tt, sl) - ((ml + l2sl) - (ms + l2ss))), 0.f);
+  }
 }
 
 // ---- final kernel: one CTA per sequence ------------------------------------------------------------------
@@ -532,6 +572,10 @@ struct LmFinalParams {
   int32_t* out_next_token;
   float* out_div;        // [B, K] or null
   float* out_resid;      // [B, K] or null
+  // KL: 0 = the usual pass over the second sweep's partials. 1 = accept scan only, before the second sweep: raises
+  // lm.need_sweep2 when some rejected row needs residual masses. 2 = full pass after a second sweep that may not
+  // have run (then every draw comes from p_large, whose tile masses the first sweep left).
+  int kl_phase;
 };
 
 // dot(hidden[row], w_t[col]) by one warp, fp32 accumulation in index order per lane then a shuffle tree
@@ -551,6 +595,7 @@ __global__ void __launch_bounds__(256) lmhead_final_kernel(const LmFinalParams F
   __shared__ float sh_div[32], sh_res[32], sh_px[32], sh_qx[32], sh_pm[32];
   __shared__ int sh_flag[32];
   __shared__ float sh_w[kLmN];
+  __shared__ double sh_seg[256];
   __shared__ int sh_L, sh_tile, sh_token;
   __shared__ float sh_target, sh_u2;
   const LmParams& P = F.lm;
@@ -561,9 +606,13 @@ __global__ void __launch_bounds__(256) lmhead_final_kernel(const LmFinalParams F
   for (int k = warp; k < K; k += nwarps) {
     const int r = b * K + k;
     double js = 0.0, big = 0.0, res = 0.0, pm = 0.0;
-    for (int t = lane; t < P.n_tiles; t += 32) {
-      const float4 v = P.part_div[static_cast<size_t>(r) * P.n_tiles + t];
-      js += v.x; big += v.y; res += v.z; pm += v.w;
+    // KL: the divergence comes from the row reduction; the second sweep's partials exist only if it ran
+    const bool have2 = F.kl_phase == 0 || (F.kl_phase == 2 && *reinterpret_cast<volatile const int*>(P.need_sweep2) != 0);
+    if (have2) {
+      for (int t = lane; t < P.n_tiles; t += 32) {
+        const float4 v = P.part_div[static_cast<size_t>(r) * P.n_tiles + t];
+        js += v.x; big += v.y; res += v.z; pm += v.w;
+      }
     }
     js = warp_reduce<OpSum>(js); res = warp_reduce<OpSum>(res); pm = warp_reduce<OpSum>(pm);
     const float4 lse = P.row_lse[r];
@@ -580,13 +629,15 @@ __global__ void __launch_bounds__(256) lmhead_final_kernel(const LmFinalParams F
       qx = ex2_approx(fmaf(Elem<__nv_bfloat16>::load(P.small + static_cast<size_t>(r) * P.V, x), c, -lse.x) - lse.y);
     }
     if (lane == 0) {
-      sh_div[k] = fmaxf(static_cast<float>(0.5 * 0.6931471805599453 * js), 0.f);
-      sh_res[k] = fmaxf(static_cast<float>(res), 0.f);
+      sh_div[k] = F.kl_phase != 0 ? P.row_div[r] : fmaxf(static_cast<float>(0.5 * 0.6931471805599453 * js), 0.f);
+      sh_res[k] = have2 ? fmaxf(static_cast<float>(res), 0.f) : __int_as_float(0x7fc00000);
       sh_pm[k] = static_cast<float>(pm);
       sh_px[k] = px; sh_qx[k] = qx; sh_flag[k] = flags;
       const bool no_dist = (flags & (kFlagSmallNonfinite | kFlagLargeNonfinite)) != 0;   // a bad token leaves D and R intact
-      if (F.out_div) F.out_div[r] = no_dist ? __int_as_float(0x7fc00000) : sh_div[k];
-      if (F.out_resid) F.out_resid[r] = no_dist ? __int_as_float(0x7fc00000) : sh_res[k];
+      if (F.kl_phase != 1) {
+        if (F.out_div) F.out_div[r] = no_dist ? __int_as_float(0x7fc00000) : sh_div[k];
+        if (F.out_resid) F.out_resid[r] = no_dist ? __int_as_float(0x7fc00000) : sh_res[k];
+      }
     }
   }
   __syncthreads();
@@ -614,31 +665,66 @@ __global__ void __launch_bounds__(256) lmhead_final_kernel(const LmFinalParams F
   __syncthreads();
   const int L = sh_L;
   u2 = sh_u2;
+  if (F.kl_phase == 1) {
+    // scan only: a rejected row with a distribution draws from the residual unless the mode is the assisted one
+    if (tid == 0 && L < K && !(sh_flag[L] & (kFlagSmallNonfinite | kFlagLargeNonfinite)) && F.mode != kModeAssisted)
+      atomicExch(P.need_sweep2, 1);
+    return;
+  }
+  const bool have2 = F.kl_phase == 0 || *reinterpret_cast<volatile const int*>(P.need_sweep2) != 0;
   int next = -1;
   if (L < K) {
     if (sh_flag[L] & (kFlagSmallNonfinite | kFlagLargeNonfinite)) {
       next = -2;
     } else {
       const int r = b * K + L;
-      const bool from_large = (F.mode == kModeAssisted) || !(sh_res[L] > 0.f);
-      // the tile that holds the target mass: first tile whose inclusive cumulative weight exceeds it
+      const bool from_large = (F.mode == kModeAssisted) || !have2 || !(sh_res[L] > 0.f);
+      const float4 lse_r = P.row_lse[r];
+      // weight of tile t: the second sweep's residual mass or mass of p; without a second sweep the mass of p from
+      // the first sweep's (max, sum) of the tile
+      auto tile_weight = [&](int t) -> double {
+        if (have2) {
+          const float4 v = P.part_div[static_cast<size_t>(r) * P.n_tiles + t];
+          return from_large ? v.w : v.z;
+        }
+        const float2 a = P.part_large[static_cast<size_t>(r) * P.n_tiles + t];
+        return static_cast<double>(a.y) * static_cast<double>(ex2_approx((a.x - lse_r.z) - lse_r.w));
+      };
+      // the tile that holds the target mass: first tile whose inclusive cumulative weight exceeds it. Two levels:
+      // every thread sums a run of consecutive tiles, one thread walks the 256 run sums and then the chosen run.
+      const int per = (P.n_tiles + static_cast<int>(blockDim.x) - 1) / static_cast<int>(blockDim.x);
+      {
+        double run = 0.0;
+        const int t0 = tid * per, t1 = min(P.n_tiles, t0 + per);
+        for (int t = t0; t < t1; ++t) run += tile_weight(t);
+        sh_seg[tid] = run;
+      }
+      __syncthreads();
       if (tid == 0) {
         double total = 0.0;
-        for (int t = 0; t < P.n_tiles; ++t) {
-          const float4 v = P.part_div[static_cast<size_t>(r) * P.n_tiles + t];
-          total += from_large ? v.w : v.z;
-        }
+        for (int g = 0; g < static_cast<int>(blockDim.x); ++g) total += sh_seg[g];
         const double target = static_cast<double>(u2) * total;
-        int pick = -1, last_pos = -1;
-        double cum = 0.0, before_pick = 0.0, before_last = 0.0;
-        for (int t = 0; t < P.n_tiles; ++t) {
-          const float4 v = P.part_div[static_cast<size_t>(r) * P.n_tiles + t];
-          const double wgt = from_large ? v.w : v.z;
-          if (wgt > 0.0) { last_pos = t; before_last = cum; }
-          if (pick < 0 && cum + wgt > target && wgt > 0.0) { pick = t; before_pick = cum; }
+        int seg = -1, last_seg = -1;
+        double cum = 0.0, before_seg = 0.0, before_last_seg = 0.0;
+        for (int g = 0; g < static_cast<int>(blockDim.x); ++g) {
+          const double wgt = sh_seg[g];
+          if (wgt > 0.0) { last_seg = g; before_last_seg = cum; }
+          if (seg < 0 && cum + wgt > target && wgt > 0.0) { seg = g; before_seg = cum; }
           cum += wgt;
         }
-        if (pick < 0) { pick = last_pos; before_pick = before_last; }
+        if (seg < 0) { seg = last_seg; before_seg = before_last_seg; }
+        int pick = -1, last_pos = -1;
+        double before_pick = 0.0, before_last = 0.0;
+        if (seg >= 0) {
+          cum = before_seg;
+          for (int t = seg * per; t < min(P.n_tiles, (seg + 1) * per); ++t) {
+            const double wgt = tile_weight(t);
+            if (wgt > 0.0) { last_pos = t; before_last = cum; }
+            if (pick < 0 && cum + wgt > target && wgt > 0.0) { pick = t; before_pick = cum; }
+            cum += wgt;
+          }
+          if (pick < 0) { pick = last_pos; before_pick = before_last; }
+        }
         sh_tile = pick;
         sh_target = static_cast<float>(target - before_pick);
         sh_token = -1;

@@ -779,6 +779,9 @@ int pyramidsd_verify_stage_noalloc(const void* logits_small, const void* logits_
 int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args) {
   if (args == nullptr || args->struct_size != sizeof(psd_lmhead_args)) return PSD_ERR_INVALID_ARG;
   if (args->tile_variant < PSD_LMHEAD_TILES_AUTO || args->tile_variant > PSD_LMHEAD_TILES_ONE_SM || args->seq_index_base < 0) return PSD_ERR_INVALID_ARG;
+  if (!valid_div(args->div_kind) || args->reserved0 != 0) return PSD_ERR_INVALID_ARG;
+  if (args->div_kind == PSD_DIV_TV) return PSD_ERR_UNSUPPORTED;
+  const bool kl = args->div_kind == PSD_DIV_KL;
   const void* hidden = args->hidden;
   const void* w_t = args->w_t;
   const void* logits_small = args->logits_small;
@@ -811,7 +814,8 @@ int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args) {
   std::lock_guard<std::mutex> lock(ss->mu);
   const int n_tiles = (V + psd::kLmN - 1) / psd::kLmN;
   const size_t per = static_cast<size_t>(M) * n_tiles;
-  const size_t bytes = align_up(per * sizeof(float2)) * 2 + align_up(per * sizeof(float4)) + align_up(static_cast<size_t>(M) * sizeof(float4));
+  const size_t bytes = align_up(per * sizeof(float2)) * 2 + align_up(per * sizeof(float4)) + align_up(static_cast<size_t>(M) * sizeof(float4)) +
+                       align_up(per * sizeof(float)) + align_up(static_cast<size_t>(M) * sizeof(float)) + kAlign;
   rc = ensure_status(ss);
   if (rc != PSD_OK) return rc;
   t_last_scratch = ss; t_last_status = ss->status; t_last_stream = stream;
@@ -850,14 +854,27 @@ int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args) {
   L.part_large = reinterpret_cast<float2*>(ws); ws += align_up(per * sizeof(float2));
   L.part_small = reinterpret_cast<float2*>(ws); ws += align_up(per * sizeof(float2));
   L.part_div = reinterpret_cast<float4*>(ws); ws += align_up(per * sizeof(float4));
-  L.row_lse = reinterpret_cast<float4*>(ws);
+  L.row_lse = reinterpret_cast<float4*>(ws); ws += align_up(static_cast<size_t>(M) * sizeof(float4));
   L.status = ss->status;
+  if (kl) {
+    L.part_t = reinterpret_cast<float*>(ws); ws += align_up(per * sizeof(float));
+    L.row_div = reinterpret_cast<float*>(ws); ws += align_up(static_cast<size_t>(M) * sizeof(float));
+    L.need_sweep2 = reinterpret_cast<int*>(ws);
+    // the residual masses are wanted as an output: the second sweep runs whatever the accept scan finds
+    if (cudaMemsetAsync(L.need_sweep2, out_resid_mass != nullptr ? 1 : 0, sizeof(int), stream) != cudaSuccess) return PSD_ERR_CUDA;
+  }
   static bool attr_set[kMaxDevices] = {};
   int dev = 0;
   cudaGetDevice(&dev);
   if (!attr_set[dev]) {
-    if (cudaFuncSetAttribute(psd::lmhead_sweep_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLmSmemBytes)) != cudaSuccess ||
-        cudaFuncSetAttribute(psd::lmhead_sweep_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLmSmemBytes)) != cudaSuccess) {
+    const int one = static_cast<int>(psd::kLmSmemBytes), two = static_cast<int>(psd::kLm2SmemBytes);
+    const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    if (cudaFuncSetAttribute(psd::lmhead_sweep_kernel<1, false>, at, one) != cudaSuccess ||
+        cudaFuncSetAttribute(psd::lmhead_sweep_kernel<1, true>, at, one) != cudaSuccess ||
+        cudaFuncSetAttribute(psd::lmhead_sweep_kernel<2, false>, at, one) != cudaSuccess ||
+        cudaFuncSetAttribute(psd::lmhead_sweep2sm_kernel<1, false>, at, two) != cudaSuccess ||
+        cudaFuncSetAttribute(psd::lmhead_sweep2sm_kernel<1, true>, at, two) != cudaSuccess ||
+        cudaFuncSetAttribute(psd::lmhead_sweep2sm_kernel<2, false>, at, two) != cudaSuccess) {
       cudaGetLastError();
       return PSD_ERR_CUDA;
     }
@@ -867,70 +884,57 @@ int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args) {
   if (sms <= 0) sms = 1;
   // the two-SM (cta_group::2) sweeps are the default
   const bool use_pair = args->tile_variant != PSD_LMHEAD_TILES_ONE_SM;
+  CUtensorMap map_a2, map_b2;   // the pair's A / B boxes are 64 x 128
   if (use_pair) {
-    static bool pair_attr[kMaxDevices] = {};
-    if (!pair_attr[dev]) {
-      if (cudaFuncSetAttribute(psd::lmhead_sweep2sm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLm2SmemBytes)) != cudaSuccess ||
-          cudaFuncSetAttribute(psd::lmhead_sweep2sm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(psd::kLm2SmemBytes)) != cudaSuccess) {
-        cudaGetLastError();
-        return PSD_ERR_CUDA;
-      }
-      pair_attr[dev] = true;
-    }
-    // the pair's A / B boxes are 64 x 128
-    CUtensorMap map_a2, map_b2;
-    {
-      const cuuint64_t dims_a[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(M)};
-      const cuuint64_t dims_b[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(V)};
-      const cuuint64_t strides[1] = {static_cast<cuuint64_t>(d_model) * 2};
-      const cuuint32_t box[2] = {psd::kLmK, 128}, estr[2] = {1, 1};
-      if (encode(&map_a2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(hidden), dims_a, strides, box, estr,
-                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
-      if (encode(&map_b2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w_t), dims_b, strides, box, estr,
-                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
-    }
-    const int n_tiles2 = (n_tiles + 1) / 2;
-    const int pairs = n_tiles2 < sms / 2 ? n_tiles2 : sms / 2;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(2 * (pairs > 0 ? pairs : 1)));
-    cfg.blockDim = dim3(psd::kLmThreads);
-    cfg.dynamicSmemBytes = psd::kLm2SmemBytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = 1;
-    TimedLaunch timed(stream, 0);
-    // more than 256 rows: one pair of sweeps per block of 256 rows (the weight is streamed once per block and sweep)
-    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
-      L.row0 = r0;
-      if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<1>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
-    }
-    psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);
-    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
-      L.row0 = r0;
-      if (cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<2>, map_a2, map_b2, L) != cudaSuccess) { cudaGetLastError(); return PSD_ERR_CUDA; }
-    }
-    L.row0 = 0;
-  } else {
-    const unsigned grid = static_cast<unsigned>(n_tiles < sms ? n_tiles : sms);
-    TimedLaunch timed(stream, 0);
-    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
-      L.row0 = r0;
-      psd::lmhead_sweep_kernel<1><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
-    }
-    psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);
-    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
-      L.row0 = r0;
-      psd::lmhead_sweep_kernel<2><<<grid, psd::kLmThreads, psd::kLmSmemBytes, stream>>>(map_a, map_b, L);
-    }
-    L.row0 = 0;
+    const cuuint64_t dims_a[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(M)};
+    const cuuint64_t dims_b[2] = {static_cast<cuuint64_t>(d_model), static_cast<cuuint64_t>(V)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(d_model) * 2};
+    const cuuint32_t box[2] = {psd::kLmK, 128}, estr[2] = {1, 1};
+    if (encode(&map_a2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(hidden), dims_a, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
+    if (encode(&map_b2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w_t), dims_b, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return PSD_ERR_CUDA;
   }
+  const int n_tiles2 = (n_tiles + 1) / 2;
+  const int pairs = n_tiles2 < sms / 2 ? n_tiles2 : sms / 2;
+  const unsigned grid_one = static_cast<unsigned>(n_tiles < sms ? n_tiles : sms);
+  // one GEMM sweep over every block of 256 rows (the weight is streamed once per block and sweep)
+  auto launch_sweep = [&](int sweep) -> bool {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    if (use_pair) {
+      cfg.gridDim = dim3(static_cast<unsigned>(2 * (pairs > 0 ? pairs : 1)));
+      cfg.dynamicSmemBytes = psd::kLm2SmemBytes;
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.attrs = at;
+      cfg.numAttrs = 1;
+    } else {
+      cfg.gridDim = dim3(grid_one);
+      cfg.dynamicSmemBytes = psd::kLmSmemBytes;
+    }
+    cfg.blockDim = dim3(psd::kLmThreads);
+    cfg.stream = stream;
+    for (int r0 = 0; r0 < M; r0 += psd::kLmM) {
+      L.row0 = r0;
+      cudaError_t e;
+      if (use_pair) {
+        if (sweep == 2) e = cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<2, false>, map_a2, map_b2, L);
+        else if (kl) e = cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<1, true>, map_a2, map_b2, L);
+        else e = cudaLaunchKernelEx(&cfg, psd::lmhead_sweep2sm_kernel<1, false>, map_a2, map_b2, L);
+      } else {
+        if (sweep == 2) e = cudaLaunchKernelEx(&cfg, psd::lmhead_sweep_kernel<2, false>, map_a, map_b, L);
+        else if (kl) e = cudaLaunchKernelEx(&cfg, psd::lmhead_sweep_kernel<1, true>, map_a, map_b, L);
+        else e = cudaLaunchKernelEx(&cfg, psd::lmhead_sweep_kernel<1, false>, map_a, map_b, L);
+      }
+      if (e != cudaSuccess) { cudaGetLastError(); return false; }
+    }
+    L.row0 = 0;
+    return true;
+  };
   psd::LmFinalParams F{};
-  F.lm = L;
   F.hidden = static_cast<const __nv_bfloat16*>(hidden);
   F.w_t = static_cast<const __nv_bfloat16*>(w_t);
   F.B = B; F.K = K;
@@ -942,11 +946,28 @@ int pyramidsd_verify_fused_lmhead_ex(const psd_lmhead_args* args) {
   F.out_next_token = out_next_token;
   F.out_div = out_div;
   F.out_resid = out_resid_mass;
+  uint64_t launches = 0;
+  {
+    TimedLaunch timed(stream, 0);
+    if (!launch_sweep(1)) return PSD_ERR_CUDA;
+    psd::lmhead_reduce_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, stream>>>(L);
+    if (kl) {
+      // Kullback-Leibler: the divergences are known after one sweep. The accept scan says whether any rejected row
+      // needs residual masses; only then does the second sweep do anything.
+      F.lm = L;
+      F.kl_phase = 1;
+      psd::lmhead_final_kernel<<<static_cast<unsigned>(B), 256, 0, stream>>>(F);
+      ++launches;
+    }
+    if (!launch_sweep(2)) return PSD_ERR_CUDA;
+  }
+  F.lm = L;
+  F.kl_phase = kl ? 2 : 0;
   {
     TimedLaunch timed(stream, 1);
     psd::lmhead_final_kernel<<<static_cast<unsigned>(B), 256, 0, stream>>>(F);
   }
-  g_launches.fetch_add(2 + 2 * static_cast<uint64_t>((M + psd::kLmM - 1) / psd::kLmM), std::memory_order_relaxed);
+  g_launches.fetch_add(launches + 2 + 2 * static_cast<uint64_t>((M + psd::kLmM - 1) / psd::kLmM), std::memory_order_relaxed);
   return check_launch();
 }
 

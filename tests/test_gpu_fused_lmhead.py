@@ -29,16 +29,17 @@ def make_case(B, K, d, V, seed, sigma_q=0.7, w_scale=0.02):
     return h.contiguous(), w_t.contiguous(), z_q, tok.contiguous()
 
 
-def run_both(psd, oracle, h, w_t, z_q, tok, tau, mode, seed=3, offset=5, tile_variant=None):
+def run_both(psd, oracle, h, w_t, z_q, tok, tau, mode, seed=3, offset=5, tile_variant=None, div_kind=0, want_resid=None):
     dev = torch.device("cuda:0")
     out = psd.verify_fused_lmhead(h.to(dev), w_t.to(dev), z_q.to(dev), tok.to(dev), tau, mode, seed, offset,
-                                  tile_variant=tile_variant)
+                                  tile_variant=tile_variant, div_kind=div_kind, want_resid=want_resid)
     torch.cuda.synchronize()
     assert psd.last_status() == 0
     gpu = {k: v.cpu().numpy() for k, v in out.items() if isinstance(v, torch.Tensor)}
     B, K, V = z_q.shape
     z = oracle.lmhead_logits(host_bits(h), host_bits(w_t.T.contiguous()), n_threads=16).reshape(B, K, V)
-    orc = oracle.verify_stage_mixed(host_bits(z_q), z, tok.numpy(), np.float32(tau), mode, seed, offset, n_threads=16)
+    orc = oracle.verify_stage_mixed(host_bits(z_q), z, tok.numpy(), np.float32(tau), mode, seed, offset, div_kind=div_kind,
+                                    n_threads=16)
     orc["z_large"], orc["z_small"], orc["tokens"], orc["seed"], orc["offset"] = z, host_bits(z_q), tok.numpy(), seed, offset
     return gpu, orc
 
@@ -83,8 +84,11 @@ def classify_mismatch(oracle, gpu, orc, b, tau, mode, gid=None):
 
 
 def check(oracle, gpu, orc, tau, mode, max_token_ties=1):
-    assert np.abs(gpu["div"] - orc["div"]).max() < 2e-3, np.abs(gpu["div"] - orc["div"]).max()
-    assert np.abs(gpu["resid_mass"] - orc["resid_mass"]).max() < 2e-3
+    fin = np.isfinite(orc["div"])
+    assert np.abs(gpu["div"][fin] - orc["div"][fin]).max() < 2e-3, np.abs(gpu["div"][fin] - orc["div"][fin]).max()
+    assert np.all(np.isinf(gpu["div"][np.isinf(orc["div"])]))
+    if "resid_mass" in gpu:
+        assert np.abs(gpu["resid_mass"] - orc["resid_mass"]).max() < 2e-3
     ties = 0
     for b in range(len(orc["accept_len"])):
         if int(gpu["accept_len"][b]) == int(orc["accept_len"][b]) and int(gpu["next_token"][b]) == int(orc["next_token"][b]):
@@ -171,6 +175,40 @@ def test_fused_lmhead_one_sm_variant_agrees(psd, oracle):
     check(oracle, gpu, orc, 0.1, 0)
     gpu2, _ = run_both(psd, oracle, h, w_t, z_q, tok, 0.1, 0)
     assert np.array_equal(gpu["accept_len"], gpu2["accept_len"])
+
+
+@pytest.mark.parametrize("tile_variant", [None, 1])
+def test_fused_lmhead_kl_single_sweep(psd, oracle, tile_variant):
+    """KL(large || small): the divergences come out of the first GEMM sweep; the second one only serves residual masses.
+    Threshold mode with a threshold that splits the rows (rejected rows draw from the residual: the second sweep runs),
+    the same without the residual output, everything accepted (no draw: it returns at once), the assisted mode (draws
+    from p_large off the first sweep's tile sums), strict mode, and a masked small logit under a live large one
+    (divergence +inf). Two row blocks, ragged last tile."""
+    KL = 2
+    h, w_t, z_q, tok = make_case(40, 8, 256, 1500, seed=88, w_scale=0.08)
+    probe, orc = run_both(psd, oracle, h, w_t, z_q, tok, 1e9, 0, div_kind=KL, tile_variant=tile_variant)
+    check(oracle, probe, orc, 1e9, 0)
+    assert np.all(probe["accept_len"] == 8) and np.all(probe["next_token"] == -1)
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 1e9, 0, div_kind=KL, want_resid=False, tile_variant=tile_variant)   # one sweep
+    check(oracle, gpu, orc, 1e9, 0)
+    assert np.array_equal(gpu["div"], probe["div"])
+    tau = float(np.float32(np.median(orc["div"])))
+    for want_resid in (True, False):
+        gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, tau, 0, div_kind=KL, want_resid=want_resid, tile_variant=tile_variant)
+        check(oracle, gpu, orc, tau, 0, max_token_ties=3)
+        assert 0 < orc["accept_len"].sum() < 40 * 8 and np.all((gpu["next_token"] >= 0) == (gpu["accept_len"] < 8))
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.0, 3, div_kind=KL, want_resid=False, tile_variant=tile_variant)   # assisted
+    check(oracle, gpu, orc, 0.0, 3, max_token_ties=3)
+    assert 0 < orc["accept_len"].sum() < 40 * 8
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, 0.0, 1, div_kind=KL, want_resid=False, tile_variant=tile_variant)   # strict
+    check(oracle, gpu, orc, 0.0, 1, max_token_ties=3)
+    z_q[3, 2, 700:760] = -float("inf")
+    gpu, orc = run_both(psd, oracle, h, w_t, z_q, tok, tau, 0, div_kind=KL, tile_variant=tile_variant)
+    assert np.isinf(orc["div"][3, 2]) and np.isinf(gpu["div"][3, 2]) and gpu["accept_len"][3] <= 2
+    check(oracle, gpu, orc, tau, 0, max_token_ties=3)
+    dev = torch.device("cuda:0")
+    bad = psd.verify_fused_lmhead(h.to(dev), w_t.to(dev), z_q.to(dev), tok.to(dev), 0.1, div_kind=1, raise_on_error=False)
+    assert bad["status"] == psd.ERR_UNSUPPORTED          # total variation does not separate: no fused form
 
 
 def test_fused_lmhead_more_than_one_row_block(psd, oracle):
