@@ -1228,16 +1228,16 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, boo
     }
     // Small clusters fill more SMs (148 with one or two CTAs, 135 with three, 132 with four on B200; eight
     // CTAs place only 120), but for a large vocabulary their slice exceeds the ring and has to be streamed
-    // twice. Estimated time = rounds of co-resident clusters / CTAs per row, times a measured factor:
-    //   resident: 1 + 0.01 per CTA of the cluster (the per-row exchange);
-    //   streamed twice: 1.0 (its hand-offs of two chunks at a time make up for the second copy: at equal
-    //   estimates it measures 0 to 3 % faster), plus up to 0.3 once the bytes between a chunk's first and second copy --
-    //   one slice pair per CTA in flight -- outgrow what L2 keeps (48 MB and up: measured 1.04 at 55 MB,
-    //   1.25 at 90 MB).
+    // twice. Estimated time = rounds of co-resident clusters / CTAs per row, times a factor fitted to sweeps
+    // over the cluster size (V = 128256 and 152064, bf16 and fp32, 1536 to 3072 rows):
+    //   resident: 1 + 0.049 per CTA of the cluster (the per-row exchange, and a pipeline that is one row deep);
+    //   streamed twice: 1 + 0.056 per CTA; and once the bytes between a slice's first and second copy -- one row
+    //   per co-resident cluster -- pass 60 MB, L2 no longer serves the second copy: x 1.5 with fp32 logits, which
+    //   then wait for DRAM twice, x 1.08 with bf16 logits, whose arithmetic hides most of it.
     auto rounds_per_cta = [&](int c, int n_active) {
       return static_cast<double>((rows + n_active - 1) / n_active) / c;
     };
-    double best = found ? (1.0 + 0.01 * cs) * rounds_per_cta(cs, cluster_max_active_any(dtype, P.div_kind, cs)) : 1e300;
+    double best = found ? (1.0 + 0.049 * cs) * rounds_per_cta(cs, cluster_max_active_any(dtype, P.div_kind, cs)) : 1e300;
     for (int c2 = 8; c2 >= 1; --c2) {
       int sl2 = 0, ch2 = 0;
       cluster_slices(P.V, es, c2, &sl2, &ch2);
@@ -1245,8 +1245,8 @@ inline bool cluster_geometry(const StageParams& P, int dtype, int forced_cs, boo
       const int na = cluster_max_active_any(dtype, P.div_kind, c2);
       if (na <= 0) continue;
       const double in_flight_mb = 2.0 * sl2 * es * static_cast<double>(na < rows ? na : rows) * c2 / 1048576.0;
-      double factor = 1.0;
-      if (in_flight_mb > 48.0) factor += 0.3 * ((in_flight_mb - 48.0) / 48.0 < 1.0 ? (in_flight_mb - 48.0) / 48.0 : 1.0);
+      double factor = 1.0 + 0.056 * c2;
+      if (in_flight_mb > 60.0) factor *= (es == 4 ? 1.5 : 1.08);
       const double t = factor * rounds_per_cta(c2, na);
       if (t < best) { best = t; cs = c2; slice = sl2; chunks = ch2; restream = true; found = true; }
     }

@@ -319,8 +319,8 @@ def test_cluster_occupancy_query(psd):
     assert cs == 2 and n >= 64
     cs, n = psd.cluster_occupancy(4, 24, 128256, psd.BF16)      # 96 rows: three rounds of 33 clusters of 4 beat two of 74 pairs
     assert cs == 4 and n >= 16
-    cs, n = psd.cluster_occupancy(256, 8, 152064, psd.F32)      # fp32: streamed twice on clusters that fill 130+ SMs
-    assert cs in (4, 5, 6) and n >= 20
+    cs, n = psd.cluster_occupancy(256, 8, 152064, psd.F32)      # fp32: streamed twice on the smallest clusters whose rows in flight fit L2
+    assert cs in (3, 4) and n >= 30
     cs, n = psd.cluster_occupancy(1, 4, 32000, psd.F32)
     assert cs >= 2 and n >= 1
     assert psd.cluster_occupancy(4, 4, 1001, psd.F32) == (0, 0)
