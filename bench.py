@@ -204,8 +204,10 @@ def run_ours(args):
     clocks = sampler.stop()
     # The same K steps once more with an event pair around every launch, for the per-kernel durations of the
     # roofline. Kept out of the pass above: the event records between launches cost a few microseconds each.
+    timed_cap = 4096               # timed launches the library's event timing holds
+    ev_steps = min(args.steps, timed_cap // 4)
     binding.kernel_timing_begin()
-    for i in range(args.steps):
+    for i in range(ev_steps):
         step(args.warmup + i)
     torch.cuda.synchronize()
     ms_rs, n_rs, ms_fin, n_fin = binding.kernel_timing_end()
@@ -218,12 +220,11 @@ def run_ours(args):
     pos_by_buf = [positions_per_step(w, o) for o in outs]
     n_pos = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(args.steps))
     row_bytes = 2 * w.V * es
-    rs_bytes = n_pos * row_bytes   # the statistics kernel streams each verified row pair once
-    timed_cap = 4096               # launches the library's event timing holds; beyond it only the first ones are timed
-    launches_per_step = {"fused": 2, "rows": 2, "separate": 4}.get(args.two_stage) or (4 if launches >= 3 * args.steps else 2)
-    if launches_per_step * args.steps > timed_cap:
-        steps_timed = timed_cap // launches_per_step
-        rs_bytes = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(steps_timed)) * row_bytes
+    # the statistics kernel streams each verified row pair once; the event pass covered the first ev_steps steps
+    rs_bytes = sum(pos_by_buf[(args.warmup + i) % n_bufs] for i in range(ev_steps)) * row_bytes
+    # statistics launches per step: 1 when one launch covers both stages, 2 when the call runs stage by stage (a
+    # finalisation, one or three launches, is timed as one)
+    stats_per_step = max(1, round(n_rs / ev_steps))
 
     # ---- acceptance rates and near ties of the rounds that were timed (one more call per round, with rows) ----
     acc = {"rows_q": 0, "acc_q": 0, "rows_t": 0, "acc_t": 0, "near_q": 0, "near_t": 0}
@@ -305,7 +306,7 @@ def run_ours(args):
                          "traffic": None, "launches": n_rs, "avg_launch_ms": ms_rs / max(n_rs, 1),
                          "finalize_ms_per_launch": ms_fin / max(n_fin, 1),
                          # statistics time per step of the event pass over the step time of the timed pass
-                         "share_of_step": (ms_rs / max(n_rs // (launches_per_step // 2), 1)) / (ms_total / args.steps)
+                         "share_of_step": (ms_rs / ev_steps) / (ms_total / args.steps)
                                           if ms_total > 0 else None,
                          "timing": "CUDA events around every launch, in a second pass over the same K steps"},
             "gpu_launches": launches_all, "clocks": clocks,
@@ -334,7 +335,7 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, rounds)
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
-        traffic = read_profile_traffic(w, "pairs" if args.two_stage == "fused" else "rows") if launches_per_step == 2 else None
+        traffic = read_profile_traffic(w, "pairs" if args.two_stage == "fused" else "rows") if stats_per_step == 1 else None
         if traffic is not None:
             line["roofline"]["traffic"] = traffic
         print(json.dumps(line))

@@ -40,29 +40,53 @@ struct RowView {
   float c, m2l, l2sl, m2s, l2ss;
   bool from_large;  // weights are p_large itself (assisted variant, or an all-zero residual)
 
-  // weights of the kFinElemsPerThread consecutive indices starting at i0 (0 beyond V)
-  __device__ __forceinline__ void weights(int i0, float* w) const {
+  static constexpr int kVecs = kFinElemsPerThread / Elem<T>::kPerVec;   // 16-byte vectors per thread, tile and model
+
+  // whether the thread's indices starting at i0 can be taken as whole vectors
+  __device__ __forceinline__ bool whole(int i0) const { return vec_ok && i0 + kFinElemsPerThread <= V; }
+  // the raw vectors of those indices: loads only, so that a caller can have several tiles' loads in flight
+  __device__ __forceinline__ void fetch(int i0, uint4* rl, uint4* rs) const {
+    constexpr int E = Elem<T>::kPerVec;
+#pragma unroll
+    for (int h = 0; h < kVecs; ++h) {
+      rl[h] = ldg_vec(large, i0 / E + h);
+      rs[h] = ldg_vec(small, i0 / E + h);
+    }
+  }
+  __device__ __forceinline__ void weights_of(const float* xl, const float* xs, float* w) const {
+#pragma unroll
+    for (int j = 0; j < kFinElemsPerThread; ++j) {
+      const float p = ex2_approx(fmaf(xl[j], c, -m2l) - l2sl);
+      const float q = ex2_approx(fmaf(xs[j], c, -m2s) - l2ss);
+      w[j] = from_large ? p : fmaxf(p - q, 0.f);
+    }
+  }
+  // weights from vectors fetched earlier
+  __device__ __forceinline__ void weights_fetched(const uint4* rl, const uint4* rs, float* w) const {
     constexpr int E = Elem<T>::kPerVec;
     float xl[kFinElemsPerThread], xs[kFinElemsPerThread];
-    if (vec_ok && i0 + kFinElemsPerThread <= V) {
 #pragma unroll
-      for (int h = 0; h < kFinElemsPerThread / E; ++h) {
-        Elem<T>::unpack(ldg_vec(large, i0 / E + h), xl + h * E);
-        Elem<T>::unpack(ldg_vec(small, i0 / E + h), xs + h * E);
-      }
+    for (int h = 0; h < kVecs; ++h) {
+      Elem<T>::unpack(rl[h], xl + h * E);
+      Elem<T>::unpack(rs[h], xs + h * E);
+    }
+    weights_of(xl, xs, w);
+  }
+  // weights of the kFinElemsPerThread consecutive indices starting at i0 (0 beyond V)
+  __device__ __forceinline__ void weights(int i0, float* w) const {
+    if (whole(i0)) {
+      uint4 rl[kVecs], rs[kVecs];
+      fetch(i0, rl, rs);
+      weights_fetched(rl, rs, w);
     } else {
+      float xl[kFinElemsPerThread], xs[kFinElemsPerThread];
 #pragma unroll
       for (int j = 0; j < kFinElemsPerThread; ++j) {
         const bool in = i0 + j < V;
         xl[j] = in ? Elem<T>::load(large, i0 + j) : -INFINITY;
         xs[j] = in ? Elem<T>::load(small, i0 + j) : -INFINITY;
       }
-    }
-#pragma unroll
-    for (int j = 0; j < kFinElemsPerThread; ++j) {
-      const float p = ex2_approx(fmaf(xl[j], c, -m2l) - l2sl);
-      const float q = ex2_approx(fmaf(xs[j], c, -m2s) - l2ss);
-      w[j] = from_large ? p : fmaxf(p - q, 0.f);
+      weights_of(xl, xs, w);
     }
   }
 };
@@ -74,6 +98,191 @@ struct FinShared {
   int sh_L, sh_nv, sh_flags, sh_tile, sh_warp, sh_token;
   float sh_u2, sh_m2l, sh_l2sl, sh_m2s, sh_l2ss, sh_resid, sh_target;
 };
+
+// What the accept scan of one sequence hands to the draw: the first rejected position (or the number of valid
+// positions when all were accepted) and the statistics of that position's row.
+struct ScanOut {
+  int L, nv, flags;
+  float u2, m2l, l2sl, m2s, l2ss, resid;
+};
+
+// Accept bits and prefix length of sequence b, by one full warp: lane k owns position k (K <= 32). Every lane
+// returns the same values. `write_rows`: this warp also writes the per-row outputs. `nv_given` >= 0 replaces
+// P.n_valid[b], and `tokens_given` (with `n_given` entries; positions beyond it count as token 0) replaces
+// P.tokens for this sequence.
+template <typename T>
+__device__ __forceinline__ ScanOut scan_unit(const StageParams& P, const int b, const int lane, const bool write_rows,
+                                             const int nv_given, const int32_t* tokens_given, const int n_given) {
+  const int K = P.K, V = P.V;
+  const T* large_seq = static_cast<const T*>(P.large) + b * P.seq_stride_large;
+  const T* small_seq = static_cast<const T*>(P.small) + b * P.seq_stride_small;
+  int nv = K;
+  if (nv_given >= 0) nv = min(nv_given, K);
+  else if (P.n_valid != nullptr) nv = min(max(P.n_valid[b], 0), K);
+
+  bool acc = true;  // lanes beyond nv never end the prefix
+  RowStats st{};
+  float u = 0.f, u2 = 0.f;
+  int flags = 0;
+  if (lane < nv) {
+    const int r = b * K + lane;
+    st = P.stats[r];
+    const int x = (tokens_given != nullptr) ? (lane < n_given ? tokens_given[lane] : 0) : P.tokens[r];
+    flags = st.flags | ((x < 0 || x >= V) ? kFlagTokenRange : 0);
+    row_uniforms(P.seed, P.offset, static_cast<unsigned>((P.seq_base + b) * K + lane), &u, &u2);
+    const float nanf_ = __int_as_float(0x7fc00000);
+    float px = nanf_, qx = nanf_;
+    bool coin_ok = false;
+    if (!flags) {
+      const long long off = static_cast<long long>(lane) * V + x;
+      px = ex2_approx(fmaf(Elem<T>::load(large_seq, off), P.c, -st.m2_large) - st.l2s_large);
+      qx = ex2_approx(fmaf(Elem<T>::load(small_seq, off), P.c, -st.m2_small) - st.l2s_small);
+      // standard SD: accept with probability min(1, p_large(x) / p_small(x))
+      const float rho = (qx > 0.f) ? __fdiv_rn(px, qx) : (px > 0.f ? INFINITY : 0.f);
+      coin_ok = u < fminf(1.f, rho);
+    }
+    const bool fuzzy_ok = st.div <= P.threshold;
+    if (P.mode == kModeFuzzy) acc = fuzzy_ok;
+    else if (P.mode == kModeStrict || P.mode == kModeAssisted) acc = coin_ok;
+    else acc = fuzzy_ok || coin_ok;
+    if (flags) acc = false;
+    if (write_rows) {
+      if (P.out_div) P.out_div[r] = st.div;
+      if (P.out_resid_mass) P.out_resid_mass[r] = st.resid;
+      if (P.out_p_small_tok) P.out_p_small_tok[r] = qx;
+      if (P.out_p_large_tok) P.out_p_large_tok[r] = px;
+      if (P.out_row_flags) P.out_row_flags[r] = flags;
+    }
+  } else if (lane < K && write_rows) {
+    const int r = b * K + lane;
+    if (P.out_div) P.out_div[r] = 0.f;
+    if (P.out_resid_mass) P.out_resid_mass[r] = 0.f;
+    if (P.out_p_small_tok) P.out_p_small_tok[r] = 0.f;
+    if (P.out_p_large_tok) P.out_p_large_tok[r] = 0.f;
+    if (P.out_row_flags) P.out_row_flags[r] = 0;
+  }
+  const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
+  const int L = rejected ? (__ffs(rejected) - 1) : nv;  // first rejected position, or all accepted
+  const int src = min(L, 31);   // L < nv <= 32 when a rejection exists; otherwise the row data go unused
+  ScanOut o;
+  o.L = L;
+  o.nv = nv;
+  o.flags = __shfl_sync(0xffffffffu, flags, src);
+  o.u2 = __shfl_sync(0xffffffffu, u2, src);
+  o.m2l = __shfl_sync(0xffffffffu, st.m2_large, src);
+  o.l2sl = __shfl_sync(0xffffffffu, st.l2s_large, src);
+  o.m2s = __shfl_sync(0xffffffffu, st.m2_small, src);
+  o.l2ss = __shfl_sync(0xffffffffu, st.l2s_small, src);
+  o.resid = __shfl_sync(0xffffffffu, st.resid, src);
+  return o;
+}
+
+// The results of one sequence, by one thread: prefix length, next token, and in the two-stage wrapper the stage-2
+// window (Fig. 1): accepted draft tokens, then the correction token.
+__device__ __forceinline__ void write_results(const StageParams& P, const int b, const int L, const int next) {
+  P.out_accept_len[b] = L;
+  P.out_next_token[b] = next;
+  if (P.window != nullptr) {
+    const int have = L + (next >= 0 ? 1 : 0);
+    const int n2 = min(have, P.K_window);
+    P.n_window[b] = n2;
+    if (P.fill_out != nullptr && b < P.fill_cap) P.fill_out[b] = n2;
+    for (int j = 0; j < P.K_window; ++j)
+      P.window[b * P.K_window + j] = (j < n2) ? ((j < L) ? P.tokens[b * P.K + j] : next) : 0;
+  }
+}
+
+// Level 0 of the draw, by one thread, once every tile's total is in S.tile_total: the first tile whose inclusive
+// cumulative weight exceeds the target, else the last non-empty tile. Leaves the tile in S.sh_tile (-1: no
+// positive weight at all; -2: the residual weights all came out zero, take the totals again over p_large) and
+// the target that remains inside it in S.sh_target.
+__device__ __forceinline__ void pick_tile(FinShared& S, const int n_tiles, const bool from_large) {
+  const double* tile_total = S.tile_total;
+  double total = 0.0;
+  for (int j = 0; j < n_tiles; ++j) total += tile_total[j];
+  const double target = static_cast<double>(S.sh_u2) * total;
+  const bool redo = !(total > 0.0) && !from_large;
+  int pick = -1, last_pos = -1;
+  double cum = 0.0, cum_before_pick = 0.0, cum_before_last = 0.0;
+  for (int j = 0; j < n_tiles; ++j) {
+    const double nxt = cum + tile_total[j];
+    if (tile_total[j] > 0.0) { last_pos = j; cum_before_last = cum; }
+    if (pick < 0 && nxt > target && tile_total[j] > 0.0) { pick = j; cum_before_pick = cum; }
+    cum = nxt;
+  }
+  if (pick < 0) { pick = last_pos; cum_before_pick = cum_before_last; }
+  S.sh_tile = redo ? -2 : pick;
+  S.sh_token = -1;
+  S.sh_target = static_cast<float>(target - cum_before_pick);
+}
+
+// Levels 1 to 3 of the draw inside the chosen tile, by the whole CTA: warps, lanes, the thread's own elements.
+// Leaves the token in S.sh_token (valid after the closing barrier).
+template <typename T>
+__device__ __forceinline__ void descend_tile(const RowView<T>& row, FinShared& S, const int tile) {
+  float (&warp_total)[32] = S.warp_total;
+  int &sh_warp = S.sh_warp, &sh_token = S.sh_token;
+  float &sh_target = S.sh_target;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float w[kFinElemsPerThread];
+  {
+    // level 1: warps of the chosen tile
+    const int i0 = tile * kFinTile + tid * kFinElemsPerThread;
+    row.weights(i0, w);
+    float ts = 0.f;
+#pragma unroll
+    for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
+    // inclusive scan of thread sums across the warp (fixed shuffle tree)
+    float incl = ts;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float up = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    if (lane == 31) warp_total[warp] = incl;
+    __syncthreads();
+    if (tid == 0) {
+      const float target = sh_target;
+      int pick = -1, last_pos = -1;
+      float cum = 0.f, before_pick = 0.f, before_last = 0.f;
+      for (int j = 0; j < kFinThreads / 32; ++j) {
+        const float nxt = cum + warp_total[j];
+        if (warp_total[j] > 0.f) { last_pos = j; before_last = cum; }
+        if (pick < 0 && nxt > target && warp_total[j] > 0.f) { pick = j; before_pick = cum; }
+        cum = nxt;
+      }
+      if (pick < 0) { pick = last_pos; before_pick = before_last; }
+      sh_warp = pick;
+      sh_target = target - before_pick;
+    }
+    __syncthreads();
+    if (warp == sh_warp) {
+      // level 2: lanes of the chosen warp
+      const float target = sh_target;
+      const float excl = incl - ts;  // only used as the offset handed to the next level
+      const unsigned hit = __ballot_sync(0xffffffffu, incl > target && ts > 0.f);
+      const unsigned pos = __ballot_sync(0xffffffffu, ts > 0.f);
+      const int pick_lane = hit ? (__ffs(hit) - 1) : (pos ? 31 - __clz(pos) : -1);
+      if (lane == pick_lane) {
+        // level 3: the thread's own consecutive elements
+        const float t3 = target - excl;
+        float run = 0.f;
+        int choice = -1, last_pos = -1;
+#pragma unroll
+        for (int e = 0; e < kFinElemsPerThread; ++e) {
+          run += w[e];
+          if (w[e] > 0.f) {
+            last_pos = e;
+            if (choice < 0 && run > t3) choice = e;
+          }
+        }
+        if (choice < 0) choice = last_pos;
+        sh_token = (choice >= 0) ? i0 + choice : -1;
+      }
+    }
+    __syncthreads();
+  }
+}
 
 // One stage's finalisation of sequence b; every thread of the CTA calls it. With CL > 1 the CTAs of a
 // cluster all call it for the same sequence: each repeats the (cheap) accept scan, the tile sums of the draw
@@ -97,63 +306,17 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
   const T* large_seq = static_cast<const T*>(P.large) + b * P.seq_stride_large;
   const T* small_seq = static_cast<const T*>(P.small) + b * P.seq_stride_small;
 
-  int nv = K;
-  if (nv_given >= 0) nv = min(nv_given, K);
-  else if (P.n_valid != nullptr) nv = min(max(P.n_valid[b], 0), K);
-
   // ---- accept bits and prefix length: lane k of warp 0 owns position k (K <= 32) ----
   if (warp == 0) {
-    bool acc = true;  // lanes beyond nv never end the prefix
-    RowStats st{};
-    float u = 0.f, u2 = 0.f;
-    int flags = 0;
-    if (lane < nv) {
-      const int r = b * K + lane;
-      st = P.stats[r];
-      const int x = (tokens_given != nullptr) ? (lane < n_given ? tokens_given[lane] : 0) : P.tokens[r];
-      flags = st.flags | ((x < 0 || x >= V) ? kFlagTokenRange : 0);
-      row_uniforms(P.seed, P.offset, static_cast<unsigned>((P.seq_base + b) * K + lane), &u, &u2);
-      const float nanf_ = __int_as_float(0x7fc00000);
-      float px = nanf_, qx = nanf_;
-      bool coin_ok = false;
-      if (!flags) {
-        const long long off = static_cast<long long>(lane) * V + x;
-        px = ex2_approx(fmaf(Elem<T>::load(large_seq, off), P.c, -st.m2_large) - st.l2s_large);
-        qx = ex2_approx(fmaf(Elem<T>::load(small_seq, off), P.c, -st.m2_small) - st.l2s_small);
-        // standard SD: accept with probability min(1, p_large(x) / p_small(x))
-        const float rho = (qx > 0.f) ? __fdiv_rn(px, qx) : (px > 0.f ? INFINITY : 0.f);
-        coin_ok = u < fminf(1.f, rho);
-      }
-      const bool fuzzy_ok = st.div <= P.threshold;
-      if (P.mode == kModeFuzzy) acc = fuzzy_ok;
-      else if (P.mode == kModeStrict || P.mode == kModeAssisted) acc = coin_ok;
-      else acc = fuzzy_ok || coin_ok;
-      if (flags) acc = false;
-      if (cl_rank == 0) {
-        if (P.out_div) P.out_div[r] = st.div;
-        if (P.out_resid_mass) P.out_resid_mass[r] = st.resid;
-        if (P.out_p_small_tok) P.out_p_small_tok[r] = qx;
-        if (P.out_p_large_tok) P.out_p_large_tok[r] = px;
-        if (P.out_row_flags) P.out_row_flags[r] = flags;
-      }
-    } else if (lane < K && cl_rank == 0) {
-      const int r = b * K + lane;
-      if (P.out_div) P.out_div[r] = 0.f;
-      if (P.out_resid_mass) P.out_resid_mass[r] = 0.f;
-      if (P.out_p_small_tok) P.out_p_small_tok[r] = 0.f;
-      if (P.out_p_large_tok) P.out_p_large_tok[r] = 0.f;
-      if (P.out_row_flags) P.out_row_flags[r] = 0;
-    }
-    const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
-    const int L = rejected ? (__ffs(rejected) - 1) : nv;  // first rejected position, or all accepted
-    if (lane == min(L, 31)) {  // L < nv <= 32 when a rejection exists; otherwise the row data go unused
-      sh_L = L;
-      sh_nv = nv;
-      sh_flags = flags;
-      sh_u2 = u2;
-      sh_m2l = st.m2_large; sh_l2sl = st.l2s_large;
-      sh_m2s = st.m2_small; sh_l2ss = st.l2s_small;
-      sh_resid = st.resid;
+    const ScanOut o = scan_unit<T>(P, b, lane, cl_rank == 0, nv_given, tokens_given, n_given);
+    if (lane == 0) {
+      sh_L = o.L;
+      sh_nv = o.nv;
+      sh_flags = o.flags;
+      sh_u2 = o.u2;
+      sh_m2l = o.m2l; sh_l2sl = o.l2sl;
+      sh_m2s = o.m2s; sh_l2ss = o.l2ss;
+      sh_resid = o.resid;
     }
   }
   __syncthreads();
@@ -261,25 +424,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
       __syncthreads();
     }
     if (CL > 1) fin_cluster_sync();   // every CTA now holds every tile's total
-    if (tid == 0) {
-      double total = 0.0;
-      for (int j = 0; j < n_tiles; ++j) total += tile_total[j];
-      const double target = static_cast<double>(sh_u2) * total;
-      const bool redo = !(total > 0.0) && !row.from_large;
-      // first tile whose inclusive cumulative weight exceeds the target; else the last non-empty tile
-      int pick = -1, last_pos = -1;
-      double cum = 0.0, cum_before_pick = 0.0, cum_before_last = 0.0;
-      for (int j = 0; j < n_tiles; ++j) {
-        const double nxt = cum + tile_total[j];
-        if (tile_total[j] > 0.0) { last_pos = j; cum_before_last = cum; }
-        if (pick < 0 && nxt > target && tile_total[j] > 0.0) { pick = j; cum_before_pick = cum; }
-        cum = nxt;
-      }
-      if (pick < 0) { pick = last_pos; cum_before_pick = cum_before_last; }
-      sh_tile = redo ? -2 : pick;
-      sh_token = -1;
-      sh_target = static_cast<float>(target - cum_before_pick);
-    }
+    if (tid == 0) pick_tile(S, n_tiles, row.from_large);
     __syncthreads();
     if (sh_tile != -2) break;
     row.from_large = true;            // every CTA of the cluster holds the same totals and takes the same turn
@@ -289,82 +434,16 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
     const int tile = sh_tile;
     writer = (CL > 1 && tile >= 0) ? static_cast<unsigned>(tile % CL) : 0u;   // the CTA that summed the chosen tile goes on
     if (tile >= 0 && cl_rank == writer) {
-      // level 1: warps of the chosen tile
-      const int i0 = tile * kFinTile + tid * kFinElemsPerThread;
-      row.weights(i0, w);
-      float ts = 0.f;
-#pragma unroll
-      for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
-      // inclusive scan of thread sums across the warp (fixed shuffle tree)
-      float incl = ts;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const float up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-      }
-      if (lane == 31) warp_total[warp] = incl;
-      __syncthreads();
-      if (tid == 0) {
-        const float target = sh_target;
-        int pick = -1, last_pos = -1;
-        float cum = 0.f, before_pick = 0.f, before_last = 0.f;
-        for (int j = 0; j < kFinThreads / 32; ++j) {
-          const float nxt = cum + warp_total[j];
-          if (warp_total[j] > 0.f) { last_pos = j; before_last = cum; }
-          if (pick < 0 && nxt > target && warp_total[j] > 0.f) { pick = j; before_pick = cum; }
-          cum = nxt;
-        }
-        if (pick < 0) { pick = last_pos; before_pick = before_last; }
-        sh_warp = pick;
-        sh_target = target - before_pick;
-      }
-      __syncthreads();
-      if (warp == sh_warp) {
-        // level 2: lanes of the chosen warp
-        const float target = sh_target;
-        const float excl = incl - ts;  // only used as the offset handed to the next level
-        const unsigned hit = __ballot_sync(0xffffffffu, incl > target && ts > 0.f);
-        const unsigned pos = __ballot_sync(0xffffffffu, ts > 0.f);
-        const int pick_lane = hit ? (__ffs(hit) - 1) : (pos ? 31 - __clz(pos) : -1);
-        if (lane == pick_lane) {
-          // level 3: the thread's own consecutive elements
-          const float t3 = target - excl;
-          float run = 0.f;
-          int choice = -1, last_pos = -1;
-#pragma unroll
-          for (int e = 0; e < kFinElemsPerThread; ++e) {
-            run += w[e];
-            if (w[e] > 0.f) {
-              last_pos = e;
-              if (choice < 0 && run > t3) choice = e;
-            }
-          }
-          if (choice < 0) choice = last_pos;
-          sh_token = (choice >= 0) ? i0 + choice : -1;
-        }
-      }
-      __syncthreads();
+      descend_tile<T>(row, S, tile);
       next = sh_token;
     }
   }
 
-  if (tid == 0 && cl_rank == writer) {
-    P.out_accept_len[b] = L;
-    P.out_next_token[b] = next;
-    if (P.window != nullptr) {
-      // stage-2 window of the two-stage wrapper (Fig. 1): accepted draft tokens, then the correction token
-      const int have = L + (next >= 0 ? 1 : 0);
-      const int n2 = min(have, P.K_window);
-      P.n_window[b] = n2;
-      if (P.fill_out != nullptr && b < P.fill_cap) P.fill_out[b] = n2;
-      for (int j = 0; j < P.K_window; ++j)
-        P.window[b * P.K_window + j] = (j < n2) ? ((j < L) ? P.tokens[b * K + j] : next) : 0;
-    }
-  }
+  if (tid == 0 && cl_rank == writer) write_results(P, b, L, next);
 }
 
 template <typename T, int CL>
-__global__ void __launch_bounds__(kFinThreads) finalize_kernel(const StageParams P) {
+__global__ void __launch_bounds__(kFinThreads, 1) finalize_kernel(const StageParams P) {
   __shared__ FinShared S;
   finalize_sequence<T, CL>(P, blockIdx.x / CL, S);
   if (CL > 1) fin_cluster_sync();   // nobody leaves while a peer may still post tile sums into its shared memory
@@ -418,6 +497,265 @@ __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_split_kernel(con
     finalize_sequence<T, CL>(P2, b, S, sh_n2, P1.tokens + b * P1.K, sh_L1);
   }
   if (CL > 1) fin_cluster_sync();
+}
+
+// ---- finalisation of a large batch in three launches -------------------------------------------------------
+// With one CTA (or pair) per sequence a draw is a chain of dependent steps on one SM -- the tile totals alone take
+// a microsecond per tile -- while the SMs whose sequences accepted everything idle; and when every sequence
+// draws, the CTAs come in waves. For batches that fill the GPU the work is cut differently. A scan launch (one
+// warp per sequence and stage) takes the accept bits, finishes the sequences that need no draw and leaves a record
+// for each one that does. A tile launch of one CTA per SM spreads level 0 of all draws, the (record, tile) pairs,
+// over all CTAs. A pick launch then gives each draw a CTA for the pick and levels 1 to 3. Launch boundaries order
+// the three; no CTA waits for another and nothing is counted atomically. Each tile total, the pick and the descent
+// are the code of the one-launch form, so both forms return the same bits.
+constexpr int kDrawMaxTiles = 32;      // V <= 262144
+constexpr int kDrawMaxUnits = 4096;    // sequences x stages of one call
+constexpr int kScanWarps = 4;
+
+struct DrawRecord {
+  int L;
+  float u2, m2l, l2sl, m2s, l2ss, resid;
+  int pad;
+};
+
+struct DrawScratch {
+  int* need;            // [units] 1: the unit draws
+  int* list;            // [0]: number of drawing units; [1 + d]: the d-th of them, in unit order
+  DrawRecord* record;   // [units]
+  double* tile_total;   // [units][kDrawMaxTiles]
+};
+
+__host__ __device__ inline size_t draw_scratch_bytes(long long units) {
+  return static_cast<size_t>(units) * (2 * sizeof(int) + sizeof(DrawRecord) + kDrawMaxTiles * sizeof(double)) + 256;
+}
+
+// The three launches may start while the launch before them drains; they read nothing of it before this.
+__device__ __forceinline__ void wait_for_previous_launch() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next launch on the stream, if it was launched as a dependent, be scheduled from here on.
+__device__ __forceinline__ void release_next_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+// The window length and token source of the stage-2 half of a fuzzy pyramid: stage 1's threshold scan again.
+__device__ __forceinline__ void stage1_prefix(const StageParams& P1, const int K2, const int b, const int lane, int* L1, int* n2) {
+  const int K = P1.K;
+  bool acc = true;
+  int flags = 0;
+  if (lane < K) {
+    const RowStats st = P1.stats[b * K + lane];
+    const int x = P1.tokens[b * K + lane];
+    flags = st.flags | ((x < 0 || x >= P1.V) ? kFlagTokenRange : 0);
+    acc = (st.div <= P1.threshold) && !flags;
+  }
+  const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
+  *L1 = rejected ? (__ffs(rejected) - 1) : K;
+  const int flags_L = __shfl_sync(0xffffffffu, flags, min(*L1, 31));
+  // a correction token follows the accepted prefix unless everything was accepted or the rejected row has no distribution
+  const int has_next = (*L1 < K && !(flags_L & (kFlagSmallNonfinite | kFlagLargeNonfinite))) ? 1 : 0;
+  *n2 = min(*L1 + has_next, K2);
+}
+
+// Scan launch: unit = sequence (n_stages == 1) or 2 * sequence + stage (the side-by-side form of a fuzzy pyramid).
+template <typename T>
+__global__ void __launch_bounds__(kScanWarps * 32) finalize_scan_kernel(const StageParams P1, const StageParams P2, const int n_stages,
+                                                                        const DrawScratch ds) {
+  wait_for_previous_launch();
+  release_next_launch();
+  const int lane = threadIdx.x & 31;
+  const int unit = blockIdx.x * kScanWarps + (threadIdx.x >> 5);
+  if (unit >= n_stages * P1.B) return;   // whole warps leave
+  const int b = (n_stages == 2) ? unit >> 1 : unit;
+  const bool second = (n_stages == 2) && (unit & 1);
+  ScanOut o;
+  if (!second) {
+    o = scan_unit<T>(P1, b, lane, true, -1, nullptr, 0);
+  } else {
+    int L1, n2;
+    stage1_prefix(P1, P2.K, b, lane, &L1, &n2);
+    o = scan_unit<T>(P2, b, lane, true, n2, P1.tokens + b * P1.K, L1);
+  }
+  if (lane == 0) {
+    int next = -1;
+    bool draw = false;
+    if (o.L < o.nv) {
+      if (o.flags & (kFlagSmallNonfinite | kFlagLargeNonfinite)) next = -2;   // no distribution to draw from
+      else draw = true;
+    }
+    ds.need[unit] = draw ? 1 : 0;
+    if (draw) {
+      DrawRecord r;
+      r.L = o.L; r.u2 = o.u2; r.m2l = o.m2l; r.l2sl = o.l2sl; r.m2s = o.m2s; r.l2ss = o.l2ss; r.resid = o.resid; r.pad = 0;
+      ds.record[unit] = r;
+    } else {
+      write_results(second ? P2 : P1, b, o.L, next);
+    }
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ RowView<T> draw_row(const StageParams& P, const int b, const DrawRecord& r) {
+  RowView<T> row;
+  row.large = static_cast<const T*>(P.large) + b * P.seq_stride_large + static_cast<long long>(r.L) * P.V;
+  row.small = static_cast<const T*>(P.small) + b * P.seq_stride_small + static_cast<long long>(r.L) * P.V;
+  row.V = P.V;
+  row.vec_ok = ((reinterpret_cast<uintptr_t>(row.large) | reinterpret_cast<uintptr_t>(row.small)) & 15u) == 0 &&
+               (P.V % Elem<T>::kPerVec) == 0;
+  row.c = P.c;
+  row.m2l = r.m2l; row.l2sl = r.l2sl;
+  row.m2s = r.m2s; row.l2ss = r.l2ss;
+  row.from_large = (P.mode == kModeAssisted) || !(r.resid > 0.f);
+  return row;
+}
+
+template <typename T>
+struct TileShared {
+  RowView<T> row[kFinBatch];            // the rows of a batch of (record, tile) pairs
+  double* out[kFinBatch];               // where each pair's total goes
+  int i_base[kFinBatch];                // first vocabulary index of each pair's tile
+  float warp_tile[kFinBatch][32];
+  unsigned short list[kDrawMaxUnits];   // the units that draw, in unit order
+  int warp_count[32];
+  int n_list;
+};
+
+// Tile launch: level 0 of every draw. One CTA per SM; any grid size gives the same totals.
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads) finalize_tiles_kernel(const StageParams P1, const StageParams P2, const int n_stages,
+                                                                     const DrawScratch ds) {
+  __shared__ TileShared<T> S;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int units = n_stages * P1.B;
+  // every CTA builds the same list of drawing units, in unit order; CTA 0 leaves it for the pick launch
+  if (tid == 0) S.n_list = 0;
+  wait_for_previous_launch();
+  release_next_launch();
+  __syncthreads();
+  for (int base = 0; base < units; base += kFinThreads) {
+    const int unit = base + tid;
+    const bool need = unit < units && ds.need[unit] != 0;
+    const unsigned m = __ballot_sync(0xffffffffu, need);
+    if (lane == 0) S.warp_count[warp] = __popc(m);
+    __syncthreads();
+    int before = S.n_list;
+    for (int k = 0; k < warp; ++k) before += S.warp_count[k];
+    if (need) {
+      const int pos = before + __popc(m & ((1u << lane) - 1u));
+      S.list[pos] = static_cast<unsigned short>(unit);
+      if (blockIdx.x == 0) ds.list[1 + pos] = unit;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int total = S.n_list;
+      for (int k = 0; k < kFinThreads / 32; ++k) total += S.warp_count[k];
+      S.n_list = total;
+    }
+    __syncthreads();
+  }
+  const int n_list = S.n_list;
+  if (blockIdx.x == 0 && tid == 0) ds.list[0] = n_list;
+  if (n_list == 0) return;
+  const int n_tiles = (P1.V + kFinTile - 1) / kFinTile;
+  const int items = n_list * n_tiles;   // <= kDrawMaxUnits * kDrawMaxTiles
+
+  for (int first = blockIdx.x; first < items; first += static_cast<int>(gridDim.x) * kFinBatch) {
+    const int nb = min(kFinBatch, (items - first + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x));
+    if (tid < nb) {
+      const int item = first + tid * static_cast<int>(gridDim.x);
+      const int unit = S.list[item / n_tiles], j = item % n_tiles;
+      const bool second = (n_stages == 2) && (unit & 1);
+      S.row[tid] = draw_row<T>(second ? P2 : P1, (n_stages == 2) ? unit >> 1 : unit, ds.record[unit]);
+      S.out[tid] = ds.tile_total + unit * kDrawMaxTiles + j;
+      S.i_base[tid] = j * kFinTile;
+    }
+    __syncthreads();
+    // the loads of kTileDepth pairs (32 registers of vectors) are issued before the first of them is used
+    constexpr int kTileDepth = 4 / RowView<T>::kVecs;
+    for (int m = 0; m < nb; m += kTileDepth) {
+      uint4 rl[kTileDepth][RowView<T>::kVecs], rs[kTileDepth][RowView<T>::kVecs];
+      bool fetched[kTileDepth];
+#pragma unroll
+      for (int d = 0; d < kTileDepth; ++d) {
+        fetched[d] = false;
+        if (m + d < nb) {
+          const int i0 = S.i_base[m + d] + tid * kFinElemsPerThread;
+          fetched[d] = S.row[m + d].whole(i0);
+          if (fetched[d]) S.row[m + d].fetch(i0, rl[d], rs[d]);
+        }
+      }
+#pragma unroll
+      for (int d = 0; d < kTileDepth; ++d) {
+        if (m + d < nb) {   // uniform across the CTA
+          float w[kFinElemsPerThread];
+          if (fetched[d]) S.row[m + d].weights_fetched(rl[d], rs[d], w);
+          else S.row[m + d].weights(S.i_base[m + d] + tid * kFinElemsPerThread, w);
+          float ts = 0.f;
+#pragma unroll
+          for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
+          ts = warp_reduce<OpSum>(ts);
+          if (lane == 0) S.warp_tile[m + d][warp] = ts;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < nb) {
+      double tt = 0.0;
+      for (int k = 0; k < 32; ++k) tt += static_cast<double>(S.warp_tile[tid][k]);
+      *S.out[tid] = tt;
+    }
+    __syncthreads();   // the batch's shared memory is free again
+  }
+}
+
+// Pick launch: the pick among the tile totals and levels 1 to 3, one draw per CTA at a time.
+template <typename T>
+__global__ void __launch_bounds__(kFinThreads) finalize_pick_kernel(const StageParams P1, const StageParams P2, const int n_stages,
+                                                                    const DrawScratch ds) {
+  __shared__ FinShared S;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  wait_for_previous_launch();
+  const int n_list = ds.list[0];
+  const int n_tiles = (P1.V + kFinTile - 1) / kFinTile;
+  for (int d = blockIdx.x; d < n_list; d += gridDim.x) {
+    const int unit = ds.list[1 + d];
+    const bool second = (n_stages == 2) && (unit & 1);
+    const StageParams& P = second ? P2 : P1;
+    const int b = (n_stages == 2) ? unit >> 1 : unit;
+    const DrawRecord rec = ds.record[unit];
+    RowView<T> row = draw_row<T>(P, b, rec);
+    if (tid < n_tiles) S.tile_total[tid] = ds.tile_total[unit * kDrawMaxTiles + tid];
+    if (tid == 0) S.sh_u2 = rec.u2;
+    __syncthreads();
+    if (tid == 0) pick_tile(S, n_tiles, row.from_large);
+    __syncthreads();
+    if (S.sh_tile == -2) {
+      // the residual weights all came out zero although the row's residual mass did not: the totals again, over p_large
+      row.from_large = true;
+      for (int j = 0; j < n_tiles; ++j) {
+        float w[kFinElemsPerThread];
+        row.weights(j * kFinTile + tid * kFinElemsPerThread, w);
+        float ts = 0.f;
+#pragma unroll
+        for (int e = 0; e < kFinElemsPerThread; ++e) ts += w[e];
+        ts = warp_reduce<OpSum>(ts);
+        if (lane == 0) S.warp_tile[0][warp] = ts;
+        __syncthreads();
+        if (tid == 0) {
+          double tt = 0.0;
+          for (int k = 0; k < 32; ++k) tt += static_cast<double>(S.warp_tile[0][k]);
+          S.tile_total[j] = tt;
+        }
+        __syncthreads();
+      }
+      if (tid == 0) pick_tile(S, n_tiles, true);
+      __syncthreads();
+    }
+    const int tile = S.sh_tile;
+    int next = -1;
+    if (tile >= 0) {
+      descend_tile<T>(row, S, tile);
+      next = S.sh_token;
+    }
+    if (tid == 0) write_results(P, b, rec.L, next);
+    __syncthreads();   // S is free for the next draw
+  }
 }
 
 }  // namespace psd

@@ -59,6 +59,8 @@ struct StreamScratch {
   size_t out4_bytes = 0;
   void* lm_ws = nullptr;    // partial sums of the fused LM-head path
   size_t lm_ws_bytes = 0;
+  void* draw = nullptr;     // records and tile totals of the three-launch finalisation
+  size_t draw_bytes = 0;
 };
 struct DeviceState {
   std::mutex mu;
@@ -266,8 +268,64 @@ int fin_cluster_size(long long units) {
    : (cl) == 2 ? launch_fin_clusters(psd::KERNEL<T, 2>, 2, units, stream, __VA_ARGS__)                      \
                : launch_fin_clusters(psd::KERNEL<T, 1>, 1, units, stream, __VA_ARGS__))
 
-int launch_finalize(const StageParams& P, int dtype, cudaStream_t stream) {
+// Whether a finalisation of `units` sequences (x stages) goes as three launches (scan, tile totals, pick): batches for
+// which the one-launch form would give a draw fewer than four CTAs, within the limits of the draw records.
+bool split_finalize(long long units, int V, bool bonus, const StreamScratch* ss) {
+  if (ss == nullptr || bonus) return false;
+  if (fin_cluster_size(units) == 4 || units > psd::kDrawMaxUnits) return false;
+  return (V + psd::kFinTile - 1) / psd::kFinTile <= psd::kDrawMaxTiles;
+}
+
+// A launch that may begin while the launch before it on the stream drains (programmatic dependent launch): the
+// kernel itself waits, with griddepcontrol.wait, before it reads what that launch wrote.
+template <typename Kernel, typename... Args>
+cudaError_t launch_dependent(Kernel kernel, unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+int launch_finalize_split(const StageParams& P1, const StageParams& P2, int n_stages, int dtype, cudaStream_t stream,
+                        StreamScratch* ss) {
+  const long long units = static_cast<long long>(n_stages) * P1.B;
+  int rc = grow(ss, &ss->draw, &ss->draw_bytes, psd::draw_scratch_bytes(units));
+  if (rc != PSD_OK) return rc;
+  psd::DrawScratch d;
+  char* base = static_cast<char*>(ss->draw);
+  d.tile_total = reinterpret_cast<double*>(base);
+  base += static_cast<size_t>(units) * psd::kDrawMaxTiles * sizeof(double);
+  d.record = reinterpret_cast<psd::DrawRecord*>(base);
+  base += static_cast<size_t>(units) * sizeof(psd::DrawRecord);
+  d.need = reinterpret_cast<int*>(base);
+  d.list = d.need + units;   // 1 + units entries at most: the 256 spare bytes hold the count
+  int sms = psd::cluster_sm_count();
+  if (sms <= 0) sms = 148;
+  const unsigned scan_ctas = static_cast<unsigned>((units + psd::kScanWarps - 1) / psd::kScanWarps);
+  TimedLaunch timed(stream, 1);
+  if (dtype == PSD_F32) {
+    launch_dependent(psd::finalize_scan_kernel<float>, scan_ctas, psd::kScanWarps * 32, stream, P1, P2, n_stages, d);
+    launch_dependent(psd::finalize_tiles_kernel<float>, sms, psd::kFinThreads, stream, P1, P2, n_stages, d);
+    launch_dependent(psd::finalize_pick_kernel<float>, sms, psd::kFinThreads, stream, P1, P2, n_stages, d);
+  } else {
+    launch_dependent(psd::finalize_scan_kernel<__nv_bfloat16>, scan_ctas, psd::kScanWarps * 32, stream, P1, P2, n_stages, d);
+    launch_dependent(psd::finalize_tiles_kernel<__nv_bfloat16>, sms, psd::kFinThreads, stream, P1, P2, n_stages, d);
+    launch_dependent(psd::finalize_pick_kernel<__nv_bfloat16>, sms, psd::kFinThreads, stream, P1, P2, n_stages, d);
+  }
+  g_launches.fetch_add(3, std::memory_order_relaxed);
+  return check_launch();
+}
+
+int launch_finalize(const StageParams& P, int dtype, cudaStream_t stream, StreamScratch* ss = nullptr) {
   if (P.B == 0) return PSD_OK;
+  if (split_finalize(P.B, P.V, P.bonus != 0, ss)) return launch_finalize_split(P, P, 1, dtype, stream, ss);
   TimedLaunch timed(stream, 1);
   const int cl = fin_cluster_size(P.B);
   const unsigned units = static_cast<unsigned>(P.B);
@@ -367,7 +425,7 @@ int run_stage_locked(const psd_stage_args* a, StreamScratch* ss, int* status, cu
     rc = launch_rowstats(P, a->dtype, a->kernel_variant, a->cluster_size, stream);
     if (rc != PSD_OK) return rc;
   }
-  return launch_finalize(P, a->dtype, stream);
+  return launch_finalize(P, a->dtype, stream, ss);
 }
 
 int run_stage(const psd_stage_args* a) {
@@ -550,6 +608,8 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
   PS.stats2 = P2.stats;
   rc = launch_rowstats(PS, dtype, variant, 0, stream, policy == PSD_TWO_STAGE_FUSED_ROWS || policy == PSD_TWO_STAGE_AUTO);
   if (rc != PSD_OK) return rc;
+  if (a->mode_q == PSD_FUZZY && a->mode_t == PSD_FUZZY && split_finalize(2ll * B, V, P1.bonus != 0 || P2.bonus != 0, ss))
+    return launch_finalize_split(P1, P2, 2, dtype, stream, ss);
   {
     TimedLaunch timed(stream, 1);
     cudaError_t e;
@@ -1040,12 +1100,12 @@ int pyramidsd_release_stream(void* cuda_stream) {
     if (!e.used || e.stream != stream) continue;
     std::lock_guard<std::mutex> lock(e.mu);
     if (cudaStreamSynchronize(stream) != cudaSuccess) return PSD_ERR_CUDA;
-    void** owned[] = {&e.ws, reinterpret_cast<void**>(&e.status), &e.stage[0], &e.stage[1], &e.stage[2], &e.stage[3], &e.out4, &e.lm_ws};
+    void** owned[] = {&e.ws, reinterpret_cast<void**>(&e.status), &e.stage[0], &e.stage[1], &e.stage[2], &e.stage[3], &e.out4, &e.lm_ws, &e.draw};
     for (void** p : owned) {
       if (*p) cudaFree(*p);
       *p = nullptr;
     }
-    e.ws_bytes = e.out4_bytes = e.lm_ws_bytes = 0;
+    e.ws_bytes = e.out4_bytes = e.lm_ws_bytes = e.draw_bytes = 0;
     for (size_t& b : e.stage_bytes) b = 0;
     if (t_last_scratch == &e) { t_last_scratch = nullptr; t_last_status = nullptr; }
     e.used = false;

@@ -492,6 +492,9 @@ __device__ __forceinline__ V warp_sum(V v) { return warp_reduce<OpSum>(v); }
 template <typename T, int DIV, bool RS, bool TRI>
 __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cluster_kernel(const StageParams P, const ClusterGeom G) {
   static_assert(RS || !TRI, "row triples are streamed twice");
+  // a next launch that was made a programmatic dependent (the scan of the finalisation) may be scheduled from here
+  // on; it waits for this grid's end before it reads a statistic
+  asm volatile("griddepcontrol.launch_dependents;");
   extern __shared__ unsigned char smem_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   ClusterCtl* ctl = reinterpret_cast<ClusterCtl*>(ring + static_cast<size_t>(kClSlots) * kClSlotBytes);
