@@ -330,21 +330,24 @@ int pyramidsd_row_uniforms(uint64_t philox_seed, uint64_t offset, int n_rows, fl
 size_t pyramidsd_workspace_bytes(int B, int K, int V, psd_dtype dtype);
 
 /* How the two-stage calls schedule their launches (per host thread; every schedule returns the same results, bit
- * for bit: all of them cut a row over the CTAs of a cluster the same way).
- *   PSD_TWO_STAGE_FUSED     two launches: one statistics launch over the B*K_d stage-1 row pairs and all B*K_q
- *                           stage-2 row pairs, one finalisation launch for both stages. Best when windows are
+ * for bit: all of them cut a row over the CTAs of a cluster the same way). A "finalisation" below is one launch (a
+ * cluster of CTAs per sequence), or, for batches that fill the GPU on calls that use the library's own scratch,
+ * three small launches that hand over to one another (accept scan; the tile totals of every draw, spread over all
+ * SMs; pick and descent) -- again with the same bits.
+ *   PSD_TWO_STAGE_FUSED     two steps: one statistics launch over the B*K_d stage-1 row pairs and all B*K_q
+ *                           stage-2 row pairs, one finalisation for both stages. Best when windows are
  *                           (nearly) full, as in the paper's pipeline, which keeps drafting until the window holds
  *                           K_q tokens (Fig. 1).
- *   PSD_TWO_STAGE_SEPARATE  four launches, stage by stage; stage 2 then skips the rows beyond each window, which
+ *   PSD_TWO_STAGE_SEPARATE  four steps, stage by stage; stage 2 then skips the rows beyond each window, which
  *                           wins when acceptance is low and windows are short.
  *   PSD_TWO_STAGE_AUTO      (the default) the library chooses between the two per call. Stage 1 also leaves each
  *                           sequence's window length in a small host-mapped buffer (no copy, no synchronisation);
  *                           a later call with the same B and K_q on this device reads whatever lengths are there
  *                           -- those of a recent call -- and runs stage by stage when the unfilled part of the
  *                           windows is more than a tenth of all rows and the batch has at least 1024 rows, else
- *                           in two launches, over row triples where they apply (FUSED_ROWS below). The first call
- *                           of a shape runs in two launches.
- *   PSD_TWO_STAGE_FUSED_ROWS two launches like FUSED, but positions k < K_q are walked as row triples (draft,
+ *                           in two steps, over row triples where they apply (FUSED_ROWS below). The first call
+ *                           of a shape runs in two steps.
+ *   PSD_TWO_STAGE_FUSED_ROWS two steps like FUSED, but positions k < K_q are walked as row triples (draft,
  *                           qualifier, target): the qualifier row, which stage 1 uses as its large model and
  *                           stage 2 as its small one (Fig. 1), is read, widened and normalised once --
  *                           (2 K_d + K_q) V s bytes instead of 2 (K_d + K_q) V s. Applies where the statistics
