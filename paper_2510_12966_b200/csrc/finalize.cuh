@@ -515,18 +515,20 @@ constexpr int kScanWarps = 4;
 struct DrawRecord {
   int L;
   float u2, m2l, l2sl, m2s, l2ss, resid;
-  int pad;
+  int unit;
 };
 
 struct DrawScratch {
   int* need;            // [units] 1: the unit draws
-  int* list;            // [0]: number of drawing units; [1 + d]: the d-th of them, in unit order
-  DrawRecord* record;   // [units]
-  double* tile_total;   // [units][kDrawMaxTiles]
+  int* count;           // [0]: number of drawing units
+  DrawRecord* record;   // [units] by unit, written by the scan
+  DrawRecord* drawn;    // [d]: the record of the d-th drawing unit (in unit order), gathered by the tile launch so
+                        // that the pick launch finds all it needs at addresses it knows from its block index
+  double* tile_total;   // [d][kDrawMaxTiles]
 };
 
 __host__ __device__ inline size_t draw_scratch_bytes(long long units) {
-  return static_cast<size_t>(units) * (2 * sizeof(int) + sizeof(DrawRecord) + kDrawMaxTiles * sizeof(double)) + 256;
+  return static_cast<size_t>(units) * (sizeof(int) + 2 * sizeof(DrawRecord) + kDrawMaxTiles * sizeof(double)) + 256;
 }
 
 // The three launches may start while the launch before them drains; they read nothing of it before this.
@@ -582,7 +584,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) finalize_scan_kernel(const St
     ds.need[unit] = draw ? 1 : 0;
     if (draw) {
       DrawRecord r;
-      r.L = o.L; r.u2 = o.u2; r.m2l = o.m2l; r.l2sl = o.l2sl; r.m2s = o.m2s; r.l2ss = o.l2ss; r.resid = o.resid; r.pad = 0;
+      r.L = o.L; r.u2 = o.u2; r.m2l = o.m2l; r.l2sl = o.l2sl; r.m2s = o.m2s; r.l2ss = o.l2ss; r.resid = o.resid; r.unit = unit;
       ds.record[unit] = r;
     } else {
       write_results(second ? P2 : P1, b, o.L, next);
@@ -623,7 +625,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_tiles_kernel(const Stage
   __shared__ TileShared<T> S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int units = n_stages * P1.B;
-  // every CTA builds the same list of drawing units, in unit order; CTA 0 leaves it for the pick launch
+  // every CTA builds the same list of drawing units, in unit order
   if (tid == 0) S.n_list = 0;
   wait_for_previous_launch();
   release_next_launch();
@@ -639,7 +641,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_tiles_kernel(const Stage
     if (need) {
       const int pos = before + __popc(m & ((1u << lane) - 1u));
       S.list[pos] = static_cast<unsigned short>(unit);
-      if (blockIdx.x == 0) ds.list[1 + pos] = unit;
+      if (pos % static_cast<int>(gridDim.x) == static_cast<int>(blockIdx.x)) ds.drawn[pos] = ds.record[unit];   // for the pick launch
     }
     __syncthreads();
     if (tid == 0) {
@@ -650,7 +652,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_tiles_kernel(const Stage
     __syncthreads();
   }
   const int n_list = S.n_list;
-  if (blockIdx.x == 0 && tid == 0) ds.list[0] = n_list;
+  if (blockIdx.x == 0 && tid == 0) ds.count[0] = n_list;
   if (n_list == 0) return;
   const int n_tiles = (P1.V + kFinTile - 1) / kFinTile;
   const int items = n_list * n_tiles;   // <= kDrawMaxUnits * kDrawMaxTiles
@@ -659,10 +661,11 @@ __global__ void __launch_bounds__(kFinThreads) finalize_tiles_kernel(const Stage
     const int nb = min(kFinBatch, (items - first + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x));
     if (tid < nb) {
       const int item = first + tid * static_cast<int>(gridDim.x);
-      const int unit = S.list[item / n_tiles], j = item % n_tiles;
+      const int d = item / n_tiles, j = item % n_tiles;
+      const int unit = S.list[d];
       const bool second = (n_stages == 2) && (unit & 1);
       S.row[tid] = draw_row<T>(second ? P2 : P1, (n_stages == 2) ? unit >> 1 : unit, ds.record[unit]);
-      S.out[tid] = ds.tile_total + unit * kDrawMaxTiles + j;
+      S.out[tid] = ds.tile_total + d * kDrawMaxTiles + j;
       S.i_base[tid] = j * kFinTile;
     }
     __syncthreads();
@@ -711,16 +714,24 @@ __global__ void __launch_bounds__(kFinThreads) finalize_pick_kernel(const StageP
   __shared__ FinShared S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   wait_for_previous_launch();
-  const int n_list = ds.list[0];
   const int n_tiles = (P1.V + kFinTile - 1) / kFinTile;
+  // the first draw's record and totals are asked for together with the count (stale but allocated memory if this
+  // CTA has no draw)
+  const bool may = static_cast<int>(blockIdx.x) < n_stages * P1.B;
+  DrawRecord rec = may ? ds.drawn[blockIdx.x] : DrawRecord{};
+  double tt = (may && tid < n_tiles) ? ds.tile_total[blockIdx.x * kDrawMaxTiles + tid] : 0.0;
+  const int n_list = ds.count[0];
   for (int d = blockIdx.x; d < n_list; d += gridDim.x) {
-    const int unit = ds.list[1 + d];
+    if (d != static_cast<int>(blockIdx.x)) {
+      rec = ds.drawn[d];
+      if (tid < n_tiles) tt = ds.tile_total[d * kDrawMaxTiles + tid];
+    }
+    const int unit = rec.unit;
     const bool second = (n_stages == 2) && (unit & 1);
     const StageParams& P = second ? P2 : P1;
     const int b = (n_stages == 2) ? unit >> 1 : unit;
-    const DrawRecord rec = ds.record[unit];
     RowView<T> row = draw_row<T>(P, b, rec);
-    if (tid < n_tiles) S.tile_total[tid] = ds.tile_total[unit * kDrawMaxTiles + tid];
+    if (tid < n_tiles) S.tile_total[tid] = tt;
     if (tid == 0) S.sh_u2 = rec.u2;
     __syncthreads();
     if (tid == 0) pick_tile(S, n_tiles, row.from_large);

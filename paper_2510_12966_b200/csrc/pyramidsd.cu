@@ -304,8 +304,10 @@ int launch_finalize_split(const StageParams& P1, const StageParams& P2, int n_st
   base += static_cast<size_t>(units) * psd::kDrawMaxTiles * sizeof(double);
   d.record = reinterpret_cast<psd::DrawRecord*>(base);
   base += static_cast<size_t>(units) * sizeof(psd::DrawRecord);
+  d.drawn = reinterpret_cast<psd::DrawRecord*>(base);
+  base += static_cast<size_t>(units) * sizeof(psd::DrawRecord);
   d.need = reinterpret_cast<int*>(base);
-  d.list = d.need + units;   // 1 + units entries at most: the 256 spare bytes hold the count
+  d.count = d.need + units;   // in the 256 spare bytes
   int sms = psd::cluster_sm_count();
   if (sms <= 0) sms = 148;
   const unsigned scan_ctas = static_cast<unsigned>((units + psd::kScanWarps - 1) / psd::kScanWarps);
