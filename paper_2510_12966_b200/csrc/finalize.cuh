@@ -31,6 +31,11 @@ __device__ __forceinline__ void fin_remote_store(double* local, unsigned rank, d
   asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
 }                               // tiles summed between two CTA-wide barriers
 
+// A finalisation launch may start while the launch before it drains; it reads nothing of that launch before this.
+__device__ __forceinline__ void wait_for_previous_launch() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next launch on the stream, if it was launched as a dependent, be scheduled from here on.
+__device__ __forceinline__ void release_next_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 template <typename T>
 struct RowView {
   const T* large;
@@ -445,6 +450,7 @@ __device__ __forceinline__ void finalize_sequence(const StageParams& P, const in
 template <typename T, int CL>
 __global__ void __launch_bounds__(kFinThreads, 1) finalize_kernel(const StageParams P) {
   __shared__ FinShared S;
+  wait_for_previous_launch();
   finalize_sequence<T, CL>(P, blockIdx.x / CL, S);
   if (CL > 1) fin_cluster_sync();   // nobody leaves while a peer may still post tile sums into its shared memory
 }
@@ -455,6 +461,7 @@ __global__ void __launch_bounds__(kFinThreads, 1) finalize_kernel(const StagePar
 template <typename T, int CL>
 __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_kernel(const StageParams P1, const StageParams P2) {
   __shared__ FinShared S;
+  wait_for_previous_launch();
   finalize_sequence<T, CL>(P1, blockIdx.x / CL, S);
   __threadfence();
   __syncthreads();
@@ -471,6 +478,7 @@ __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_kernel(const Sta
 template <typename T, int CL>
 __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_split_kernel(const StageParams P1, const StageParams P2) {
   __shared__ FinShared S;
+  wait_for_previous_launch();
   __shared__ int sh_L1, sh_n2;
   const int unit = blockIdx.x / CL, b = unit >> 1;
   if ((unit & 1) == 0) {
@@ -530,11 +538,6 @@ struct DrawScratch {
 __host__ __device__ inline size_t draw_scratch_bytes(long long units) {
   return static_cast<size_t>(units) * (sizeof(int) + 2 * sizeof(DrawRecord) + kDrawMaxTiles * sizeof(double)) + 256;
 }
-
-// The three launches may start while the launch before them drains; they read nothing of it before this.
-__device__ __forceinline__ void wait_for_previous_launch() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// Lets the next launch on the stream, if it was launched as a dependent, be scheduled from here on.
-__device__ __forceinline__ void release_next_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
 
 // The window length and token source of the stage-2 half of a fuzzy pyramid: stage 1's threshold scan again.
 __device__ __forceinline__ void stage1_prefix(const StageParams& P1, const int K2, const int b, const int lane, int* L1, int* n2) {

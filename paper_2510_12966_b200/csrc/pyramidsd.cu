@@ -245,13 +245,17 @@ cudaError_t launch_fin_clusters(Kernel kernel, int cl, unsigned units, cudaStrea
   cfg.blockDim = dim3(psd::kFinThreads);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = static_cast<unsigned>(cl);
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  // a programmatic dependent of the statistics launch before it: its CTAs may be placed while that launch drains,
+  // and wait (griddepcontrol.wait, their first instruction) for its end before they read a statistic
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
