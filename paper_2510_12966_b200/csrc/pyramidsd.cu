@@ -272,11 +272,13 @@ int fin_cluster_size(long long units) {
    : (cl) == 2 ? launch_fin_clusters(psd::KERNEL<T, 2>, 2, units, stream, __VA_ARGS__)                      \
                : launch_fin_clusters(psd::KERNEL<T, 1>, 1, units, stream, __VA_ARGS__))
 
-// Whether a finalisation of `units` sequences (x stages) goes as three launches (scan, tile totals, pick): batches for
-// which the one-launch form would give a draw fewer than four CTAs, within the limits of the draw records.
+// Whether a finalisation of `units` sequences (x stages) goes as three launches (scan, tile totals, pick): batches of
+// 64 and more (measured: below that the one-launch form, four CTAs per sequence, is the faster one), within the
+// limits of the draw records.
+constexpr long long kSplitMinUnits = 64;
 bool split_finalize(long long units, int V, bool bonus, const StreamScratch* ss) {
   if (ss == nullptr || bonus) return false;
-  if (fin_cluster_size(units) == 4 || units > psd::kDrawMaxUnits) return false;
+  if (units < kSplitMinUnits || units > psd::kDrawMaxUnits) return false;
   return (V + psd::kFinTile - 1) / psd::kFinTile <= psd::kDrawMaxTiles;
 }
 
