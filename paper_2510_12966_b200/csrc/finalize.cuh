@@ -138,7 +138,9 @@ __device__ __forceinline__ ScanOut scan_unit(const StageParams& P, const int b, 
     const float nanf_ = __int_as_float(0x7fc00000);
     float px = nanf_, qx = nanf_;
     bool coin_ok = false;
-    if (!flags) {
+    // the token's two probabilities decide the coin flip; the threshold rule needs them only as outputs
+    const bool want_p = P.mode != kModeFuzzy || P.out_p_small_tok != nullptr || P.out_p_large_tok != nullptr;
+    if (!flags && want_p) {
       const long long off = static_cast<long long>(lane) * V + x;
       px = ex2_approx(fmaf(Elem<T>::load(large_seq, off), P.c, -st.m2_large) - st.l2s_large);
       qx = ex2_approx(fmaf(Elem<T>::load(small_seq, off), P.c, -st.m2_small) - st.l2s_small);
