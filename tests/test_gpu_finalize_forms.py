@@ -121,3 +121,53 @@ def test_three_launch_form_against_oracle(psd, oracle, wl, mode):
         assert rep["tie_resid"] <= K      # sequence 5's rows, whose residual single precision cannot tell from zero
         assert 0 < orc["accept_len"].sum() < B * K
     assert ties <= 4
+
+
+def test_three_launch_form_on_two_streams_from_two_threads(psd, wl):
+    """The draw records and tile totals belong to the stream a call runs on: two host threads, each on a stream of its
+    own, issue three-launch finalisations of different shapes back to back; every result equals the one the same call
+    gives alone."""
+    import threading
+    dev = torch.device("cuda:0")
+    cases = []
+    t = [x.to(dev) for x in wl.make_pyramid_inputs(48, 8, 4, 32768, "bf16", seed=131, sigma_q=0.4, sigma_d=0.8)]
+    probe = psd.verify_ex(*t, 1e9, 1e9)
+    tau_q, tau_t = float(probe["div_q"].median()), float(probe["div_t"].median())
+    call_a = lambda **kw: psd.verify_ex(*t, tau_q, tau_t, psd.FUZZY, psd.FUZZY, 2, 8, schedule=psd.TWO_STAGE_FUSED, **kw)
+    s = [x.to(dev) for x in wl.make_stage_inputs(100, 5, 20000, "f32", seed=132, sigma=0.6)]
+    call_b = lambda **kw: psd.verify_stage_ex(*s, 0.03, psd.STRICT, 4, 1, **kw)
+    for call in (call_a, call_b):
+        n0 = psd.launch_count()
+        ref = call()
+        torch.cuda.synchronize()
+        assert psd.launch_count() - n0 == 4 and int((ref["next_token"] >= 0).sum()) > 0
+        cases.append((call, ref))
+    errors = []
+
+    def worker(idx):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            call, ref = cases[idx]
+            with torch.cuda.stream(stream):
+                for it in range(40):
+                    out = call(stream=stream)
+                    if it % 8 == 7:
+                        stream.synchronize()
+                        for k, v in ref.items():
+                            if torch.is_tensor(v):
+                                x, y = (v.view(torch.int32), out[k].view(torch.int32)) if v.dtype == torch.float32 else (v, out[k])
+                                if not torch.equal(x, y):
+                                    errors.append((idx, it, k))
+                stream.synchronize()
+                if psd.last_status() != psd.OK:
+                    errors.append((idx, "status"))
+        except Exception as e:   # noqa: BLE001
+            errors.append((idx, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors[:5]
