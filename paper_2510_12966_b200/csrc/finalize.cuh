@@ -296,7 +296,7 @@ __device__ __forceinline__ void descend_tile(const RowView<T>& row, FinShared& S
 // are split between them and exchanged through distributed shared memory, and the CTA that owns the chosen
 // tile finishes the draw and writes the results. `nv_given` >= 0 replaces P.n_valid[b], and `tokens_given`
 // (with `n_given` entries; positions beyond it count as token 0) replaces P.tokens for this sequence: that
-// is how stage 2 of a fuzzy pyramid runs without waiting for stage 1's draw.
+// is how a stage 2 that accepts by the threshold rule runs without waiting for stage 1's draw.
 template <typename T, int CL>
 __device__ __forceinline__ void finalize_sequence(const StageParams& P, const int b, FinShared& S, const int nv_given = -1,
                                                   const int32_t* tokens_given = nullptr, const int n_given = 0) {
@@ -472,11 +472,23 @@ __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_kernel(const Sta
   if (CL > 1) fin_cluster_sync();
 }
 
-// Fuzzy mode only: the stage-2 half of the pyramid does not need stage 1's drawn token -- the accept bits
-// depend on the divergences alone, and the window length follows from stage 1's accept scan -- so the two
-// stages of a sequence run side by side, one cluster each. Cluster 2b is stage 1 (it also writes the
-// window); cluster 2b+1 repeats stage 1's cheap scan to get the window length, then runs stage 2 on the
-// accepted draft prefix.
+// The window of the stage-2 half of a pyramid whose stage 2 uses the threshold rule, by one full warp: stage 1's
+// accept scan again (whatever its rule: the coin flips are functions of the row index), without its outputs. The
+// window holds the accepted prefix and, unless everything was accepted or the rejected row has no distribution, the
+// correction token; which token that is does not matter to a threshold test.
+template <typename T>
+__device__ __forceinline__ void stage1_prefix(const StageParams& P1, const int K2, const int b, const int lane, int* L1, int* n2) {
+  const ScanOut o = scan_unit<T>(P1, b, lane, false, -1, nullptr, 0);
+  const int has_next = (o.L < o.nv && !(o.flags & (kFlagSmallNonfinite | kFlagLargeNonfinite))) ? 1 : 0;
+  *L1 = o.L;
+  *n2 = min(o.L + has_next, K2);
+}
+
+// Stage 2 by the threshold rule (stage 1 by any rule, the assisted variant of Sec. 3.4 among them): the stage-2
+// half of the pyramid does not need stage 1's drawn token -- its accept bits depend on the divergences alone, and
+// the window length follows from stage 1's accept scan -- so the two stages of a sequence run side by side, one
+// cluster each. Cluster 2b is stage 1 (it also writes the window); cluster 2b+1 repeats stage 1's cheap scan to
+// get the window length, then runs stage 2 on the accepted draft prefix.
 template <typename T, int CL>
 __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_split_kernel(const StageParams P1, const StageParams P2) {
   __shared__ FinShared S;
@@ -487,21 +499,9 @@ __global__ void __launch_bounds__(kFinThreads) finalize_pyramid_split_kernel(con
     finalize_sequence<T, CL>(P1, b, S);
   } else {
     if (threadIdx.x < 32) {
-      const int lane = threadIdx.x, K = P1.K;
-      bool acc = true;
-      int flags = 0;
-      if (lane < K) {
-        const RowStats st = P1.stats[b * K + lane];
-        const int x = P1.tokens[b * K + lane];
-        flags = st.flags | ((x < 0 || x >= P1.V) ? kFlagTokenRange : 0);
-        acc = (st.div <= P1.threshold) && !flags;
-      }
-      const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
-      const int L1 = rejected ? (__ffs(rejected) - 1) : K;
-      const int flags_L = __shfl_sync(0xffffffffu, flags, min(L1, 31));
-      // a correction token follows the accepted prefix unless everything was accepted or the rejected row has no distribution
-      const int has_next = (L1 < K && !(flags_L & (kFlagSmallNonfinite | kFlagLargeNonfinite))) ? 1 : 0;
-      if (lane == 0) { sh_L1 = L1; sh_n2 = min(L1 + has_next, P2.K); }
+      int L1, n2;
+      stage1_prefix<T>(P1, P2.K, b, threadIdx.x, &L1, &n2);
+      if (threadIdx.x == 0) { sh_L1 = L1; sh_n2 = n2; }
     }
     __syncthreads();
     finalize_sequence<T, CL>(P2, b, S, sh_n2, P1.tokens + b * P1.K, sh_L1);
@@ -541,26 +541,7 @@ __host__ __device__ inline size_t draw_scratch_bytes(long long units) {
   return static_cast<size_t>(units) * (sizeof(int) + 2 * sizeof(DrawRecord) + kDrawMaxTiles * sizeof(double)) + 256;
 }
 
-// The window length and token source of the stage-2 half of a fuzzy pyramid: stage 1's threshold scan again.
-__device__ __forceinline__ void stage1_prefix(const StageParams& P1, const int K2, const int b, const int lane, int* L1, int* n2) {
-  const int K = P1.K;
-  bool acc = true;
-  int flags = 0;
-  if (lane < K) {
-    const RowStats st = P1.stats[b * K + lane];
-    const int x = P1.tokens[b * K + lane];
-    flags = st.flags | ((x < 0 || x >= P1.V) ? kFlagTokenRange : 0);
-    acc = (st.div <= P1.threshold) && !flags;
-  }
-  const unsigned rejected = ~__ballot_sync(0xffffffffu, acc);
-  *L1 = rejected ? (__ffs(rejected) - 1) : K;
-  const int flags_L = __shfl_sync(0xffffffffu, flags, min(*L1, 31));
-  // a correction token follows the accepted prefix unless everything was accepted or the rejected row has no distribution
-  const int has_next = (*L1 < K && !(flags_L & (kFlagSmallNonfinite | kFlagLargeNonfinite))) ? 1 : 0;
-  *n2 = min(*L1 + has_next, K2);
-}
-
-// Scan launch: unit = sequence (n_stages == 1) or 2 * sequence + stage (the side-by-side form of a fuzzy pyramid).
+// Scan launch: unit = sequence (n_stages == 1) or 2 * sequence + stage (the side-by-side form of a pyramid).
 template <typename T>
 __global__ void __launch_bounds__(kScanWarps * 32) finalize_scan_kernel(const StageParams P1, const StageParams P2, const int n_stages,
                                                                         const DrawScratch ds) {
@@ -576,7 +557,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) finalize_scan_kernel(const St
     o = scan_unit<T>(P1, b, lane, true, -1, nullptr, 0);
   } else {
     int L1, n2;
-    stage1_prefix(P1, P2.K, b, lane, &L1, &n2);
+    stage1_prefix<T>(P1, P2.K, b, lane, &L1, &n2);
     o = scan_unit<T>(P2, b, lane, true, n2, P1.tokens + b * P1.K, L1);
   }
   if (lane == 0) {

@@ -616,13 +616,13 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
   PS.stats2 = P2.stats;
   rc = launch_rowstats(PS, dtype, variant, 0, stream, policy == PSD_TWO_STAGE_FUSED_ROWS || policy == PSD_TWO_STAGE_AUTO);
   if (rc != PSD_OK) return rc;
-  if (a->mode_q == PSD_FUZZY && a->mode_t == PSD_FUZZY && split_finalize(2ll * B, V, P1.bonus != 0 || P2.bonus != 0, ss))
+  if (a->mode_t == PSD_FUZZY && split_finalize(2ll * B, V, P1.bonus != 0 || P2.bonus != 0, ss))
     return launch_finalize_split(P1, P2, 2, dtype, stream, ss);
   {
     TimedLaunch timed(stream, 1);
     cudaError_t e;
-    if (a->mode_q == PSD_FUZZY && a->mode_t == PSD_FUZZY) {
-      // threshold-only acceptance in both stages: stage 2 needs nothing of stage 1's drawn token, the stages run side by side
+    if (a->mode_t == PSD_FUZZY) {
+      // threshold rule in stage 2: it needs nothing of stage 1's drawn token, the stages run side by side
       const int cl = fin_cluster_size(2ll * B);
       if (dtype == PSD_F32) e = PSD_FIN_DISPATCH(finalize_pyramid_split_kernel, float, cl, 2u * B, stream, P1, P2);
       else e = PSD_FIN_DISPATCH(finalize_pyramid_split_kernel, __nv_bfloat16, cl, 2u * B, stream, P1, P2);

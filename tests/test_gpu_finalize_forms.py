@@ -8,6 +8,7 @@ import pytest
 import torch
 
 from parity_utils import compare_stage, gpu_stage_to_numpy, host_bits
+from test_gpu_pyramid_ex import check_pyramid_ex
 
 pytestmark = pytest.mark.gpu
 
@@ -72,7 +73,8 @@ def test_three_launches_equal_one_launch_single_stage(psd, wl, dtype, V):
     assert drew > 2 * B
 
 
-def test_three_launches_equal_one_launch_pyramid(psd, wl):
+@pytest.mark.parametrize("mode_q", [0, 1, 3])    # threshold, coin flip, assisted (PSD_A of Sec. 3.4 with stage 2 fuzzy)
+def test_three_launches_equal_one_launch_pyramid(psd, oracle, wl, mode_q):
     dev = torch.device("cuda:0")
     B, K_d, K_q, V = 60, 6, 4, 24576
     zd, zq, zt, tok = wl.make_pyramid_inputs(B, K_d, K_q, V, "bf16", seed=61, sigma_q=0.3, sigma_d=0.6)
@@ -85,9 +87,9 @@ def test_three_launches_equal_one_launch_pyramid(psd, wl):
     ws = torch.empty(psd.pyramid_workspace_bytes(B, K_d, K_q, V, psd.dtype_code(dd[0])), dtype=torch.uint8, device=dev)
     for schedule in (psd.TWO_STAGE_FUSED, psd.TWO_STAGE_FUSED_ROWS):
         n0 = psd.launch_count()
-        a = psd.verify_ex(*dd, tau_q, tau_t, psd.FUZZY, psd.FUZZY, 5, 9, schedule=schedule)
+        a = psd.verify_ex(*dd, tau_q, tau_t, mode_q, psd.FUZZY, 5, 9, schedule=schedule)
         n1 = psd.launch_count()
-        b = psd.verify_ex(*dd, tau_q, tau_t, psd.FUZZY, psd.FUZZY, 5, 9, schedule=schedule, workspace=ws)
+        b = psd.verify_ex(*dd, tau_q, tau_t, mode_q, psd.FUZZY, 5, 9, schedule=schedule, workspace=ws)
         n2 = psd.launch_count()
         torch.cuda.synchronize()
         assert psd.last_status() == 0
@@ -99,6 +101,14 @@ def test_three_launches_equal_one_launch_pyramid(psd, wl):
                     x, y = x.view(torch.int32), y.view(torch.int32)
                 assert torch.equal(x, y), k
         assert 0 < int(a["accept_len_q"].sum()) < B * K_d and int((a["next_token"] >= 0).sum()) > 0
+    # and against the oracle, without the two spoiled sequences' rows in the way of the helper's element-wise checks
+    keep = [i for i in range(B) if i not in (2, 7)]
+    sub = [t[keep].contiguous() for t in (zd, zq, zt, tok)]
+    out = psd.verify_ex(*[t.to(dev) for t in sub], tau_q, tau_t, mode_q, psd.FUZZY, 5, 9)
+    torch.cuda.synchronize()
+    ties, n, orc = check_pyramid_ex(oracle, gpu_stage_to_numpy(out), tuple(host_bits(t) for t in sub[:3]), sub[3].numpy(),
+                                    "bf16", mode_q, psd.FUZZY, tau_q, tau_t, 5, 9)
+    assert ties <= 3 and n >= len(keep) - 2
 
 
 @pytest.mark.parametrize("mode", [0, 1, 3])
