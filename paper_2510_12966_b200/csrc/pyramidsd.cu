@@ -573,9 +573,10 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
         ds->fill_Kq = K_q;
         ds->fill_calls = 0;
       }
-      // The stores into mapped host memory cost the finalisation kernel a few microseconds: while windows are full
-      // (two launches) the lengths are asked for on every sixteenth call only, stage by stage on every call.
-      if (separate || (ds->fill_calls++ % 16u) == 0u) fill_out = ds->fill_dev;
+      // The stores into mapped host memory cost the finalisation a few microseconds: the lengths are asked for on
+      // every sixteenth call while windows are full, on every fourth while the call runs stage by stage (which is
+      // how long a change of regime can go unnoticed).
+      if ((ds->fill_calls++ % (separate ? 4u : 16u)) == 0u) fill_out = ds->fill_dev;
     }
   }
   const int variant = a->kernel_variant;
