@@ -484,6 +484,11 @@ __device__ __forceinline__ void div_accumulate(const float2 (&xl)[N], const floa
 template <typename V>
 __device__ __forceinline__ V warp_sum(V v) { return warp_reduce<OpSum>(v); }
 
+// A next launch that was made a programmatic dependent of this one (the finalisation) may be scheduled once every
+// warp of every CTA has been here; it still waits for this grid's end before it reads a statistic. Every warp comes
+// here after it has traded its registers, so no CTA placed early can be in the way of that trade.
+__device__ __forceinline__ void release_dependent_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 // ---- the kernel -------------------------------------------------------------------------------------
 // RS = false: a CTA's slice of a row fits the ring and is copied in once. RS = true ("re-stream"): the slice is
 // larger than the ring (small clusters, which is what fills every SM of the device), so it is copied in
@@ -492,9 +497,6 @@ __device__ __forceinline__ V warp_sum(V v) { return warp_reduce<OpSum>(v); }
 template <typename T, int DIV, bool RS, bool TRI>
 __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cluster_kernel(const StageParams P, const ClusterGeom G) {
   static_assert(RS || !TRI, "row triples are streamed twice");
-  // a next launch that was made a programmatic dependent (the scan of the finalisation) may be scheduled from here
-  // on; it waits for this grid's end before it reads a statistic
-  asm volatile("griddepcontrol.launch_dependents;");
   extern __shared__ unsigned char smem_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   ClusterCtl* ctl = reinterpret_cast<ClusterCtl*>(ring + static_cast<size_t>(kClSlots) * kClSlotBytes);
@@ -581,6 +583,7 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
 
     if (is_a) {
       if (RS) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kClRegsA));
+      release_dependent_launch();
       constexpr int kVecStride = kClAWarps * 32 * 16;   // bytes between a lane's vectors
       // ================================ pass A ================================
       // A row is summed optimistically against one reference per model, taken from the warp's first
@@ -701,6 +704,7 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
     } else {
       // ================================ pass B ================================
       if (RS) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kClRegsB));
+      release_dependent_launch();
       constexpr int N = Pairs<T>::kN;
       constexpr int PSI = sizeof(T) == 2 ? kPsiDegBf16 : 7;
       constexpr int kVecStride = kClBWarps * 32 * 16;   // bytes between a lane's vectors
@@ -789,6 +793,7 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
     }
   } else if (warp == kClConsumerWarps || warp == kClConsumerWarps + 3) {
     if (RS) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kClRegsService));
+    release_dependent_launch();
     // ================================ loader ================================
     // One thread per ring: the whole ring, or (slice streamed twice) pass A's slots [0, RA) from this warp and
     // pass B's slots [RA, R) from the last warp. The two streams run freely; pass B's copy of a chunk is
@@ -871,6 +876,7 @@ __global__ void __launch_bounds__(RS ? kClThreadsRS : kClThreads, 1) rowstats_cl
     // first agent holds a(m) back until the second one has closed row m - kClDepth + 1.
     // A row triple carries a second 16-byte record through every step (third model / second pair).
     if (RS) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kClRegsService));
+    release_dependent_launch();
     const float inv_c = 1.f / P.c;
 
     auto event_a = [&](int n, bool tri) {
