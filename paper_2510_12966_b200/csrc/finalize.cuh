@@ -1,9 +1,11 @@
-// Finalisation kernel: one CTA per sequence. Warp 0 turns the per-row statistics into accept bits
-// (fuzzy threshold test of Sec. 3.1/3.2, or the standard-SD coin flip), a ballot gives the accepted
-// prefix length (Sec. 1), and, when a position was rejected, the whole CTA draws the correction token
-// from the residual max(0, p_large - p_small) (Sec. 3.4) — or from p_large in the assisted variant —
-// by a hierarchical inverse CDF in vocabulary order: tiles, then warps, then lanes, then elements,
-// each level picking the first child whose inclusive cumulative weight exceeds the remaining target.
+// Finalisation: a warp turns a sequence's per-row statistics into accept bits (fuzzy threshold test of
+// Sec. 3.1/3.2, or the standard-SD coin flip), a ballot gives the accepted prefix length (Sec. 1), and, when a
+// position was rejected, the correction token is drawn from the residual max(0, p_large - p_small) (Sec. 3.4) --
+// or from p_large in the assisted variant -- by a hierarchical inverse CDF in vocabulary order: tiles of 8192
+// indices, then warps, then lanes, then elements, each level picking the first child whose inclusive cumulative
+// weight exceeds the remaining target. Two forms share this code and return the same bits: one launch with a CTA
+// (or a cluster of CTAs) per sequence, and, for batches that fill the GPU, three small launches that spread the
+// tile totals of all draws over all SMs (second half of this file).
 #pragma once
 
 #include "common.cuh"
