@@ -15,6 +15,7 @@ stage-2 rows inside each sequence's window). Prints ONE JSON line on rank 0.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -152,10 +153,12 @@ def run_ours(args):
                 "rows": binding.TWO_STAGE_FUSED_ROWS}[args.two_stage]
     cfg, w = workload_from_name(args.workload)
     if args.batch > 0:
-        import dataclasses
         w = dataclasses.replace(w, B=args.batch, name=f"{w.name}[B={args.batch}]")
+    if args.tau_q is not None or args.tau_t is not None:
+        # other thresholds than the workload's (how the step depends on the share of rejected windows)
+        w = dataclasses.replace(w, tau_q=w.tau_q if args.tau_q is None else args.tau_q,
+                                tau_t=w.tau_t if args.tau_t is None else args.tau_t, name=f"{w.name}[tau overridden]")
     if args.logits_dtype and args.logits_dtype != w.dtype:
-        import dataclasses
         w = dataclasses.replace(w, dtype=args.logits_dtype, name=f"{w.name}[{args.logits_dtype}]")
     es = 2 if w.dtype == "bf16" else 4
 
@@ -424,7 +427,6 @@ def run_fused(args):
     binding.set_stream()
     w = workloads.CONFIGS[5]
     if args.vocab > 0:
-        import dataclasses
         w = dataclasses.replace(w, V=args.vocab, name=f"{w.name}[V={args.vocab}]")
     M = w.B * w.K_d
     h, w_t, z_q, tok = workloads.make_fused_inputs(w.B, w.K_d, w.V, w.d_model, seed=5000, sigma_q=w.sigma_q, device=dev)
@@ -435,7 +437,6 @@ def run_fused(args):
     div_kind = binding.DIV_KL if kl else binding.DIV_JS
     lm_mode = binding.ASSISTED if args.lmhead_mode == "assisted" else binding.FUZZY
     if args.lmhead_tau is not None:
-        import dataclasses
         w = dataclasses.replace(w, tau_t=args.lmhead_tau)
 
     def step(i):
@@ -638,6 +639,8 @@ def main():
     ap.add_argument("--lmhead-div", choices=["js", "kl"], default="js", help="divergence of the fused LM-head workload (cfg5)")
     ap.add_argument("--lmhead-mode", choices=["fuzzy", "assisted"], default="fuzzy", help="acceptance mode of cfg5")
     ap.add_argument("--lmhead-tau", type=float, default=None, help="threshold of cfg5 (default: the workload's)")
+    ap.add_argument("--tau-q", type=float, default=None, help="override the qualifier-stage threshold of cfg2-cfg4")
+    ap.add_argument("--tau-t", type=float, default=None, help="override the target-stage threshold of cfg2-cfg4")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
