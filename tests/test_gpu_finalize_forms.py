@@ -181,3 +181,51 @@ def test_three_launch_form_on_two_streams_from_two_threads(psd, wl):
     for th in threads:
         th.join()
     assert not errors, errors[:5]
+
+
+def test_three_launch_form_replayed_from_a_cuda_graph(psd, wl):
+    """The statistics launch and the three dependent finalisation launches captured into a CUDA graph (after two
+    calls on the capturing stream, which size the library's buffers): replays on new contents of the same input
+    buffers return what eager calls return."""
+    dev = torch.device("cuda:0")
+    B, K_d, K_q, V = 40, 6, 4, 16384
+    rounds = [[x.to(dev) for x in wl.make_pyramid_inputs(B, K_d, K_q, V, "bf16", seed=140 + i, sigma_q=0.4, sigma_d=0.8)]
+              for i in range(3)]
+    probe = psd.verify_ex(*rounds[0], 1e9, 1e9)
+    tau_q, tau_t = float(probe["div_q"].median()), float(probe["div_t"].median())
+    psd.set_two_stage_policy(psd.TWO_STAGE_FUSED)
+    try:
+        eager = []
+        for r in rounds:
+            n0 = psd.launch_count()
+            eager.append(psd.verify(*r, tau_q, tau_t, psd.FUZZY, 11, 4))
+            torch.cuda.synchronize()
+            assert psd.launch_count() - n0 == 4
+        assert len({tuple(e["next_token"].tolist()) for e in eager}) == 3
+        bufs = [t.clone() for t in rounds[0]]
+        out = {k: torch.empty(B, dtype=torch.int32, device=dev) for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")}
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.stream(side):
+                psd.set_stream()
+                for _ in range(2):
+                    psd.verify(*bufs, tau_q, tau_t, psd.FUZZY, 11, 4, out=out)
+                side.synchronize()
+                with torch.cuda.graph(g, stream=side):
+                    psd.set_stream()
+                    psd.verify(*bufs, tau_q, tau_t, psd.FUZZY, 11, 4, out=out)
+        finally:
+            psd.set_stream()
+        for r, e in zip(rounds, eager):
+            for dst, src in zip(bufs, r):
+                dst.copy_(src)
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            for k in out:
+                assert torch.equal(out[k], e[k]), k
+    finally:
+        psd.set_two_stage_policy(psd.TWO_STAGE_DEFAULT)
+    assert psd.last_status() == 0
