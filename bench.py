@@ -171,13 +171,14 @@ def run_ours(args):
     outs = [{k: torch.empty(w.B, dtype=torch.int32, device=dev)
              for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")} for _ in range(n_bufs)]
     mode, seed = binding.FUZZY, 0
+    div_kind = {"js": binding.DIV_JS, "kl": binding.DIV_KL}[args.div]
 
     # every rank's B sequences are a slice of one global batch of world * B: the sequence base keeps each row's
     # random draws those of the global batch
     def step(i):
         zd, zq, zt, tok = rounds[i % n_bufs]
         binding.verify_ex(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, None, seed, 2 * i, seq_index_base=rank * w.B,
-                          schedule=schedule, want_rows=False, want_window=False, out=outs[i % n_bufs])
+                          schedule=schedule, div_kind=div_kind, want_rows=False, want_window=False, out=outs[i % n_bufs])
 
     def barrier():
         if world > 1:
@@ -232,7 +233,8 @@ def run_ours(args):
     # ---- acceptance rates and near ties of the rounds that were timed (one more call per round, with rows) ----
     acc = {"rows_q": 0, "acc_q": 0, "rows_t": 0, "acc_t": 0, "near_q": 0, "near_t": 0}
     for zd, zq, zt, tok in rounds:
-        o = binding.verify_ex(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, None, seed, 0, seq_index_base=rank * w.B, schedule=schedule)
+        o = binding.verify_ex(zd, zq, zt, tok, w.tau_q, w.tau_t, mode, None, seed, 0, seq_index_base=rank * w.B, schedule=schedule,
+                              div_kind=div_kind)
         torch.cuda.synchronize()
         nw = o["n_window"]
         inside = torch.arange(w.K_q, device=dev)[None, :] < nw[:, None]
@@ -290,7 +292,8 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "timed_regions": args.regions, "ms_per_step_min_max": [min(region_ms) / args.steps, max(region_ms) / args.steps],
             "config": {"workload": f"{w.name}: B={w.B} per GPU, V={w.V}, {w.dtype} logits, K_draft={w.K_d}, "
-                                   f"K_qual={w.K_q}, tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0, two-stage schedule {args.two_stage}",
+                                   f"K_qual={w.K_q}, tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0, two-stage schedule {args.two_stage}"
+                                   + (", divergence KL(large||small) in one pass" if args.div == "kl" else ""),
                        "logits_dtype": w.dtype, "arithmetic": "f32 (logits widened from %s)" % w.dtype,
                        "positions_per_step": n_pos / args.steps,
                        "acceptance": {"beta_qualifier_stage": acc["acc_q"] / max(acc["rows_q"], 1),
@@ -639,6 +642,9 @@ def main():
     ap.add_argument("--lmhead-div", choices=["js", "kl"], default="js", help="divergence of the fused LM-head workload (cfg5)")
     ap.add_argument("--lmhead-mode", choices=["fuzzy", "assisted"], default="fuzzy", help="acceptance mode of cfg5")
     ap.add_argument("--lmhead-tau", type=float, default=None, help="threshold of cfg5 (default: the workload's)")
+    ap.add_argument("--div", choices=["js", "kl"], default="js",
+                    help="divergence of cfg2-cfg4: Jensen-Shannon (the reading taken for the paper's Div) or KL(large||small), "
+                         "whose terms separate and whose statistics take one pass over the logits")
     ap.add_argument("--tau-q", type=float, default=None, help="override the qualifier-stage threshold of cfg2-cfg4")
     ap.add_argument("--tau-t", type=float, default=None, help="override the target-stage threshold of cfg2-cfg4")
     ap.add_argument("--no-e2e", action="store_true")

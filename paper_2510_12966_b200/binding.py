@@ -370,9 +370,10 @@ def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, p
                     B=None, K=None, V=None, n_valid=None, inv_temperature=0.0, div_kind=DIV_JS,
                     seq_stride_small=0, seq_stride_large=0, want_rows=True, workspace=None, stream=None,
                     kernel_variant=KERNEL_AUTO, cluster_size=0, raise_on_error=True, large_has_bonus_row=False,
-                    seq_index_base=0):
+                    seq_index_base=0, want_resid=None):
     """``pyramidsd_verify_stage_ex``: every option exposed. Returns a dict of device tensors (+ "status").
-    With ``large_has_bonus_row`` the large logits are [B, K + 1, V]."""
+    With ``large_has_bonus_row`` the large logits are [B, K + 1, V]. ``want_resid`` (default: as ``want_rows``) asks
+    for the rows' residual masses; without them the KL divergence takes the one-pass statistics kernel."""
     if B is None:
         B, K, V = logits_small.shape
         assert tuple(logits_large.shape) == (B, K + (1 if large_has_bonus_row else 0), V)
@@ -380,8 +381,9 @@ def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, p
     dev = logits_small.device
     out = {"accept_len": torch.empty(B, dtype=torch.int32, device=dev),
            "next_token": torch.empty(B, dtype=torch.int32, device=dev)}
+    want_resid = want_rows if want_resid is None else (want_resid and want_rows)
     if want_rows:
-        for k in ("div", "p_small_tok", "p_large_tok", "resid_mass"):
+        for k in ("div", "p_small_tok", "p_large_tok") + (("resid_mass",) if want_resid else ()):
             out[k] = torch.empty((B, K), dtype=torch.float32, device=dev)
         out["row_flags"] = torch.empty((B, K), dtype=torch.int32, device=dev)
     a = StageArgs()
@@ -402,7 +404,8 @@ def verify_stage_ex(logits_small, logits_large, tokens, threshold, mode=FUZZY, p
         a.out_div = out["div"].data_ptr()
         a.out_p_small_tok = out["p_small_tok"].data_ptr()
         a.out_p_large_tok = out["p_large_tok"].data_ptr()
-        a.out_resid_mass = out["resid_mass"].data_ptr()
+        if want_resid:
+            a.out_resid_mass = out["resid_mass"].data_ptr()
         a.out_row_flags = out["row_flags"].data_ptr()
     if workspace is not None:
         a.workspace = workspace.data_ptr()
@@ -445,7 +448,7 @@ def verify(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t,
 def verify_ex(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau_t, mode_q=FUZZY, mode_t=None,
               philox_seed=0, offset=0, *, seq_index_base=0, target_has_bonus_row=False, schedule=TWO_STAGE_DEFAULT,
               inv_temperature=0.0, div_kind=DIV_JS, want_rows=True, want_window=True, workspace=None, stream=None,
-              kernel_variant=KERNEL_AUTO, raise_on_error=True, out=None):
+              kernel_variant=KERNEL_AUTO, raise_on_error=True, out=None, want_resid=None):
     """``pyramidsd_verify_ex``: the two-stage pyramid with per-stage modes, a sequence base, per-row outputs, the
     window, a caller workspace and an explicit schedule. Returns a dict of device tensors (+ "status"). ``out`` may
     bring the four [B] int32 result tensors (keys accept_len_q, next_token_q, accept_len, next_token)."""
@@ -473,8 +476,11 @@ def verify_ex(logits_draft, logits_qual, logits_target, draft_tokens, tau_q, tau
     a.target_has_bonus_row, a.schedule = (1 if target_has_bonus_row else 0), int(schedule)
     for k in ("accept_len_q", "next_token_q", "accept_len", "next_token"):
         setattr(a, "out_" + k, _dev_ptr(out[k], torch.int32, k))
+    want_resid = want_rows if want_resid is None else (want_resid and want_rows)
     if want_rows:
         for k, n in (("div_q", K_d), ("resid_q", K_d), ("div_t", K_q), ("resid_t", K_q)):
+            if k.startswith("resid") and not want_resid:
+                continue   # without residual masses the KL divergence takes the one-pass statistics kernel
             out[k] = torch.empty((B, n), dtype=torch.float32, device=dev)
             setattr(a, "out_" + k, out[k].data_ptr())
     if want_window:

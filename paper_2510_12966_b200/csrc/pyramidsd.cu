@@ -14,6 +14,7 @@
 #include "finalize.cuh"
 #include "rowstats_baseline.cuh"
 #include "rowstats_cluster.cuh"
+#include "rowstats_onepass.cuh"
 #include "lmhead_fused.cuh"
 
 namespace {
@@ -196,11 +197,25 @@ int check_launch() {
 }
 
 // Statistics pass for one stage: picks the kernel variant and launches it. `allow_triples`: a wrapper launch may
-// walk its rows as (draft, qualifier, target) triples where the geometry streams them twice.
+// walk its rows as (draft, qualifier, target) triples where the geometry streams them twice. `resid_wanted`: some
+// caller output takes the rows' residual masses (without them the KL divergence goes through the one-pass kernel).
+// `onepass`: 1 / 0 = the caller has decided for / against the one-pass kernel (a two-stage call decides once, on its
+// whole shape, so that all its schedules run the same arithmetic); -1 = decide here.
 int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_size, cudaStream_t stream,
-                    bool allow_triples = false) {
+                    bool allow_triples = false, bool resid_wanted = true, int onepass = -1) {
   const long long rows = static_cast<long long>(P.B) * P.K;
   if (rows == 0 && P.K2 == 0) return PSD_OK;
+  if (onepass < 0) onepass = (variant == PSD_KERNEL_AUTO && cluster_size == 0 && psd::onepass_applies(P, dtype, resid_wanted)) ? 1 : 0;
+  if (onepass == 1) {
+    TimedLaunch timed(stream, 0);
+    if (psd::launch_rowstats_onepass(P, dtype, stream) != 0) {
+      const cudaError_t e = cudaGetLastError();
+      std::fprintf(stderr, "pyramidsd: one-pass kernel launch failed: %s\n", cudaGetErrorString(e));
+      return PSD_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return check_launch();
+  }
   bool use_cluster = false;
   psd::ClusterGeom geom{};
   if (variant != PSD_KERNEL_BASELINE) {
@@ -415,7 +430,7 @@ cudaStream_t pick_stream(const psd_stage_args* a) {
 // Runs one stage with the scratch entry `ss` (held by the caller); `window_out`/`n_window_out`/`K_window` non-null
 // make the finalisation also build the stage-2 window of the wrapper.
 int run_stage_locked(const psd_stage_args* a, StreamScratch* ss, int* status, cudaStream_t stream, int32_t* window_out,
-                     int32_t* n_window_out, int K_window, int32_t* fill_out = nullptr) {
+                     int32_t* n_window_out, int K_window, int32_t* fill_out = nullptr, int onepass = -1) {
   int rc = PSD_OK;
   void* ws = a->workspace;
   if (ws == nullptr) {
@@ -430,7 +445,7 @@ int run_stage_locked(const psd_stage_args* a, StreamScratch* ss, int* status, cu
   P.fill_out = fill_out;
   P.fill_cap = kFillCap;
   if (a->K > 0) {
-    rc = launch_rowstats(P, a->dtype, a->kernel_variant, a->cluster_size, stream);
+    rc = launch_rowstats(P, a->dtype, a->kernel_variant, a->cluster_size, stream, false, P.out_resid_mass != nullptr, onepass);
     if (rc != PSD_OK) return rc;
   }
   return launch_finalize(P, a->dtype, stream, ss);
@@ -580,6 +595,8 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
     }
   }
   const int variant = a->kernel_variant;
+  const bool resid_any = a->out_resid_q != nullptr || a->out_resid_t != nullptr;
+  int onepass = 0;
   if (separate) {
     // stage by stage: stage 2's statistics run after stage 1 has fixed the windows and skip the rows beyond them.
     // Both launches take the cluster size the single-launch schedule would pick, so a row's vocabulary is
@@ -592,10 +609,11 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
       PS.K2 = K_q;
       psd::ClusterGeom g{};
       if (variant != PSD_KERNEL_BASELINE && psd::cluster_geometry(PS, dtype, 0, false, false, &g)) s1.cluster_size = s2.cluster_size = g.cs;
+      onepass = (variant == PSD_KERNEL_AUTO && psd::onepass_applies(PS, dtype, resid_any)) ? 1 : 0;
     }
-    rc = run_stage_locked(&s1, ss, status, stream, window, n_window, K_q, fill_out);
+    rc = run_stage_locked(&s1, ss, status, stream, window, n_window, K_q, fill_out, onepass);
     if (rc != PSD_OK) return rc;
-    return run_stage_locked(&s2, ss, status, stream, nullptr, nullptr, 0);
+    return run_stage_locked(&s2, ss, status, stream, nullptr, nullptr, 0, nullptr, onepass);
   }
   // Two launches for the whole pyramid. The statistics of both stages are independent of the stage-1
   // outcome (only the token looked up in a row and the window length depend on it), so one launch of
@@ -615,7 +633,8 @@ int verify_two_stage_locked(const psd_pyramid_args* a, StreamScratch* ss, int* s
   PS.seq_stride_large2 = P2.seq_stride_large;
   PS.K2 = K_q;
   PS.stats2 = P2.stats;
-  rc = launch_rowstats(PS, dtype, variant, 0, stream, policy == PSD_TWO_STAGE_FUSED_ROWS || policy == PSD_TWO_STAGE_AUTO);
+  rc = launch_rowstats(PS, dtype, variant, 0, stream, policy == PSD_TWO_STAGE_FUSED_ROWS || policy == PSD_TWO_STAGE_AUTO,
+                       P1.out_resid_mass != nullptr || P2.out_resid_mass != nullptr);
   if (rc != PSD_OK) return rc;
   if (a->mode_t == PSD_FUZZY && split_finalize(2ll * B, V, P1.bonus != 0 || P2.bonus != 0, ss))
     return launch_finalize_split(P1, P2, 2, dtype, stream, ss);
