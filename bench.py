@@ -303,7 +303,8 @@ def run_ours(args):
                        "l2_policy": "inputs larger than L2 (one round = %.0f MB), two rounds alternate" %
                                     ((2 * w.K_d + w.K_q) * w.B * w.V * es / 1e6),
                        "gb_per_s_whole_step": n_pos_all * row_bytes / (ms_total * 1e-3) / 1e9},
-            "roofline": {"bound": "hbm", "kernel": "rowstats (per-row softmax/divergence statistics)",
+            "roofline": {"bound": "hbm", "kernel": "rowstats (per-row softmax/divergence statistics%s)" %
+                                                   (", KL in one pass over the logits" if args.div == "kl" else ""),
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                          "bytes_counted": "2*V*s per verified row pair (the call made); the least a two-stage call can "
@@ -318,8 +319,9 @@ def run_ours(args):
             "gpu_launches": launches_all, "clocks": clocks,
         }
         # The same kernel against the special-function unit, its first ceiling with bf16 logits: four ex2 per
-        # index pair (two per pass), 16 results per clock and SM, 148 SMs at the sampled SM clock.
-        n_ex2 = 4.0 * rs_bytes / (2 * es)
+        # index pair (two per pass; two in all when KL takes one pass), 16 results per clock and SM, 148 SMs at the
+        # sampled SM clock.
+        n_ex2 = (2.0 if args.div == "kl" else 4.0) * rs_bytes / (2 * es)   # KL in one pass: one ex2 per index and model
         xu_peak = 16.0 * 148 * (clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0) * 1e6
         line["roofline"]["special_function_unit"] = {
             "achieved": n_ex2 / (ms_rs * 1e-3) if ms_rs > 0 else 0.0, "peak": xu_peak, "unit": "ex2/s",
@@ -341,7 +343,8 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, rounds)
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
-        traffic = read_profile_traffic(w, "pairs" if args.two_stage == "fused" else "rows") if stats_per_step == 1 else None
+        form = "kl" if args.div == "kl" else ("pairs" if args.two_stage == "fused" else "rows")
+        traffic = read_profile_traffic(w, form) if stats_per_step == 1 else None
         if traffic is not None:
             line["roofline"]["traffic"] = traffic
         print(json.dumps(line))
