@@ -65,6 +65,13 @@ typedef enum {
   PSD_ASSISTED = 3           /* strict acceptance; on rejection draw from p_large itself (Sec. 3.4) */
 } psd_mode;
 
+/* The divergence `Div` of Sec. 3.1, which the paper leaves open ("a divergence measure"): Jensen-Shannon in nats
+ * (the default: bounded by ln 2, so the paper's thresholds 0.2 .. 0.5 mean something), total variation, or
+ * KL(large || small). The terms of KL separate -- sum_i p_i (log p_i - log q_i) needs the normalisers only as two
+ * numbers at the end -- so a call with PSD_DIV_KL that asks for no per-row residual masses (out_resid_mass, or
+ * out_resid_q / out_resid_t, NULL) and has at least one row per SM takes both softmaxes and the divergence in ONE
+ * pass over the logits: half the exponentials of the other kinds and every byte read once, which on bf16 logits
+ * is the difference between the special-function unit and HBM as the bound. */
 typedef enum { PSD_DIV_JS = 0, PSD_DIV_TV = 1, PSD_DIV_KL = 2 } psd_div_kind;
 
 typedef enum {
@@ -113,7 +120,7 @@ typedef struct psd_stage_args {
   float* out_div;                /* [B, K] device or NULL */
   float* out_p_small_tok;        /* [B, K] device or NULL */
   float* out_p_large_tok;        /* [B, K] device or NULL */
-  float* out_resid_mass;         /* [B, K] device or NULL */
+  float* out_resid_mass;         /* [B, K] device or NULL (NULL lets PSD_DIV_KL take one pass: see psd_div_kind) */
   int32_t* out_row_flags;        /* [B, K] device or NULL */
   void* workspace;               /* device, >= pyramidsd_workspace_bytes(B, K, V, dtype), 256-byte aligned; NULL = library-owned */
   size_t workspace_bytes;
