@@ -38,7 +38,9 @@ def statistics_ms(psd, call):
     return out, ms, n
 
 
-@pytest.mark.parametrize("dtype,V,B,K", [("f32", 4100, 40, 4), ("bf16", 8200, 30, 5), ("bf16", 50264, 20, 8), ("f32", 32000, 38, 4)])
+# the last two shapes give every CTA eight and four rows (the partial buffers and their barriers go round several times)
+@pytest.mark.parametrize("dtype,V,B,K", [("f32", 4100, 40, 4), ("bf16", 8200, 30, 5), ("bf16", 50264, 20, 8), ("f32", 32000, 38, 4),
+                                         ("bf16", 4096, 150, 8), ("f32", 6000, 100, 6)])
 def test_one_pass_against_oracle(psd, oracle, wl, dtype, V, B, K):
     dev = torch.device("cuda:0")
     zs, zl, tok = wl.make_stage_inputs(B, K, V, dtype, seed=600 + V, sigma=0.6)
@@ -143,3 +145,31 @@ def test_one_pass_in_every_schedule_of_the_two_stage_call(psd, oracle, wl, dtype
     assert np.array_equal(gpu["accept_len"][same], orc["accept_len"][same])
     assert (gpu["next_token"][same] == orc["next_token"][same]).sum() >= same.sum() - 1
     assert 0 < orc["accept_len_q"].sum() < B * K_d
+
+
+def test_full_size_config3_with_kl_sampled(psd, oracle, wl):
+    """The launch configuration `bench.py --div kl` times (B=64, V=128256, K=16/8, bf16), checked on sampled sequences:
+    the oracle runs them with their indices in the batch, so the coin flips and draws are those of the full call."""
+    dev = torch.device("cuda:0")
+    zd, zq, zt, tok = wl.workload_inputs(3, 0, device="cpu")
+    dd = [t.to(dev) for t in (zd, zq, zt, tok)]
+    probe = psd.verify_ex(*dd, 1e9, 1e9, div_kind=KL)
+    tau_q, tau_t = float(probe["div_q"].median()), float(probe["div_t"].median())
+    psd.kernel_timing_begin()
+    out = psd.verify_ex(*dd, tau_q, tau_t, 0, 0, 0, 4, div_kind=KL, want_resid=False)
+    torch.cuda.synchronize()
+    ms, n, _, _ = psd.kernel_timing_end()
+    assert psd.last_status() == 0 and n == 1
+    gpu = gpu_stage_to_numpy(out)
+    ids = np.array([0, 17, 40, 63])
+    sub = [host_bits(t[ids]) for t in (zd, zq, zt)]
+    orc = oracle.verify(*sub, tok.numpy()[ids], np.float32(tau_q), np.float32(tau_t), 0, 0, 4, div_kind=KL, n_threads=8, seq_ids=ids)
+    o1 = oracle.verify_stage(sub[0], sub[1], tok.numpy()[ids], np.float32(tau_q), 0, 0, 4, div_kind=KL, n_threads=8, seq_ids=ids)
+    assert np.abs(gpu["div_q"][ids] - o1["div"]).max() <= TOL["bf16"]["val"]
+    near = np.abs(o1["div"] - tau_q).min() < 1e-4
+    if not near:
+        assert np.array_equal(gpu["accept_len_q"][ids], orc["accept_len_q"])
+        same = gpu["next_token_q"][ids] == orc["next_token_q"]
+        assert same.sum() >= len(ids) - 1
+        assert np.array_equal(gpu["accept_len"][ids][same], orc["accept_len"][same])
+    assert 0 < gpu["accept_len_q"].sum() < 64 * 16
