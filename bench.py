@@ -342,6 +342,38 @@ def run_ours(args):
             "psd_tokens_per_s": binding.model_psd_throughput(b_qd, w.K_d, args.v_draft, args.v_qual, b_tq, w.K_q, args.v_target)}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w, rounds)
+        if world == 1 and args.div == "js" and w.B * (w.K_d + w.K_q) >= 148:
+            # beside the line: the same workload with the KL divergence, whose statistics take one pass over the logits
+            # (thresholds 2.0 / 1.0, under which about the same rows are accepted as with JS at the workload's own)
+            kl_tau = (2.0, 1.0)
+
+            def kl_step(i):
+                zd, zq, zt, tok = rounds[i % n_bufs]
+                binding.verify_ex(zd, zq, zt, tok, kl_tau[0], kl_tau[1], mode, None, seed, 2 * i, schedule=schedule,
+                                  div_kind=binding.DIV_KL, want_rows=False, want_window=False, out=outs[i % n_bufs])
+            kl_steps = min(args.steps, 100)
+            for i in range(3):
+                kl_step(i)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(kl_steps):
+                kl_step(i)
+            e1.record()
+            torch.cuda.synchronize()
+            kl_ms = e0.elapsed_time(e1) / kl_steps
+            binding.kernel_timing_begin()
+            for i in range(kl_steps):
+                kl_step(i)
+            torch.cuda.synchronize()
+            kl_rs, kl_n, _, _ = binding.kernel_timing_end()
+            kl_pos = sum(positions_per_step(w, outs[i % n_bufs]) for i in range(2)) / 2.0
+            line["kl_divergence_one_pass"] = {
+                "tau_q": kl_tau[0], "tau_t": kl_tau[1], "ms_per_step": kl_ms, "positions_per_s": kl_pos / (kl_ms * 1e-3),
+                "rowstats_ms_per_launch": kl_rs / max(kl_n, 1), "rowstats_launches_per_step": kl_n / kl_steps,
+                "rowstats_gb_per_s": kl_pos * row_bytes * kl_steps / (kl_rs * 1e-3) / 1e9 if kl_rs > 0 else None,
+                "frac_of_hbm_peak": (kl_pos * row_bytes * kl_steps / (kl_rs * 1e-3) / 1e9 / peaks["hbm_gbs"]) if kl_rs > 0 else None,
+                "note": "not the line's metric: div_kind = KL(large||small) instead of the Jensen-Shannon reading of Div"}
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
         form = "kl" if args.div == "kl" else ("pairs" if args.two_stage == "fused" else "rows")
         traffic = read_profile_traffic(w, form) if stats_per_step == 1 else None
