@@ -341,7 +341,7 @@ def run_ours(args):
             "sd_tokens_per_s": binding.model_sd_throughput(b_tq, w.K_q, args.v_qual, args.v_target),
             "psd_tokens_per_s": binding.model_psd_throughput(b_qd, w.K_d, args.v_draft, args.v_qual, b_tq, w.K_q, args.v_target)}
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w, rounds)
+            line["cpu_baseline"] = cpu_baseline(w, rounds, 2 if args.div == "kl" else 0)
         if world == 1 and args.div == "js" and w.B * (w.K_d + w.K_q) >= 148:
             # beside the line: the same workload with the KL divergence, whose statistics take one pass over the logits
             # (thresholds 2.0 / 1.0, under which about the same rows are accepted as with JS at the workload's own)
@@ -587,7 +587,7 @@ def read_profile_traffic(w, form):
     return None if per_row is None else per_row * w.B * (w.K_d + w.K_q)   # rows of the fused statistics launch
 
 
-def cpu_baseline(w, rounds):
+def cpu_baseline(w, rounds, div_kind=0):
     """The CPU oracle, as it stands, on a bounded sample: the resident rounds of the workload (two rounds
     of B sequences each), one oracle call per round on all host cores."""
     import oracle
@@ -598,7 +598,8 @@ def cpu_baseline(w, rounds):
     for r in rounds:
         zd, zq, zt, tok = [workloads.to_host_bits(t) for t in r]
         t0 = time.perf_counter()
-        out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, n_threads=cores)
+        out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, div_kind=div_kind,
+                            n_threads=cores)
         dt += time.perf_counter() - t0
         n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
         pos += w.B * w.K_d + int(n2.sum())
@@ -606,7 +607,7 @@ def cpu_baseline(w, rounds):
     nb = min(4, w.B)
     zd, zq, zt, tok = [workloads.to_host_bits(t[:nb]) for t in rounds[0]]
     t0 = time.perf_counter()
-    out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, n_threads=1)
+    out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 0, div_kind=div_kind, n_threads=1)
     dt1 = time.perf_counter() - t0
     pos1 = nb * w.K_d + int(np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0)).sum())
     return {"value": pos / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -625,6 +626,9 @@ def run_reference(args):
     from paper_2510_12966_b200 import workloads
     oracle.build()
     cfg, w = workload_from_name(args.workload)
+    if args.tau_q is not None or args.tau_t is not None:
+        w = dataclasses.replace(w, tau_q=w.tau_q if args.tau_q is None else args.tau_q,
+                                tau_t=w.tau_t if args.tau_t is None else args.tau_t, name=f"{w.name}[tau overridden]")
     seqs = args.cpu_seqs if args.cpu_seqs > 0 else w.B
     cores = os.cpu_count() or 1
     rounds = [workloads.workload_inputs(cfg, i, device="cpu", B=seqs) for i in range(2)]
@@ -633,7 +637,7 @@ def run_reference(args):
     def step(i):
         zd, zq, zt, tok = hosts[i % 2]
         out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 2 * i,
-                            n_threads=cores)
+                            div_kind=2 if args.div == "kl" else 0, n_threads=cores)
         n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
         return seqs * w.K_d + int(n2.sum())
 
