@@ -372,10 +372,15 @@ def run_ours(args):
                 "tau_q": kl_tau[0], "tau_t": kl_tau[1], "ms_per_step": kl_ms, "positions_per_s": kl_pos / (kl_ms * 1e-3),
                 "rowstats_ms_per_launch": kl_rs / max(kl_n, 1), "rowstats_launches_per_step": kl_n / kl_steps,
                 "rowstats_gb_per_s": kl_pos * row_bytes * kl_steps / (kl_rs * 1e-3) / 1e9 if kl_rs > 0 else None,
-                "frac_of_hbm_peak": (kl_pos * row_bytes * kl_steps / (kl_rs * 1e-3) / 1e9 / peaks["hbm_gbs"]) if kl_rs > 0 else None,
+                # on the bytes of the call made, 2*V*s per verified row pair, as the line's roofline.frac; and on the
+                # bytes actually read when one launch walks row triples (the qualifier's rows once)
+                "frac_of_hbm_peak_on_call_bytes": (kl_pos * row_bytes * kl_steps / (kl_rs * 1e-3) / 1e9 / peaks["hbm_gbs"]) if kl_rs > 0 else None,
+                "frac_of_hbm_peak_on_bytes_read": (kl_pos * row_bytes * kl_steps / (kl_rs * 1e-3) / 1e9 / peaks["hbm_gbs"] *
+                                                   ((2 * w.K_d + w.K_q) / (2.0 * (w.K_d + w.K_q))
+                                                    if (kl_n == kl_steps and args.two_stage in ("auto", "rows")) else 1.0)) if kl_rs > 0 else None,
                 "note": "not the line's metric: div_kind = KL(large||small) instead of the Jensen-Shannon reading of Div"}
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
-        form = "kl" if args.div == "kl" else ("pairs" if args.two_stage == "fused" else "rows")
+        form = ("kl_pairs" if args.two_stage == "fused" else "kl_rows") if args.div == "kl" else ("pairs" if args.two_stage == "fused" else "rows")
         traffic = read_profile_traffic(w, form) if stats_per_step == 1 else None
         if traffic is not None:
             line["roofline"]["traffic"] = traffic

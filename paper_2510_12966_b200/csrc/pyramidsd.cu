@@ -208,7 +208,7 @@ int launch_rowstats(const StageParams& P, int dtype, int variant, int cluster_si
   if (onepass < 0) onepass = (variant == PSD_KERNEL_AUTO && cluster_size == 0 && psd::onepass_applies(P, dtype, resid_wanted)) ? 1 : 0;
   if (onepass == 1) {
     TimedLaunch timed(stream, 0);
-    if (psd::launch_rowstats_onepass(P, dtype, stream) != 0) {
+    if (psd::launch_rowstats_onepass(P, dtype, stream, allow_triples) != 0) {
       const cudaError_t e = cudaGetLastError();
       std::fprintf(stderr, "pyramidsd: one-pass kernel launch failed: %s\n", cudaGetErrorString(e));
       return PSD_ERR_CUDA;
