@@ -86,9 +86,11 @@ def test_one_pass_is_the_kernel_that_runs(psd, wl):
     for _ in range(2):
         psd.verify_stage_ex(*d, 0.1, 0, 0, 0, div_kind=KL)
         psd.verify_stage_ex(*d, 0.1, 0, 0, 0, div_kind=KL, want_resid=False)
-    _, ms_two, n_two = statistics_ms(psd, lambda: psd.verify_stage_ex(*d, 0.1, 0, 0, 0, div_kind=KL))
-    _, ms_one, n_one = statistics_ms(psd, lambda: psd.verify_stage_ex(*d, 0.1, 0, 0, 0, div_kind=KL, want_resid=False))
-    assert n_two == 1 and n_one == 1 and ms_one < 0.75 * ms_two, (ms_one, ms_two)
+    two = [statistics_ms(psd, lambda: psd.verify_stage_ex(*d, 0.1, 0, 0, 0, div_kind=KL)) for _ in range(5)]
+    one = [statistics_ms(psd, lambda: psd.verify_stage_ex(*d, 0.1, 0, 0, 0, div_kind=KL, want_resid=False)) for _ in range(5)]
+    assert all(n == 1 for _, _, n in two + one)
+    ms_two, ms_one = min(ms for _, ms, _ in two), min(ms for _, ms, _ in one)      # the best of five: a shared GPU has hiccups
+    assert ms_one < 0.75 * ms_two, (ms_one, ms_two)
 
 
 def test_one_pass_late_logits_far_above_the_first_ones(psd, oracle, wl):
