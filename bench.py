@@ -171,7 +171,7 @@ def run_ours(args):
     outs = [{k: torch.empty(w.B, dtype=torch.int32, device=dev)
              for k in ("accept_len_q", "next_token_q", "accept_len", "next_token")} for _ in range(n_bufs)]
     mode, seed = binding.FUZZY, 0
-    div_kind = {"js": binding.DIV_JS, "kl": binding.DIV_KL}[args.div]
+    div_kind = {"js": binding.DIV_JS, "kl": binding.DIV_KL, "tv": binding.DIV_TV}[args.div]
 
     # every rank's B sequences are a slice of one global batch of world * B: the sequence base keeps each row's
     # random draws those of the global batch
@@ -293,7 +293,7 @@ def run_ours(args):
             "timed_regions": args.regions, "ms_per_step_min_max": [min(region_ms) / args.steps, max(region_ms) / args.steps],
             "config": {"workload": f"{w.name}: B={w.B} per GPU, V={w.V}, {w.dtype} logits, K_draft={w.K_d}, "
                                    f"K_qual={w.K_q}, tau_q={w.tau_q}, tau_t={w.tau_t}, fuzzy mode, Philox seed 0, two-stage schedule {args.two_stage}"
-                                   + (", divergence KL(large||small) in one pass" if args.div == "kl" else ""),
+                                   + {"js": "", "kl": ", divergence KL(large||small) in one pass", "tv": ", divergence total variation"}[args.div],
                        "logits_dtype": w.dtype, "arithmetic": "f32 (logits widened from %s)" % w.dtype,
                        "positions_per_step": n_pos / args.steps,
                        "acceptance": {"beta_qualifier_stage": acc["acc_q"] / max(acc["rows_q"], 1),
@@ -321,7 +321,7 @@ def run_ours(args):
         # The same kernel against the special-function unit, its first ceiling with bf16 logits: four ex2 per
         # index pair (two per pass; two in all when KL takes one pass), 16 results per clock and SM, 148 SMs at the
         # sampled SM clock.
-        n_ex2 = (2.0 if args.div == "kl" else 4.0) * rs_bytes / (2 * es)   # KL in one pass: one ex2 per index and model
+        n_ex2 = {"js": 4.0, "kl": 2.0, "tv": 3.0}[args.div] * rs_bytes / (2 * es)   # KL in one pass: one ex2 per index and model
         xu_peak = 16.0 * 148 * (clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0) * 1e6
         line["roofline"]["special_function_unit"] = {
             "achieved": n_ex2 / (ms_rs * 1e-3) if ms_rs > 0 else 0.0, "peak": xu_peak, "unit": "ex2/s",
@@ -341,7 +341,7 @@ def run_ours(args):
             "sd_tokens_per_s": binding.model_sd_throughput(b_tq, w.K_q, args.v_qual, args.v_target),
             "psd_tokens_per_s": binding.model_psd_throughput(b_qd, w.K_d, args.v_draft, args.v_qual, b_tq, w.K_q, args.v_target)}
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w, rounds, 2 if args.div == "kl" else 0)
+            line["cpu_baseline"] = cpu_baseline(w, rounds, {"js": 0, "tv": 1, "kl": 2}[args.div])
         if world == 1 and args.div == "js" and w.B * (w.K_d + w.K_q) >= 148:
             # beside the line: the same workload with the KL divergence, whose statistics take one pass over the logits
             # (thresholds 2.0 / 1.0, under which about the same rows are accepted as with JS at the workload's own)
@@ -380,7 +380,7 @@ def run_ours(args):
                                                     if (kl_n == kl_steps and args.two_stage in ("auto", "rows")) else 1.0)) if kl_rs > 0 else None,
                 "note": "not the line's metric: div_kind = KL(large||small) instead of the Jensen-Shannon reading of Div"}
         line["traffic_note"] = "roofline.traffic is filled from the ncu capture summarised under profiles/"
-        form = ("kl_pairs" if args.two_stage == "fused" else "kl_rows") if args.div == "kl" else ("pairs" if args.two_stage == "fused" else "rows")
+        form = ("kl_" if args.div == "kl" else "tv_" if args.div == "tv" else "") + ("pairs" if args.two_stage == "fused" else "rows")
         traffic = read_profile_traffic(w, form) if stats_per_step == 1 else None
         if traffic is not None:
             line["roofline"]["traffic"] = traffic
@@ -642,7 +642,7 @@ def run_reference(args):
     def step(i):
         zd, zq, zt, tok = hosts[i % 2]
         out = oracle.verify(zd, zq, zt, tok, np.float32(w.tau_q), np.float32(w.tau_t), oracle.FUZZY, 0, 2 * i,
-                            div_kind=2 if args.div == "kl" else 0, n_threads=cores)
+                            div_kind={"js": 0, "tv": 1, "kl": 2}[args.div], n_threads=cores)
         n2 = np.minimum(w.K_q, out["accept_len_q"] + (out["next_token_q"] >= 0))
         return seqs * w.K_d + int(n2.sum())
 
@@ -686,9 +686,10 @@ def main():
     ap.add_argument("--lmhead-div", choices=["js", "kl"], default="js", help="divergence of the fused LM-head workload (cfg5)")
     ap.add_argument("--lmhead-mode", choices=["fuzzy", "assisted"], default="fuzzy", help="acceptance mode of cfg5")
     ap.add_argument("--lmhead-tau", type=float, default=None, help="threshold of cfg5 (default: the workload's)")
-    ap.add_argument("--div", choices=["js", "kl"], default="js",
-                    help="divergence of cfg2-cfg4: Jensen-Shannon (the reading taken for the paper's Div) or KL(large||small), "
-                         "whose terms separate and whose statistics take one pass over the logits")
+    ap.add_argument("--div", choices=["js", "kl", "tv"], default="js",
+                    help="divergence of cfg2-cfg4: Jensen-Shannon (the reading taken for the paper's Div), KL(large||small), "
+                         "whose terms separate and whose statistics take one pass over the logits, or total variation "
+                         "(three ex2 per index pair instead of four)")
     ap.add_argument("--tau-q", type=float, default=None, help="override the qualifier-stage threshold of cfg2-cfg4")
     ap.add_argument("--tau-t", type=float, default=None, help="override the target-stage threshold of cfg2-cfg4")
     ap.add_argument("--no-e2e", action="store_true")

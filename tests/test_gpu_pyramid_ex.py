@@ -354,3 +354,31 @@ def test_rejected_row_whose_residual_vanishes_in_single_precision_still_draws(ps
         assert torch.equal(a[k], b[k]), k
     assert a["n_window"].tolist() == [1] * B and int(a["accept_len"].max()) <= 1
     assert psd.last_status() == 0
+
+
+def test_total_variation_through_every_schedule(psd, oracle, wl):
+    """div_kind = total variation (three ex2 per index pair: pass B needs max(p, q) only) in the two-stage call: every
+    schedule, row triples included, returns the same bits, and the per-row divergences are the oracle's."""
+    dev = torch.device("cuda:0")
+    B, K_d, K_q, V = 24, 6, 4, 32768
+    zd, zq, zt, tok = wl.make_pyramid_inputs(B, K_d, K_q, V, "bf16", seed=45, sigma_q=0.3, sigma_d=0.6)
+    dd = [t.to(dev) for t in (zd, zq, zt, tok)]
+    probe = psd.verify_ex(*dd, 1e9, 1e9, div_kind=psd.DIV_TV)
+    tau_q, tau_t = float(probe["div_q"].median()), float(probe["div_t"].median())
+    outs = []
+    for schedule in (psd.TWO_STAGE_FUSED, psd.TWO_STAGE_SEPARATE, psd.TWO_STAGE_FUSED_ROWS, psd.TWO_STAGE_AUTO):
+        outs.append(psd.verify_ex(*dd, tau_q, tau_t, psd.FUZZY, psd.FUZZY, 5, 9, div_kind=psd.DIV_TV, schedule=schedule))
+        torch.cuda.synchronize()
+        assert psd.last_status() == 0
+    for o in outs[1:]:
+        for k in ("accept_len_q", "next_token_q", "accept_len", "next_token", "window", "n_window", "div_q", "resid_q"):
+            assert torch.equal(bits(outs[0][k]), bits(o[k])), k
+    gpu = gpu_stage_to_numpy(outs[0])
+    o1 = oracle.verify_stage(host_bits(zd), host_bits(zq), tok.numpy(), np.float32(tau_q), 0, 5, 9, div_kind=1, n_threads=8)
+    orc = oracle.verify(host_bits(zd), host_bits(zq), host_bits(zt), tok.numpy(), np.float32(tau_q), np.float32(tau_t), 0, 5, 9,
+                        div_kind=1, n_threads=8)
+    assert np.abs(gpu["div_q"] - o1["div"]).max() <= TOL["bf16"]["val"]
+    assert np.abs(gpu["div_q"] - gpu["resid_q"]).max() == 0.0        # the total variation is the residual mass
+    same = (gpu["accept_len_q"] == orc["accept_len_q"]) & (gpu["next_token_q"] == orc["next_token_q"])
+    assert same.sum() >= B - 2 and np.array_equal(gpu["accept_len"][same], orc["accept_len"][same])
+    assert 0 < orc["accept_len_q"].sum() < B * K_d
