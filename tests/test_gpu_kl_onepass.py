@@ -178,3 +178,21 @@ def test_full_size_configs_with_kl_sampled(psd, oracle, wl, cfg):
         assert same.sum() >= len(ids) - 1
         assert np.array_equal(gpu["accept_len"][ids][same], orc["accept_len"][same])
     assert 0 < gpu["accept_len_q"].sum() < w.B * w.K_d
+
+
+def test_one_pass_draw_on_identical_rows(psd, oracle, wl):
+    """The one-pass record carries no residual mass; a rejected row whose two distributions are identical (residual
+    exactly zero) is found out by the draw itself, which then takes p_large as the oracle does."""
+    dev = torch.device("cuda:0")
+    B, K, V = 50, 3, 8192
+    zs, zl, tok = wl.make_stage_inputs(B, K, V, "f32", seed=91, sigma=0.5)
+    zl[::2] = zs[::2]                           # every other sequence: identical rows
+    d = [t.to(dev) for t in (zs, zl, tok)]
+    out = psd.verify_stage_ex(*d, -1.0, 0, 6, 2, div_kind=KL, want_resid=False)       # tau < 0: position 0 is rejected everywhere
+    torch.cuda.synchronize()
+    assert psd.last_status() == 0
+    gpu = gpu_stage_to_numpy(out)
+    orc = oracle.verify_stage(host_bits(zs), host_bits(zl), tok.numpy(), np.float32(-1.0), 0, 6, 2, div_kind=KL, n_threads=8)
+    assert np.all(gpu["accept_len"] == 0) and np.all(gpu["next_token"] >= 0) and np.all(gpu["div"][::2] == 0.0)
+    rep = compare_stage(oracle, gpu, orc, host_bits(zs), host_bits(zl), dtype="f32", mode=0, tau=-1.0, seed=6, offset=2, div_kind=KL)
+    assert rep["tie_cdf"] <= 1 and rep["tie_div"] == 0
