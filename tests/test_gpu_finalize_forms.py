@@ -172,6 +172,7 @@ def test_three_launch_form_on_two_streams_from_two_threads(psd, wl):
                 stream.synchronize()
                 if psd.last_status() != psd.OK:
                     errors.append((idx, "status"))
+            psd.release_stream(stream)      # the library keeps scratch for sixteen streams per device
         except Exception as e:   # noqa: BLE001
             errors.append((idx, repr(e)))
 
@@ -226,6 +227,8 @@ def test_three_launch_form_replayed_from_a_cuda_graph(psd, wl):
             torch.cuda.synchronize()
             for k in out:
                 assert torch.equal(out[k], e[k]), k
+        del g
+        psd.release_stream(side)            # the graph is gone: nothing uses the stream's scratch any more
     finally:
         psd.set_two_stage_policy(psd.TWO_STAGE_DEFAULT)
     assert psd.last_status() == 0
